@@ -1,0 +1,104 @@
+"""Shared test helpers: tensor <-> bit-pattern conversions and threshold calibration.
+
+The calibration lives here (under tests/) because it calls the CPU oracle; the
+product package never does.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import eta_oracle as orc
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    """bf16 / fp16 torch tensor -> uint16 bit patterns (numpy, same shape)."""
+    assert t.dtype in (torch.bfloat16, torch.float16)
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def bf16_bits_from_f64(x: np.ndarray) -> np.ndarray:
+    """Round doubles to bf16 (via torch) and return the bit patterns."""
+    return bits(torch.from_numpy(np.asarray(x, np.float64)).to(torch.float32).to(torch.bfloat16))
+
+
+def bf16_values(b: np.ndarray) -> np.ndarray:
+    """uint16 bf16 bit patterns -> float64 values."""
+    return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def fp16_values(b: np.ndarray) -> np.ndarray:
+    return b.view(np.float16).astype(np.float64)
+
+
+def random_cache(rng, B, Hkv, T, d, b, Tcap=None, scale=1.0):
+    Tcap = Tcap or ((T + b - 1) // b) * b
+    K = bf16_bits_from_f64(rng.standard_normal((B, Hkv, Tcap, d)) * scale)
+    V = bf16_bits_from_f64(rng.standard_normal((B, Hkv, Tcap, d)))
+    lens = np.full(B, T, np.int32)
+    return orc.Cache(K, V, lens, b)
+
+
+def cache_of(wl) -> orc.Cache:
+    """Oracle view of a generated workload."""
+    return orc.Cache(bits(wl.K), bits(wl.V), wl.seq_lens.numpy().astype(np.int32).copy(), wl.spec.block_size)
+
+
+def union_density(bound, tau, seq_lens, b, G):
+    """Fraction of full blocks admitted by at least one head of their GQA group (plain threshold, no rescue)."""
+    B, Hq, NBcap = bound.shape
+    adm = ~(bound < tau[:, :, None])                     # NaN (beyond NB) compares False -> masked below
+    tot = 0
+    hit = 0
+    for i in range(B):
+        NB = int(seq_lens[i]) // b
+        u = adm[i, :, :NB].reshape(Hq // G, G, NB).any(axis=1)
+        hit += int(u.sum())
+        tot += u.size
+    return hit / max(tot, 1)
+
+
+def calibrate_bias(bound, tau_raw, seq_lens, b, G, target_union_sparsity):
+    """Per-head predictor bias such that the union block sparsity hits a target.
+
+    bound: oracle bounds [B,Hq,NBcap]; tau_raw: q̄W without bias [B,Hq].
+    For a head-density level rho, bias_h(rho) = median_i(quantile_{1-rho}(bound[i,h]) - tau_raw[i,h]);
+    rho is bisected until the union density is 1 - target.  Stand-in for a trained predictor.
+    """
+    B, Hq, _ = bound.shape
+    srt = []
+    for i in range(B):
+        NB = int(seq_lens[i]) // b
+        srt.append(np.sort(bound[i, :, :NB], axis=1))
+
+    def bias_of(rho):
+        qs = np.empty((B, Hq))
+        for i in range(B):
+            NB = srt[i].shape[1]
+            k = min(NB - 1, max(0, int(np.floor((1.0 - rho) * NB))))
+            qs[i] = srt[i][:, k]
+        return np.median(qs - tau_raw, axis=0)
+
+    lo, hi = 0.0, 1.0
+    for _ in range(30):
+        mid = 0.5 * (lo + hi)
+        bias = bias_of(mid)
+        u = union_density(bound, tau_raw + bias[None, :], seq_lens, b, G)
+        if u > 1.0 - target_union_sparsity:
+            hi = mid
+        else:
+            lo = mid
+    return bias_of(0.5 * (lo + hi)).astype(np.float32)
+
+
+def calibrate_head_const(bound, seq_lens, b, sparsity_levels):
+    """Frozen per-head constants: c_h = median_i quantile_{level_h}(bound[i,h])."""
+    B, Hq, _ = bound.shape
+    qs = np.empty((B, Hq))
+    for i in range(B):
+        NB = int(seq_lens[i]) // b
+        s = np.sort(bound[i, :, :NB], axis=1)
+        for h in range(Hq):
+            k = min(NB - 1, max(0, int(np.floor(sparsity_levels[h] * NB))))
+            qs[i, h] = s[h, k]
+    return np.median(qs, axis=0).astype(np.float32)

@@ -1,0 +1,528 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests obtains its expectation from the oracle function under
+test: they use closed forms, numpy / scipy / torch library routines, brute
+force over tiny inputs, and invariants, chosen so that a dropped term, a wrong
+sign or index or a transposed operand fails at least one of them.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+from scipy.special import lambertw
+
+from oracle import eta_oracle as orc
+from tests.helpers import bf16_bits_from_f64, bf16_values, fp16_values, random_cache
+
+
+# --------------------------------------------------------------------------
+# storage formats
+# --------------------------------------------------------------------------
+
+def test_fp16_decode_matches_numpy_for_every_bit_pattern():
+    allbits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    ref = allbits.view(np.float16).astype(np.float64)
+    got = np.array([orc.fp16_to_double(int(b)) for b in allbits])
+    assert np.array_equal(np.isnan(ref), np.isnan(got))
+    m = ~np.isnan(ref)
+    assert np.array_equal(ref[m], got[m])
+
+
+def test_fp16_encode_is_single_round_to_nearest_even():
+    rng = np.random.default_rng(1)
+    xs = np.concatenate([
+        rng.standard_normal(4000) * 10.0 ** rng.integers(-9, 5, 4000),
+        np.array([0.0, -0.0, 65504.0, 65519.999, 65520.0, 1e9, -1e9, 2.0 ** -24, 2.0 ** -25, 2.0 ** -25 * 1.0001,
+                  2.0 ** -14, 2.0 ** -14 * (1 - 2.0 ** -12), np.inf, -np.inf]),
+    ])
+    # midpoints between neighbouring fp16 values must go to the even neighbour
+    h = rng.integers(0x0001, 0x7bfe, 500).astype(np.uint16)
+    lo = h.view(np.float16).astype(np.float64)
+    hi = (h + 1).astype(np.uint16).view(np.float16).astype(np.float64)
+    xs = np.concatenate([xs, 0.5 * (lo + hi)])
+    with np.errstate(over="ignore"):
+        ref = xs.astype(np.float16).view(np.uint16)      # numpy rounds float64 -> float16 directly, RNE
+    got = np.array([orc.double_to_fp16(float(x)) for x in xs], dtype=np.uint16)
+    assert np.array_equal(ref, got)
+
+
+def test_double_rounding_case_differs_from_rounding_through_float32():
+    # 1 + 2^-11 + 2^-30 lies just above the midpoint of two fp16 values: direct rounding goes up,
+    # rounding through binary32 first lands on the midpoint and then (ties-to-even) goes down.
+    x = 1.0 + 2.0 ** -11 + 2.0 ** -30
+    assert orc.double_to_fp16(x) == 0x3c01
+    assert np.float32(x).astype(np.float16).view(np.uint16) == 0x3c00
+
+
+def test_bf16_decode_matches_torch():
+    allbits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    ref = torch.from_numpy(allbits.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+    got = np.array([orc.bf16_to_double(int(b)) for b in allbits])
+    m = ~np.isnan(ref)
+    assert np.array_equal(np.isnan(ref), np.isnan(got))
+    assert np.array_equal(ref[m], got[m])
+
+
+# --------------------------------------------------------------------------
+# block summaries (Section 3: centroid, coordinate-wise population variance, max norm)
+# --------------------------------------------------------------------------
+
+def test_summaries_match_numpy_mean_std_norm():
+    rng = np.random.default_rng(2)
+    c = random_cache(rng, B=2, Hkv=3, T=5 * 32 + 7, d=16, b=32)
+    musig, mnorm, mu, sg, M = orc.block_summaries(c, raw=True)
+    Kv = bf16_values(c.K)
+    NB = c.seq_lens[0] // 32
+    assert NB == 5
+    blocks = Kv[:, :, :NB * 32].reshape(2, 3, NB, 32, 16)
+    np.testing.assert_allclose(mu[:, :, :NB], blocks.mean(axis=3), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(sg[:, :, :NB], blocks.std(axis=3), rtol=1e-13, atol=1e-14)   # ddof=0: population
+    np.testing.assert_allclose(M[:, :, :NB], np.linalg.norm(blocks, axis=4).max(axis=3), rtol=1e-14)
+    # storage rounding: fp16 for mu and sigma (sigma, not the variance), fp32 for M
+    assert np.array_equal(musig[:, :, :NB, 0].view(np.float16), mu[:, :, :NB].astype(np.float16))
+    assert np.array_equal(musig[:, :, :NB, 1].view(np.float16), sg[:, :, :NB].astype(np.float16))
+    assert np.array_equal(mnorm[:, :, :NB], M[:, :, :NB].astype(np.float32))
+    # the partial block past NB is not summarised
+    assert not musig[:, :, NB:].any() and not mnorm[:, :, NB:].any()
+
+
+def test_summaries_of_identical_keys():
+    d, b = 16, 8
+    k = np.linspace(-1.5, 2.0, d)
+    K = bf16_bits_from_f64(np.broadcast_to(k, (1, 1, b, d)).copy())
+    c = orc.Cache(K, K.copy(), np.array([b], np.int32), b)
+    _, _, mu, sg, M = orc.block_summaries(c, raw=True)
+    kv = bf16_values(K)[0, 0, 0]
+    np.testing.assert_allclose(mu[0, 0, 0], kv, atol=1e-15)
+    assert np.all(sg[0, 0, 0] == 0.0)
+    assert M[0, 0, 0] == pytest.approx(np.linalg.norm(kv), rel=1e-15)
+
+
+def test_summaries_of_axis_pairs_have_closed_form():
+    # keys mu0 +- s_c e_c (b = 2d): centroid mu0, variance_c = 2 s_c^2 / b, exactly diagonal covariance
+    d = 8
+    b = 2 * d
+    mu0 = np.array([0.5, -1.0, 0.25, 2.0, -0.75, 1.5, 0.0, -2.0])
+    s = np.array([0.5, 1.0, 0.25, 2.0, 0.125, 1.0, 0.5, 4.0])
+    keys = np.concatenate([mu0 + np.diag(s), mu0 - np.diag(s)])       # all exactly representable in bf16
+    K = bf16_bits_from_f64(keys.reshape(1, 1, b, d))
+    assert np.array_equal(bf16_values(K)[0, 0], keys)
+    c = orc.Cache(K, K.copy(), np.array([b], np.int32), b)
+    _, _, mu, sg, M = orc.block_summaries(c, raw=True)
+    np.testing.assert_allclose(mu[0, 0, 0], mu0, atol=1e-15)
+    np.testing.assert_allclose(sg[0, 0, 0] ** 2, 2 * s ** 2 / b, rtol=1e-14)
+    assert M[0, 0, 0] == pytest.approx(max(np.linalg.norm(keys, axis=1)), rel=1e-15)
+
+
+def test_summary_invariants_and_permutation():
+    rng = np.random.default_rng(3)
+    c = random_cache(rng, B=1, Hkv=2, T=4 * 64, d=32, b=64, scale=2.0)
+    _, _, mu, sg, M = orc.block_summaries(c, raw=True)
+    Kv = bf16_values(c.K).reshape(1, 2, 4, 64, 32)
+    # second formula for the variance: E[k^2] - mu^2
+    np.testing.assert_allclose(sg ** 2, (Kv ** 2).mean(axis=3) - mu ** 2, rtol=1e-10, atol=1e-12)
+    # the largest norm dominates the root mean square norm: M^2 >= |mu|^2 + sum sigma^2
+    assert np.all(M ** 2 >= (mu ** 2).sum(-1) + (sg ** 2).sum(-1) - 1e-12)
+    # permuting the tokens inside a block changes nothing
+    perm = rng.permutation(64)
+    Kp = c.K.reshape(1, 2, 4, 64, 32)[:, :, :, perm].reshape(c.K.shape).copy()
+    _, _, mu2, sg2, M2 = orc.block_summaries(orc.Cache(Kp, c.V, c.seq_lens, 64), raw=True)
+    np.testing.assert_allclose(mu2, mu, atol=1e-14)
+    np.testing.assert_allclose(sg2, sg, atol=1e-13)
+    np.testing.assert_array_equal(M2, M)
+
+
+def test_record_size_is_the_stated_overhead():
+    # compact layout: fp16[d] + fp16[d] + fp32 per block per KV head; 1.6% of the K,V bytes at b = 64
+    for d in (64, 128):
+        rec = 2 * d + 2 * d + 4
+        kv = 2 * 64 * d * 2
+        assert rec == 4 * d + 4
+        assert round(100.0 * rec / kv, 1) == 1.6
+
+
+def test_envelope_bounds_flat_sigma():
+    # sub-block envelope: sigma <= sigma~ <= sqrt(b/4) sigma, and equality with numpy's definition
+    rng = np.random.default_rng(4)
+    c = random_cache(rng, B=1, Hkv=1, T=3 * 64, d=16, b=64)
+    _, _, mu, sg, _ = orc.block_summaries(c, raw=True)
+    _, _, mu_e, sg_e, _ = orc.block_summaries(c, envelope=True, raw=True)
+    np.testing.assert_array_equal(mu, mu_e)
+    assert np.all(sg_e >= sg - 1e-14) and np.all(sg_e <= math.sqrt(64 / 4) * sg + 1e-14)
+    Kv = bf16_values(c.K).reshape(1, 1, 3, 16, 4, 16)
+    ref = np.sqrt(((Kv - mu[:, :, :, None, None, :]) ** 2).mean(axis=4)).max(axis=3)
+    np.testing.assert_allclose(sg_e, ref, rtol=1e-13)
+
+
+# --------------------------------------------------------------------------
+# threshold predictor (Eq. tau_pred)
+# --------------------------------------------------------------------------
+
+def test_predictor_is_head_major_concat_times_W_plus_bias():
+    rng = np.random.default_rng(5)
+    B, Hq, d = 3, 4, 8
+    q = bf16_bits_from_f64(rng.standard_normal((B, Hq, d)))
+    W = rng.standard_normal((Hq * d, Hq)).astype(np.float32)
+    bias = rng.standard_normal(Hq).astype(np.float32)
+    ref = bf16_values(q).reshape(B, Hq * d) @ W.astype(np.float64) + bias.astype(np.float64)
+    np.testing.assert_allclose(orc.predict_threshold(q, W, bias), ref, rtol=1e-13, atol=1e-13)
+    # start-dense initialisation: W = 0 gives tau = bias = -8 for every query
+    tau0 = orc.predict_threshold(q, np.zeros_like(W), np.full(Hq, -8.0, np.float32))
+    assert np.all(tau0 == -8.0)
+
+
+# --------------------------------------------------------------------------
+# Score_dual (Eq. dual_bound_eq)
+# --------------------------------------------------------------------------
+
+def _setup_bound(seed=6, B=2, Hq=4, Hkv=2, T=6 * 16, d=16, b=16, scale=1.0):
+    rng = np.random.default_rng(seed)
+    c = random_cache(rng, B, Hkv, T, d, b, scale=scale)
+    q = bf16_bits_from_f64(rng.standard_normal((B, Hq, d)))
+    musig, mnorm = orc.block_summaries(c)
+    return rng, c, q, musig, mnorm
+
+
+def test_bound_matches_formula_written_with_numpy():
+    _, c, q, musig, mnorm = _setup_bound()
+    z, s = 1.5, 1 / math.sqrt(16)
+    bound, g, sp = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, z, parts=True)
+    qv = bf16_values(q)                                     # [B,Hq,d]
+    mu = fp16_values(musig[:, :, :, 0])                     # [B,Hkv,NB,d]
+    sg = fp16_values(musig[:, :, :, 1])
+    G = 2
+    for h in range(4):
+        hk = h // G
+        dot = np.einsum("bd,bjd->bj", qv[:, h], mu[:, hk])
+        var = np.einsum("bd,bjd->bj", qv[:, h] ** 2, sg[:, hk] ** 2)
+        gg = s * (dot + z * np.sqrt(var))
+        ss = s * np.linalg.norm(qv[:, h], axis=-1)[:, None] * mnorm[:, hk].astype(np.float64)
+        np.testing.assert_allclose(g[:, h], gg, rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(sp[:, h], ss, rtol=1e-12)
+        np.testing.assert_allclose(bound[:, h], np.minimum(gg, ss), rtol=1e-12, atol=1e-13)
+
+
+def test_bound_homogeneity_monotone_in_z_and_centroid_logit_at_z0():
+    _, c, q, musig, mnorm = _setup_bound(seed=7)
+    b1 = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, 1.0)
+    # positive homogeneity: Score(2q) = 2 Score(q)  (2q is exact in bf16)
+    q2 = bf16_bits_from_f64(2.0 * bf16_values(q))
+    np.testing.assert_allclose(orc.score_dual(q2, musig, mnorm, c.seq_lens, 16, 1.0), 2 * b1, rtol=1e-13)
+    # monotone in z
+    b2 = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, 2.0)
+    assert np.all(b2 >= b1 - 1e-15)
+    # z = 0: the moment term is the centroid logit
+    _, g0, _ = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, 0.0, parts=True)
+    mu = fp16_values(musig[:, :, :, 0])
+    for h in range(4):
+        ref = np.einsum("bd,bjd->bj", bf16_values(q)[:, h], mu[:, h // 2]) / 4.0
+        np.testing.assert_allclose(g0[:, h], ref, rtol=1e-12, atol=1e-14)
+
+
+def test_sphere_term_is_sound_by_brute_force_and_identical_keys_are_tight():
+    _, c, q, musig, mnorm = _setup_bound(seed=8, scale=3.0)
+    _, _, sp = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, 1.0, parts=True)
+    true_max = orc.block_max_logit(q, c)
+    # Cauchy-Schwarz: s |q| M_B >= every logit of the block (fp32 rounding of M allowed for)
+    assert np.all(sp * (1 + 1e-6) >= true_max)
+    # brute-force cross-check of block_max_logit itself with numpy
+    Kv = bf16_values(c.K).reshape(2, 2, 6, 16, 16)
+    for h in range(4):
+        ref = np.einsum("bd,bjtd->bjt", bf16_values(q)[:, h], Kv[:, h // 2]).max(-1) / 4.0
+        np.testing.assert_allclose(true_max[:, h], ref, rtol=1e-12, atol=1e-13)
+    # a block of identical keys: both terms equal the true logit when q is parallel to k; moment term always
+    d, b = 16, 8
+    k = np.linspace(-1, 1, d)
+    K = bf16_bits_from_f64(np.broadcast_to(k, (1, 1, b, d)).copy())
+    kv = bf16_values(K)[0, 0, 0]
+    cc = orc.Cache(K, K.copy(), np.array([b], np.int32), b)
+    ms, mn = orc.block_summaries(cc)
+    assert np.array_equal(fp16_values(ms[0, 0, 0, 0]), kv)      # bf16 linspace values happen to be fp16-exact
+    qq = bf16_bits_from_f64(np.random.default_rng(0).standard_normal((1, 1, d)))
+    bound, g, sp2 = orc.score_dual(qq, ms, mn, cc.seq_lens, b, 3.0, parts=True)
+    logit = float(bf16_values(qq)[0, 0] @ kv) / 4.0
+    assert g[0, 0, 0] == pytest.approx(logit, rel=1e-12, abs=1e-14)
+    assert bound[0, 0, 0] == pytest.approx(logit, rel=1e-12, abs=1e-14)
+    assert sp2[0, 0, 0] >= logit
+
+
+def test_cantelli_count_and_diagonal_case():
+    # Finite-population Cantelli: #{k: <q,k> >= <q,mu> + z sqrt(q' Sigma q)} <= floor(b/(1+z^2)) with the
+    # FULL directional variance.  With exactly diagonal covariance the stored (diagonal) form is that bound,
+    # so for z > sqrt(b-1) the oracle's moment term is a certified maximum.
+    rng = np.random.default_rng(9)
+    d, b = 8, 16
+    for z in (0.5, 1.0, 2.0, 4.0):
+        for _ in range(50):
+            keys = rng.standard_normal((b, d)) @ rng.standard_normal((d, d))
+            q = rng.standard_normal(d)
+            mu = keys.mean(0)
+            Sigma = (keys - mu).T @ (keys - mu) / b
+            thr = q @ mu + z * math.sqrt(q @ Sigma @ q)
+            assert int((keys @ q >= thr).sum()) <= math.floor(b / (1 + z * z))
+    mu0 = np.array([0.5, -1.0, 0.25, 2.0, -0.75, 1.5, 0.0, -2.0])
+    s = np.array([0.5, 1.0, 0.25, 2.0, 0.125, 1.0, 0.5, 4.0])
+    keys = np.concatenate([mu0 + np.diag(s), mu0 - np.diag(s)])
+    K = bf16_bits_from_f64(keys.reshape(1, 1, b, d))
+    c = orc.Cache(K, K.copy(), np.array([b], np.int32), b)
+    ms, mn = orc.block_summaries(c)
+    zc = math.sqrt(b - 1) * 1.001
+    for _ in range(20):
+        q = bf16_bits_from_f64(rng.standard_normal((1, 1, d)))
+        _, g, _ = orc.score_dual(q, ms, mn, c.seq_lens, b, zc, parts=True)
+        assert g[0, 0, 0] * (1 + 1e-3) + 1e-6 >= orc.block_max_logit(q, c)[0, 0, 0]
+
+
+# --------------------------------------------------------------------------
+# selection (Algorithm 3: threshold, rescue; lwb pinning)
+# --------------------------------------------------------------------------
+
+def test_selection_extremes_nesting_offset_and_start_dense():
+    rng, c, q, musig, mnorm = _setup_bound(seed=10, B=2, Hq=4, Hkv=2, T=40 * 16 + 5, d=16, b=16)
+    NB = 40
+    bound = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, 1.0)
+    full = np.zeros((2, 2, c.NBcap), np.uint8)
+    full[:, :, :NB] = 0b11
+    # tau = -inf: every full block, every head
+    sel, resc = orc.select(bound, c.seq_lens, 16, 2, tau=np.full((2, 4), -np.inf))
+    assert np.array_equal(sel, full) and np.all(resc == -1)
+    # start-dense initialisation tau = -8 on N(0,1) data: 100% of blocks pass
+    sel8, _ = orc.select(bound, c.seq_lens, 16, 2, tau=np.full((2, 4), -8.0))
+    assert np.array_equal(sel8, full)
+    # tau = +inf: only the rescue block (first argmax of the window) and the lwb pinned blocks
+    sel, resc = orc.select(bound, c.seq_lens, 16, 2, tau=np.full((2, 4), np.inf), lwb=2, rescue_window=16)
+    for i in range(2):
+        for h in range(4):
+            expect = np.zeros(c.NBcap, bool)
+            expect[NB - 2:NB] = True
+            r = int(np.argmax(bound[i, h, :16]))            # np.argmax returns the first maximiser
+            expect[r] = True
+            assert resc[i, h] == r
+            assert np.array_equal(((sel[i, h // 2] >> (h % 2)) & 1).astype(bool), expect)
+    # a pinned block inside the window counts as attended: no rescue then
+    sel, resc = orc.select(bound, c.seq_lens, 16, 2, tau=np.full((2, 4), np.inf), lwb=2, rescue_window=1 << 30)
+    assert np.all(resc == -1)
+    assert np.all(sel[:, :, :NB - 2] == 0) and np.all(sel[:, :, NB - 2:NB] == 0b11)
+    # nesting: a higher threshold admits a subset (rescue aside)
+    t1 = rng.standard_normal((2, 4)).astype(np.float32) * 0.3 + 1.0
+    s1, _ = orc.select(bound, c.seq_lens, 16, 2, tau=t1, rescue_window=1)
+    s2, _ = orc.select(bound, c.seq_lens, 16, 2, tau=t1 + 0.5, rescue_window=1)
+    assert np.all((s2[:, :, 1:] & ~s1[:, :, 1:]) == 0)
+    assert 0 < (s2 != 0).sum() < (s1 != 0).sum() < full.astype(bool).sum()
+    # plain definition with numpy for the thresholded part
+    for h in range(4):
+        ref = ~(bound[:, h, 1:NB] < t1[:, h:h + 1].astype(np.float64))
+        assert np.array_equal(((s1[:, h // 2, 1:NB] >> (h % 2)) & 1).astype(bool), ref)
+    # operating offset: sel(tau, a) = sel(tau - a, 0)   (0.25 keeps the float32 subtraction exact enough)
+    ta = np.round(t1 * 4) / 4
+    sa, _ = orc.select(bound, c.seq_lens, 16, 2, tau=ta, a=0.25)
+    sb, _ = orc.select(bound, c.seq_lens, 16, 2, tau=ta - 0.25, a=0.0)
+    assert np.array_equal(sa, sb)
+    # frozen constants are per query head and independent of the sequence
+    cst = np.array([0.5, 1.0, 1.5, 2.0], np.float32)
+    sc, _ = orc.select(bound, c.seq_lens, 16, 2, head_const=cst)
+    st, _ = orc.select(bound, c.seq_lens, 16, 2, tau=np.broadcast_to(cst, (2, 4)).copy())
+    assert np.array_equal(sc, st)
+
+
+def test_rescue_tie_goes_to_lowest_index_and_equal_bound_is_admitted():
+    bound = np.array([[[1.0, 3.0, 3.0, 2.0]]])
+    lens = np.array([4 * 8], np.int32)
+    sel, resc = orc.select(bound, lens, 8, 1, tau=np.array([[5.0]]))
+    assert resc[0, 0] == 1 and sel[0, 0].tolist() == [0, 1, 0, 0]
+    # bound == tau_eff is admitted ("bypassed" needs a strict <)
+    sel, resc = orc.select(bound, lens, 8, 1, tau=np.array([[3.0]]))
+    assert sel[0, 0].tolist() == [0, 1, 1, 0] and resc[0, 0] == -1
+    # a NaN bound is admitted (not below the threshold)
+    bn = np.array([[[1.0, np.nan, 0.0, 0.0]]])
+    sel, _ = orc.select(bn, lens, 8, 1, tau=np.array([[5.0]]))
+    assert sel[0, 0].tolist() == [0, 1, 0, 0]
+    # rescue looks only inside its window
+    sel, resc = orc.select(bound, lens, 8, 1, tau=np.array([[5.0]]), rescue_window=1)
+    assert resc[0, 0] == 0 and sel[0, 0].tolist() == [1, 0, 0, 0]
+
+
+# --------------------------------------------------------------------------
+# the shifted-SiLU gate (Section 2.2 closed forms)
+# --------------------------------------------------------------------------
+
+def test_gate_closed_forms():
+    beta, tau = 5.0, 2.81
+    f = lambda S: orc.gate(S, tau, beta)
+    # value at the threshold is tau/2 and the slope there is (1 + beta tau / 2) / 2
+    assert f(tau) == pytest.approx(tau / 2, rel=1e-15)
+    h = 1e-6
+    assert (f(tau + h) - f(tau - h)) / (2 * h) == pytest.approx(0.5 * (1 + beta * tau / 2), rel=1e-8)
+    # unique minimiser S* = -(1 + W0(e^{-1-beta tau}))/beta with value -W0(.)/beta, and -1.28/beta < S* < -1/beta
+    w = float(lambertw(math.exp(-1 - beta * tau)).real)
+    s_star = -(1 + w) / beta
+    grid = np.linspace(-3, 3, 600001)
+    vals = np.array([f(x) for x in grid[::50]])
+    assert abs(grid[::50][vals.argmin()] - s_star) < 1e-3
+    assert f(s_star) == pytest.approx(-w / beta, rel=1e-9)
+    assert -1.28 / beta < s_star < -1 / beta
+    assert (f(s_star + h) - f(s_star - h)) / (2 * h) == pytest.approx(0.0, abs=1e-8)
+    # regime 1 (tau << -2/beta): the gate is the identity on the support of the scores
+    assert orc.gate(1.3, -8.0, 1.0) == pytest.approx(1.3 / (1 + math.exp(-9.3)), rel=1e-15)
+    # sigma'(8) = 3.35e-4: the low-gradient regime of the start-dense initialisation
+    sg8 = orc.gate(1.0, 1.0 - 8.0, 1.0)                  # = sigmoid(8)
+    assert sg8 * (1 - sg8) == pytest.approx(3.35e-4, rel=2e-3)
+    # limits
+    assert orc.gate(0.7, -math.inf, 5.0) == 0.7
+    assert orc.gate(0.7, math.inf, 5.0) == 0.0
+    assert orc.gate(-3.0, math.inf, 5.0) == 0.0
+    assert orc.gate(0.7, 123.0, 0.0) == 0.35
+
+
+# --------------------------------------------------------------------------
+# gated attention over admitted blocks
+# --------------------------------------------------------------------------
+
+def _attn_case(seed=11, B=2, Hq=4, Hkv=2, T=5 * 16 + 9, d=16, b=16):
+    rng = np.random.default_rng(seed)
+    c = random_cache(rng, B, Hkv, T, d, b)
+    q = bf16_bits_from_f64(rng.standard_normal((B, Hq, d)) * 1.5)
+    return rng, c, q
+
+
+def test_minus_infinite_threshold_is_textbook_softmax_attention():
+    _, c, q = _attn_case()
+    B, Hq, d, T = 2, 4, 16, int(c.seq_lens[0])
+    full = np.full((B, 2, c.NBcap), 0b11, np.uint8)
+    out = orc.gated_block_attention(q, c, full, tau=np.full((B, Hq), -np.inf), beta=5.0)
+    # library routine: torch scaled_dot_product_attention in float64 with GQA heads expanded
+    qt = torch.from_numpy(bf16_values(q))[:, :, None, :]
+    Kt = torch.from_numpy(bf16_values(c.K))[:, :, :T].repeat_interleave(2, dim=1)
+    Vt = torch.from_numpy(bf16_values(c.V))[:, :, :T].repeat_interleave(2, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, Kt, Vt)[:, :, 0].numpy()
+    np.testing.assert_allclose(out, ref, rtol=1e-11, atol=1e-13)
+    # and the oracle's own, separately written, dense routine agrees with the library too
+    np.testing.assert_allclose(orc.dense_softmax_attention(q, c), ref, rtol=1e-11, atol=1e-13)
+
+
+def test_plus_infinite_threshold_is_the_mean_of_loaded_values_and_beta0_is_half_scale():
+    _, c, q = _attn_case(seed=12)
+    B, Hq, T = 2, 4, int(c.seq_lens[0])
+    sel = np.zeros((B, 2, c.NBcap), np.uint8)
+    sel[:, :, 1] = 0b01                                    # head 0 of each group: block 1
+    sel[:, :, 3] = 0b11                                    # both heads: block 3
+    out, logZ, ntok = orc.gated_block_attention(q, c, sel, tau=np.full((B, Hq), np.inf), extras=True)
+    Vv = bf16_values(c.V)
+    tail = list(range(5 * 16, T))
+    for h in range(Hq):
+        toks = (list(range(16, 32)) if h % 2 == 0 else []) + list(range(48, 64)) + tail
+        np.testing.assert_allclose(out[:, h], Vv[:, h // 2][:, toks].mean(axis=1), rtol=1e-12, atol=1e-14)
+        assert np.all(ntok[:, h] == len(toks))
+        np.testing.assert_allclose(logZ[:, h], math.log(len(toks)), rtol=1e-13)
+    # beta = 0: S~ = S/2, i.e. softmax attention at half the scale, for any finite tau
+    full = np.full((B, 2, c.NBcap), 0b11, np.uint8)
+    o0 = orc.gated_block_attention(q, c, full, tau=np.full((B, Hq), 0.37), beta=0.0)
+    np.testing.assert_allclose(o0, orc.dense_softmax_attention(q, c, scale=0.5 / 4.0), rtol=1e-11, atol=1e-13)
+
+
+def test_general_case_against_per_token_brute_force_and_sibling_blocks_are_not_attended():
+    rng, c, q = _attn_case(seed=13)
+    B, Hq, d, b, T = 2, 4, 16, 16, int(c.seq_lens[0])
+    NB = T // b
+    sel = rng.integers(0, 4, size=(B, 2, c.NBcap)).astype(np.uint8)
+    sel[:, :, 0] |= 1
+    tau = rng.standard_normal((B, Hq)).astype(np.float32)
+    a, beta = 0.25, 3.0
+    out, logZ, ntok = orc.gated_block_attention(q, c, sel, tau=tau, a=a, beta=beta, extras=True)
+    qv, Kv, Vv = bf16_values(q), bf16_values(c.K), bf16_values(c.V)
+    for i in range(B):
+        for h in range(Hq):
+            te = float(tau[i, h]) - a
+            num = np.zeros(d)
+            den = 0.0
+            n = 0
+            for p in range(T):
+                j = p // b
+                if j < NB and not (sel[i, h // 2, j] >> (h % 2)) & 1:
+                    continue
+                S = float(qv[i, h] @ Kv[i, h // 2, p]) / math.sqrt(d)
+                St = S / (1.0 + math.exp(-beta * (S - te)))
+                w = math.exp(St)
+                num += w * Vv[i, h // 2, p]
+                den += w
+                n += 1
+            np.testing.assert_allclose(out[i, h], num / den, rtol=1e-11, atol=1e-13)
+            assert logZ[i, h] == pytest.approx(math.log(den), rel=1e-12)
+            assert ntok[i, h] == n
+
+
+def test_exact_output_decomposition_and_skipped_mass_bound():
+    # Z_all o_train = Z_load o_block + Z_D v_D  (exact), hence
+    # |o_train - o_block| <= (Z_D / Z_all) max_{s in D} |v_s - o_block|.
+    rng, c, q = _attn_case(seed=14, T=8 * 16 + 3)
+    B, Hq, b, T = 2, 4, 16, int(c.seq_lens[0])
+    NB = T // b
+    musig, mnorm = orc.block_summaries(c)
+    tau = np.full((B, Hq), 0.9, np.float32)
+    res = orc.decode_step(q, c, musig, mnorm, tau=tau, z=1.0, beta=5.0, rescue_window=4)
+    sel = res["sel"]
+    assert 0 < sum(bin(int(x)).count("1") for x in sel.ravel()) < B * Hq * NB   # genuinely sparse
+    full = np.full_like(sel, 0b11)
+    o_train, lz_all, _ = orc.gated_block_attention(q, c, full, tau=tau, extras=True)
+    o_block, lz_load, _ = orc.gated_block_attention(q, c, sel, tau=tau, extras=True)
+    # the dropped set alone: complement of the mask; its tail tokens must not be counted twice, so
+    # compute Z_D and v_D directly
+    qv, Kv, Vv = bf16_values(q), bf16_values(c.K), bf16_values(c.V)
+    for i in range(B):
+        for h in range(Hq):
+            ZD, vD, worst = 0.0, np.zeros(16), 0.0
+            for p in range(NB * b):
+                if (sel[i, h // 2, p // b] >> (h % 2)) & 1:
+                    continue
+                S = float(qv[i, h] @ Kv[i, h // 2, p]) / 4.0
+                w = math.exp(orc.gate(S, float(np.float32(0.9)), 5.0))   # tau travels as float32
+                ZD += w
+                vD += w * Vv[i, h // 2, p]
+                worst = max(worst, float(np.linalg.norm(Vv[i, h // 2, p] - o_block[i, h])))
+            Zall, Zload = math.exp(lz_all[i, h]), math.exp(lz_load[i, h])
+            assert Zall == pytest.approx(Zload + ZD, rel=1e-12)
+            np.testing.assert_allclose(Zall * o_train[i, h], Zload * o_block[i, h] + vD, rtol=1e-10, atol=1e-12)
+            assert np.linalg.norm(o_train[i, h] - o_block[i, h]) <= (ZD / Zall) * worst + 1e-12
+
+
+def test_screening_soundness_where_the_paper_certifies_it():
+    # With z huge the bound is the sphere term alone (exact Cauchy-Schwarz): every skipped block's true
+    # maximum logit lies below tau_eff, by brute force; and then each skipped key weighs at most
+    # max(1, exp(tau_eff/2)), so Z_D <= |D| max(1, exp(tau_eff/2)).
+    rng = np.random.default_rng(15)
+    c = random_cache(rng, 1, 2, 24 * 8, 8, 8)
+    # spread the key norms so that the sphere term separates blocks
+    Kv = bf16_values(c.K) * np.repeat(rng.uniform(0.2, 2.0, (1, 2, 24)), 8, axis=2)[..., None]
+    c = orc.Cache(bf16_bits_from_f64(Kv), c.V, c.seq_lens, 8)
+    q = bf16_bits_from_f64(rng.standard_normal((1, 4, 8)))
+    musig, mnorm = orc.block_summaries(c)
+    bound, g, sp = orc.score_dual(q, musig, mnorm, c.seq_lens, 8, 1e6, parts=True)
+    np.testing.assert_array_equal(bound, sp)
+    tau = np.quantile(bound[0], 0.6, axis=1)[None, :].astype(np.float32)
+    sel, _ = orc.select(bound, c.seq_lens, 8, 2, tau=tau, rescue_window=1)
+    true_max = orc.block_max_logit(q, c)
+    skipped = 0
+    for h in range(4):
+        for j in range(24):
+            if not (sel[0, h // 2, j] >> (h % 2)) & 1:
+                skipped += 1
+                assert true_max[0, h, j] < float(tau[0, h])
+    assert skipped > 20
+    o_all, lz_all, _ = orc.gated_block_attention(q, c, np.full_like(sel, 3), tau=tau, extras=True)
+    o_blk, lz_blk, n_blk = orc.gated_block_attention(q, c, sel, tau=tau, extras=True)
+    for h in range(4):
+        ZD = math.exp(lz_all[0, h]) - math.exp(lz_blk[0, h])
+        nD = 24 * 8 - int(n_blk[0, h])
+        assert ZD <= nD * max(1.0, math.exp(float(tau[0, h]) / 2)) * (1 + 1e-9)
+
+
+def test_decode_step_composes_the_three_stages():
+    rng, c, q = _attn_case(seed=16, T=12 * 16 + 4)
+    musig, mnorm = orc.block_summaries(c)
+    tau = np.full((2, 4), 0.8, np.float32)
+    res = orc.decode_step(q, c, musig, mnorm, tau=tau, z=1.0, lwb=2, rescue_window=8)
+    bound = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, 1.0)
+    sel, _ = orc.select(bound, c.seq_lens, 16, 2, tau=tau, lwb=2, rescue_window=8)
+    assert np.array_equal(res["sel"], sel)
+    np.testing.assert_array_equal(res["out"], orc.gated_block_attention(q, c, sel, tau=tau))
