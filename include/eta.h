@@ -1,0 +1,175 @@
+/*
+ * eta.h - C ABI of the B200 (sm_100a) block-sparse decode attention of
+ * Elastic Threshold Attention (ETA).
+ *
+ * The library covers the inference path of the paper: the dual
+ * probabilistic-geometric block index (Section 3), the linear threshold
+ * predictor (Eq. tau_pred), O(1)-per-block screening with Score_dual
+ * (Eq. dual_bound_eq), and SiLU-gated attention over the surviving blocks with
+ * top-1 rescue and tail handling (Algorithm 3), plus the frozen per-head
+ * constant-threshold mode (Section 4.5, "Distilling static thresholds").
+ *
+ * Conventions that hold for every call unless stated otherwise:
+ *   - Descriptors (eta_cache_desc, eta_params) are HOST structs read during the
+ *     call.  Every other pointer is a DEVICE pointer owned by the caller.
+ *   - The library allocates no device memory, never synchronises and never
+ *     copies to the host.  All work is enqueued on `stream` (a cudaStream_t
+ *     passed as void*; NULL is the default stream).
+ *   - Return value: ETA_OK (0) or a negative eta_status.  No exception crosses
+ *     the boundary.  Problems only the device can see (a sequence longer than
+ *     the cache, a bounded wait that gave up) are OR-ed into *status_dev.
+ *   - Layouts (d = head_dim, b = block_size, G = n_q_heads / n_kv_heads;
+ *     query head h belongs to KV head h / G):
+ *       K, V     bf16, element (i, hk, t, c) at i*stride_b + hk*stride_h + t*stride_t + c
+ *                (strides in elements, stride_t a multiple of 8, base 16-byte aligned)
+ *       q        bf16 [batch, n_q_heads, d], contiguous
+ *       seq_lens int32 [batch]: tokens valid in the cache of each sequence
+ *       musig    fp16 [batch, n_kv_heads, nb_cap, 2, d]: centroid, then coordinate-wise
+ *                standard deviation (sigma, not the variance) of every full block
+ *       mnorm    fp32 [batch, n_kv_heads, nb_cap]: largest key norm of every full block
+ *       tau      fp32 [batch, n_q_heads];  head_const fp32 [n_q_heads]
+ *       out      fp32 [batch, n_q_heads, d]
+ *       sel_mask uint8 [batch, n_kv_heads, nb_cap]: bit g set iff query head hk*G+g attends
+ *                full block j.  Tokens past the last full block are always attended.
+ *   - Supported shapes: head_dim in {64, 128}; block_size in {32, 64, 128};
+ *     G in {1, 2, 4, 8}.  Anything else returns ETA_ERR_UNSUPPORTED.
+ */
+#ifndef ETA_H_
+#define ETA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum eta_status {
+    ETA_OK = 0,
+    ETA_ERR_INVALID_ARG = -1,   /* NULL pointer, inconsistent sizes, both or neither of tau / head_const */
+    ETA_ERR_UNSUPPORTED = -2,   /* shape or alignment outside the supported set */
+    ETA_ERR_WORKSPACE = -3,     /* workspace missing, misaligned (256 B) or too small */
+    ETA_ERR_CUDA = -4           /* a CUDA call failed; see eta_last_cuda_error() */
+} eta_status;
+
+/* bits written to *status_dev by the kernels */
+#define ETA_DEV_TIMEOUT      1u  /* a bounded wait inside a kernel ran out; outputs are not valid */
+#define ETA_DEV_LEN_CLAMPED  2u  /* some seq_lens[i] exceeded t_cap and was clamped */
+#define ETA_DEV_EMPTY_ROW    4u  /* some seq_lens[i] <= 0: that sequence's output is zero */
+
+/* flags of eta_params.flags */
+#define ETA_FLAG_DENSE           1u  /* baseline: admit every block and switch the gate off (softmax attention) */
+/* flags of the summary builders */
+#define ETA_BUILD_SIGMA_ENVELOPE 1u  /* store the sub-block envelope (Eq. subblock_envelope_appx) instead of sigma */
+
+typedef struct eta_cache_desc {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim, block_size;
+    int32_t t_cap;                              /* token capacity of the cache along t */
+    int32_t nb_cap;                             /* block capacity of musig / mnorm / sel_mask (>= t_cap / block_size) */
+    int64_t k_stride_b, k_stride_h, k_stride_t; /* elements */
+    int64_t v_stride_b, v_stride_h, v_stride_t; /* elements */
+} eta_cache_desc;
+
+typedef struct eta_params {
+    float z;                /* z-score of the moment term of Score_dual */
+    float a;                /* operating offset: tau_eff = tau - a (Algorithm 3) */
+    float beta;             /* gate temperature of Eq. soft_mask at inference */
+    float scale;            /* softmax scale s; <= 0 selects 1/sqrt(head_dim) */
+    int32_t lwb;            /* the last `lwb` full blocks are always attended */
+    int32_t rescue_window;  /* top-1 rescue looks at the first min(rescue_window, NB) blocks; >= 1 */
+    uint32_t flags;         /* ETA_FLAG_* */
+    int32_t ctas_per_sm;    /* launch hint for the streaming kernel: 0 = library default */
+} eta_params;
+
+/*
+ * Bytes of scratch eta_decode needs for this cache shape (independent of the
+ * sequence lengths).  The caller allocates it once, 256-byte aligned, and may
+ * reuse it across calls on the same stream.  No device is touched.
+ */
+int eta_workspace_bytes(const eta_cache_desc* desc, size_t* out_bytes);
+
+/*
+ * Section 3 (dual block index); appendix "End-to-end systems accounting"
+ * (prefill indexing: one pass over K).  For every sequence i, KV head hk and
+ * full block j < floor(seq_lens[i] / b) writes
+ *   mu = mean of the b keys, sigma_c = sqrt(mean_k (k_c - mu_c)^2) (population),
+ *   M = max_k ||k||_2
+ * as fp16 / fp16 / fp32.  Records of blocks that are not full are left untouched.
+ * Arithmetic is fp32 on the bf16 keys, two passes (mean first, then deviations).
+ * flags: ETA_BUILD_SIGMA_ENVELOPE stores max over 4-token sub-blocks of the
+ * sub-block RMS deviation from mu instead of sigma.
+ */
+int eta_build_block_summaries(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens,
+                              void* musig, float* mnorm, uint32_t flags, void* stream);
+
+/*
+ * Appendix "End-to-end systems accounting" (tail-block metadata update at every
+ * decode step).  Call after a token has been appended and seq_lens[i] bumped:
+ * for every sequence whose new length is a positive multiple of b, the block
+ * that just became full (index seq_lens[i]/b - 1) is summarised exactly as
+ * eta_build_block_summaries would; other sequences are untouched.  Stateless and
+ * idempotent.
+ */
+int eta_append_summary(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens_after,
+                       void* musig, float* mnorm, uint32_t flags, void* stream);
+
+/*
+ * Eq. tau_pred: tau[i, h] = sum_r qbar[i, r] * W[r, h] + bias[h], with qbar the
+ * head-major concatenation of the n_q_heads post-RoPE query vectors of sequence
+ * i (length n_q_heads * head_dim).  q bf16 [batch, n_q_heads, head_dim];
+ * W fp32 [n_q_heads * head_dim, n_q_heads] row-major; bias fp32 [n_q_heads];
+ * tau fp32 [batch, n_q_heads].  fp32 accumulation in a fixed order.
+ */
+int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t head_dim, const void* q,
+                          const float* W, const float* bias, float* tau, void* stream);
+
+/*
+ * Eq. dual_bound_eq, evaluated for every (sequence, query head, full block):
+ *   bound = s * min( <q, mu> + z * sqrt(sum_c q_c^2 sigma_c^2), ||q|| * M ).
+ * bound fp32 [batch, n_q_heads, nb_cap]; entries of blocks that are not full are
+ * left untouched.  Same arithmetic as the screening stage of eta_decode; meant
+ * for diagnostics and for calibrating frozen constants, not for the hot loop.
+ */
+int eta_score_dual(const eta_cache_desc* desc, const eta_params* params, const void* q,
+                   const int32_t* seq_lens, const void* musig, const float* mnorm,
+                   float* bound, void* stream);
+
+/*
+ * Algorithm 3 (screen, top-1 rescue, tail phase, chunk merge) with the
+ * GQA-grouped execution of the fused-kernel appendix, for one decode query per
+ * sequence.  Per query head h, with tau_eff = (tau[i,h] or head_const[h]) - a:
+ *   1. every full block j is admitted unless Score_dual(q_h, j) < tau_eff; the last
+ *      `lwb` full blocks are always admitted; if none of the first
+ *      min(rescue_window, NB) blocks is admitted the first one with the largest
+ *      bound among them is;
+ *   2. a block is read from HBM once per KV head if any head of the group admits it;
+ *   3. the head attends the tokens of its own admitted blocks and all tokens past
+ *      the last full block, with weights exp(S~), S~ = S * sigmoid(beta * (S - tau_eff)),
+ *      S = s <q_h, k>; out = sum w v / sum w.
+ * Exactly one of tau / head_const must be non-NULL (frozen mode = head_const).
+ * sel_mask (required) receives the per-head admission bits; stats (nullable,
+ * int32 [batch, n_kv_heads]) the number of blocks fetched per KV head;
+ * status_dev (nullable, uint32, caller-zeroed) device-side problems.
+ * bf16 operands, fp32 scores / softmax statistics / accumulators; deterministic
+ * for a given device and launch hint.  workspace: eta_workspace_bytes() bytes.
+ */
+int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q,
+               const void* K, const void* V, const int32_t* seq_lens,
+               const void* musig, const float* mnorm,
+               const float* tau, const float* head_const,
+               float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev,
+               void* workspace, size_t workspace_bytes, void* stream);
+
+/* Number of kernels one eta_decode call launches (for launch accounting). */
+int eta_decode_kernel_count(void);
+
+/* Text for an eta_status. */
+const char* eta_strerror(int code);
+
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char* eta_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ETA_H_ */

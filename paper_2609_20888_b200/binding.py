@@ -1,0 +1,197 @@
+"""Thin ctypes binding of the C-ABI library (`include/eta.h`).
+
+Argument marshalling only: torch tensors provide device memory and the current
+CUDA stream; every step of the path runs in the library's kernels.  There is no
+CPU fallback: a missing library or a CPU tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libeta_b200.so")
+
+ETA_FLAG_DENSE = 1
+ETA_BUILD_SIGMA_ENVELOPE = 1
+ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
+
+EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
+           "eta_score_dual", "eta_decode", "eta_decode_kernel_count", "eta_strerror", "eta_last_cuda_error")
+
+
+class CacheDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("block_size", ctypes.c_int32), ("t_cap", ctypes.c_int32),
+                ("nb_cap", ctypes.c_int32),
+                ("k_stride_b", ctypes.c_int64), ("k_stride_h", ctypes.c_int64), ("k_stride_t", ctypes.c_int64),
+                ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_t", ctypes.c_int64)]
+
+
+class Params(ctypes.Structure):
+    _fields_ = [("z", ctypes.c_float), ("a", ctypes.c_float), ("beta", ctypes.c_float), ("scale", ctypes.c_float),
+                ("lwb", ctypes.c_int32), ("rescue_window", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("ctas_per_sm", ctypes.c_int32)]
+
+
+class EtaError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load the in-tree library; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise EtaError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_20888_b200.build` "
+                           "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+        D, P = ctypes.POINTER(CacheDesc), ctypes.POINTER(Params)
+        lib.eta_workspace_bytes.argtypes = [D, ctypes.POINTER(ctypes.c_size_t)]
+        lib.eta_build_block_summaries.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
+        lib.eta_append_summary.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
+        lib.eta_predict_threshold.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, f32p, f32p, f32p, vp]
+        lib.eta_score_dual.argtypes = [D, P, vp, i32p, vp, f32p, f32p, vp]
+        lib.eta_decode.argtypes = [D, P, vp, vp, vp, i32p, vp, f32p, f32p, f32p, f32p, vp, i32p, vp, vp,
+                                   ctypes.c_size_t, vp]
+        lib.eta_decode_kernel_count.restype = ctypes.c_int
+        lib.eta_strerror.restype = ctypes.c_char_p
+        lib.eta_strerror.argtypes = [ctypes.c_int]
+        lib.eta_last_cuda_error.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name not in ("eta_strerror", "eta_last_cuda_error", "eta_decode_kernel_count"):
+                getattr(lib, name).restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        lib = load()
+        raise EtaError(f"{what}: {lib.eta_strerror(rc).decode()} ({rc}) {lib.eta_last_cuda_error().decode()}")
+
+
+def _dev(t: torch.Tensor | None, dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise EtaError(f"{name} must be a CUDA tensor (no CPU path exists)")
+    if dtype is not None and t.dtype != dtype:
+        raise EtaError(f"{name} must be {dtype}, got {t.dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+@dataclass
+class DecodeParams:
+    z: float = 1.0
+    a: float = 0.0
+    beta: float = 5.0
+    scale: float = 0.0
+    lwb: int = 0
+    rescue_window: int = 128
+    flags: int = 0
+    ctas_per_sm: int = 0
+
+    def c(self) -> Params:
+        return Params(self.z, self.a, self.beta, self.scale, self.lwb, self.rescue_window, self.flags,
+                      self.ctas_per_sm)
+
+
+def cache_desc(K: torch.Tensor, V: torch.Tensor, n_q_heads: int, block_size: int, nb_cap: int | None = None) -> CacheDesc:
+    """Describe a cache K, V of logical shape [batch, n_kv_heads, t_cap, head_dim] (any strides with unit
+    stride along head_dim)."""
+    B, Hkv, Tcap, d = K.shape
+    if K.stride(3) != 1 or V.stride(3) != 1 or V.shape != K.shape:
+        raise EtaError("K and V must have the same shape and unit stride along head_dim")
+    nb = nb_cap if nb_cap is not None else (Tcap + block_size - 1) // block_size
+    return CacheDesc(B, n_q_heads, Hkv, d, block_size, Tcap, nb, K.stride(0), K.stride(1), K.stride(2),
+                     V.stride(0), V.stride(1), V.stride(2))
+
+
+def eta_workspace_bytes(desc: CacheDesc) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load().eta_workspace_bytes(ctypes.byref(desc), ctypes.byref(n)), "eta_workspace_bytes")
+    return n.value
+
+
+def alloc_summaries(desc: CacheDesc, device):
+    musig = torch.zeros((desc.batch, desc.n_kv_heads, desc.nb_cap, 2, desc.head_dim), dtype=torch.float16, device=device)
+    mnorm = torch.zeros((desc.batch, desc.n_kv_heads, desc.nb_cap), dtype=torch.float32, device=device)
+    return musig, mnorm
+
+
+def eta_build_block_summaries(desc, K, seq_lens, musig, mnorm, flags: int = 0) -> None:
+    _check(load().eta_build_block_summaries(ctypes.byref(desc), _dev(K, torch.bfloat16, "K"),
+                                            _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                            _dev(mnorm, torch.float32, "mnorm"), flags, _stream()),
+           "eta_build_block_summaries")
+
+
+def eta_append_summary(desc, K, seq_lens_after, musig, mnorm, flags: int = 0) -> None:
+    _check(load().eta_append_summary(ctypes.byref(desc), _dev(K, torch.bfloat16, "K"),
+                                     _dev(seq_lens_after, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                     _dev(mnorm, torch.float32, "mnorm"), flags, _stream()),
+           "eta_append_summary")
+
+
+def eta_predict_threshold(q, W, bias, tau) -> None:
+    B, Hq, d = q.shape
+    _check(load().eta_predict_threshold(B, Hq, d, _dev(q, torch.bfloat16, "q"), _dev(W, torch.float32, "W"),
+                                        _dev(bias, torch.float32, "bias"), _dev(tau, torch.float32, "tau"), _stream()),
+           "eta_predict_threshold")
+
+
+def eta_score_dual(desc, params: DecodeParams, q, seq_lens, musig, mnorm, bound) -> None:
+    p = params.c()
+    _check(load().eta_score_dual(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
+                                 _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                 _dev(mnorm, torch.float32, "mnorm"), _dev(bound, torch.float32, "bound"), _stream()),
+           "eta_score_dual")
+
+
+def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,
+               workspace, stats=None, status=None) -> None:
+    p = params.c()
+    _check(load().eta_decode(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
+                             _dev(K, torch.bfloat16, "K"), _dev(V, torch.bfloat16, "V"),
+                             _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                             _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
+                             _dev(head_const, torch.float32, "head_const"), _dev(out, torch.float32, "out"),
+                             _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),
+                             _dev(status, torch.int32, "status"), _dev(workspace, torch.uint8, "workspace"),
+                             workspace.numel(), _stream()),
+           "eta_decode")
+
+
+def eta_decode_kernel_count() -> int:
+    return load().eta_decode_kernel_count()
+
+
+class DecodeState:
+    """Device buffers one decode loop needs (allocated once with torch; the library allocates nothing)."""
+
+    def __init__(self, K: torch.Tensor, V: torch.Tensor, n_q_heads: int, block_size: int):
+        dev = K.device
+        self.desc = cache_desc(K, V, n_q_heads, block_size)
+        self.K, self.V = K, V
+        self.musig, self.mnorm = alloc_summaries(self.desc, dev)
+        self.workspace = torch.empty(eta_workspace_bytes(self.desc) + 256, dtype=torch.uint8, device=dev)
+        off = (-self.workspace.data_ptr()) % 256
+        self.workspace = self.workspace[off:off + eta_workspace_bytes(self.desc)]
+        B, Hkv, d = self.desc.batch, self.desc.n_kv_heads, self.desc.head_dim
+        self.out = torch.empty((B, n_q_heads, d), dtype=torch.float32, device=dev)
+        self.sel_mask = torch.zeros((B, Hkv, self.desc.nb_cap), dtype=torch.uint8, device=dev)
+        self.tau = torch.empty((B, n_q_heads), dtype=torch.float32, device=dev)
+        self.stats = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)

@@ -1,0 +1,81 @@
+// Host-side plumbing of the C ABI: status text, argument validation and the
+// scratch layout shared by the kernels of eta_decode.
+#include <stdio.h>
+#include <string.h>
+
+#include "eta_common.cuh"
+
+namespace eta {
+
+static thread_local char g_cuda_error[256] = "";
+
+void set_cuda_error(cudaError_t e, const char* where) {
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", where, cudaGetErrorString(e));
+}
+
+int validate_desc(const eta_cache_desc* d) {
+    if (!d) return ETA_ERR_INVALID_ARG;
+    if (d->batch <= 0 || d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->t_cap <= 0 || d->nb_cap <= 0)
+        return ETA_ERR_INVALID_ARG;
+    if (d->n_q_heads % d->n_kv_heads != 0) return ETA_ERR_INVALID_ARG;
+    int G = d->n_q_heads / d->n_kv_heads;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return ETA_ERR_UNSUPPORTED;
+    if (d->head_dim != 64 && d->head_dim != 128) return ETA_ERR_UNSUPPORTED;
+    if (d->block_size != 32 && d->block_size != 64 && d->block_size != 128) return ETA_ERR_UNSUPPORTED;
+    if ((int64_t)d->nb_cap * d->block_size < d->t_cap - d->block_size + 1) return ETA_ERR_INVALID_ARG;
+    if (d->nb_cap >= (1 << 24)) return ETA_ERR_UNSUPPORTED;   // block index shares a word with the head bits
+    if (d->k_stride_t % 8 || d->k_stride_h % 8 || d->k_stride_b % 8) return ETA_ERR_UNSUPPORTED;
+    if (d->v_stride_t % 8 || d->v_stride_h % 8 || d->v_stride_b % 8) return ETA_ERR_UNSUPPORTED;
+    if (d->k_stride_t < d->head_dim || d->v_stride_t < d->head_dim) return ETA_ERR_INVALID_ARG;
+    return ETA_OK;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+WsLayout ws_layout(const eta_cache_desc* d) {
+    WsLayout L;
+    int G = d->n_q_heads / d->n_kv_heads;
+    L.rows = d->batch * d->n_kv_heads;
+    L.nseg = (d->nb_cap + SEG - 1) / SEG;
+    L.entries = L.rows * (L.nseg + 1);
+    size_t off = 0;
+    L.hdr = off;        off = align_up(off + 8 * sizeof(int32_t), 256);
+    L.seg_count = off;  off = align_up(off + sizeof(int32_t) * (size_t)L.rows * L.nseg, 256);
+    L.seg_list = off;   off = align_up(off + sizeof(int32_t) * (size_t)L.rows * L.nseg * LSTRIDE, 256);
+    L.seg_resc = off;   off = align_up(off + sizeof(RescueRec) * (size_t)L.rows * L.nseg * G, 256);
+    L.pref = off;       off = align_up(off + sizeof(int32_t) * ((size_t)L.entries + 1), 256);
+    L.cta_start = off;  off = align_up(off + sizeof(int4) * (size_t)MAX_CTAS, 256);
+    L.tau_eff = off;    off = align_up(off + sizeof(float) * (size_t)d->batch * d->n_q_heads, 256);
+    size_t slots = (size_t)MAX_CTAS + L.rows;
+    L.part_ml = off;    off = align_up(off + sizeof(float2) * slots * G, 256);
+    L.part_o = off;     off = align_up(off + sizeof(float) * slots * G * d->head_dim, 256);
+    L.total = off;
+    return L;
+}
+
+}  // namespace eta
+
+extern "C" {
+
+int eta_workspace_bytes(const eta_cache_desc* desc, size_t* out_bytes) {
+    if (!out_bytes) return ETA_ERR_INVALID_ARG;
+    int rc = eta::validate_desc(desc);
+    if (rc != ETA_OK) return rc;
+    *out_bytes = eta::ws_layout(desc).total;
+    return ETA_OK;
+}
+
+const char* eta_strerror(int code) {
+    switch (code) {
+        case ETA_OK: return "ok";
+        case ETA_ERR_INVALID_ARG: return "invalid argument";
+        case ETA_ERR_UNSUPPORTED: return "unsupported shape or alignment";
+        case ETA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case ETA_ERR_CUDA: return "CUDA error (see eta_last_cuda_error)";
+        default: return "unknown status";
+    }
+}
+
+const char* eta_last_cuda_error(void) { return eta::g_cuda_error; }
+
+}  // extern "C"

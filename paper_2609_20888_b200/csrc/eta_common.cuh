@@ -1,0 +1,160 @@
+// Shared declarations of the ETA decode library: status plumbing, the scratch
+// layout every kernel of eta_decode agrees on, and thin wrappers over the PTX
+// the kernels use (mbarrier, bulk / tensor TMA copies, warp MMA).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/eta.h"
+
+namespace eta {
+
+// ---------------------------------------------------------------- host side
+void set_cuda_error(cudaError_t e, const char* where);
+inline int check_launch(const char* where) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e, where); return ETA_ERR_CUDA; }
+    return ETA_OK;
+}
+int validate_desc(const eta_cache_desc* d);
+
+// Screening works on segments of SEG consecutive block records of one
+// (sequence, KV head) row; a segment's survivors are compacted into a list of
+// LSTRIDE slots (SEG plus room for one rescued block per query head).
+constexpr int SEG = 64;
+constexpr int LSTRIDE = SEG + 8;
+constexpr int MAX_CTAS = 1024;       // upper bound on streaming CTAs (sizes the scratch)
+constexpr int MAX_ENTRIES = 49152;   // plan kernel keeps the unit prefix in shared memory
+
+// Scratch layout (byte offsets from a 256-byte aligned base).
+struct WsLayout {
+    int rows;        // batch * n_kv_heads
+    int nseg;        // segments per row
+    int entries;     // rows * (nseg + 1): one pseudo-segment per row holds the tail unit
+    size_t hdr;      // int32[8]: [0] total units U, [1] streaming CTAs P
+    size_t seg_count;   // int32 [rows * nseg]
+    size_t seg_list;    // int32 [rows * nseg * LSTRIDE]: block index | head bits << 24
+    size_t seg_resc;    // {int cnt; float maxb; int arg; int pad} [rows * nseg * G]
+    size_t pref;        // int32 [entries + 1] exclusive prefix of units per entry
+    size_t cta_start;   // int4 [MAX_CTAS]: {u0, u1, first entry, 0}
+    size_t tau_eff;     // float [batch * n_q_heads]
+    size_t part_ml;     // float2 [(MAX_CTAS + rows) * G]
+    size_t part_o;      // float [(MAX_CTAS + rows) * G * d]
+    size_t total;
+};
+WsLayout ws_layout(const eta_cache_desc* d);
+
+struct RescueRec { int cnt; float maxb; int arg; int pad; };
+
+// Arguments of the screening and planning kernels (defined in eta_screen.cu, launched from eta_decode).
+struct ScreenArgs {
+    const __nv_bfloat16* q;
+    const __half* musig;
+    const float* mnorm;
+    const int32_t* seq_lens;
+    const float* tau;
+    const float* head_const;
+    float z, a, scale;
+    int lwb, rescue_window;
+    uint32_t flags;
+    int Hq, Hkv, b, t_cap, nb_cap, nseg;
+    int32_t* seg_count;
+    int32_t* seg_list;
+    RescueRec* seg_resc;
+    float* tau_eff;
+    uint8_t* sel_mask;
+};
+struct PlanArgs {
+    const int32_t* seq_lens;
+    int Hkv, G, b, t_cap, nb_cap, nseg, rows, entries, rescue_window, n_ctas;
+    int32_t* seg_count;
+    int32_t* seg_list;
+    const RescueRec* seg_resc;
+    uint8_t* sel_mask;
+    int32_t* pref;
+    int4* cta_start;
+    int32_t* hdr;
+    int32_t* stats;
+    uint32_t* status;
+};
+int launch_screen(const ScreenArgs& a, int rows, int D, int G, cudaStream_t s);
+int launch_plan(const PlanArgs& a, cudaStream_t s);
+
+// -------------------------------------------------------------- device side
+#ifdef __CUDACC__
+
+constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls before a bounded wait gives up
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out (the caller then abandons the work
+// and reports ETA_DEV_TIMEOUT instead of spinning forever).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// 1-D bulk copy global -> shared, completion counted on an mbarrier.
+// Both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// 4-D tiled copy global -> shared through a tensor map (no multicast).
+__device__ __forceinline__ void tma_load_4d(void* dst, const void* tmap, int x, int y, int z, int w, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const void* tmap) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
+}
+
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
+
+#endif  // __CUDACC__
+}  // namespace eta

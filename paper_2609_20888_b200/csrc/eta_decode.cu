@@ -1,0 +1,595 @@
+// Streaming stage of eta_decode: SiLU-gated attention over the surviving blocks
+// (Algorithm 3, attention lines and tail phase; Eq. mult_attn at inference), the
+// GQA-grouped execution of the fused-kernel appendix, and the associative
+// (m, l, O) merge of its "two-stage reduction".
+//
+// Work is the flattened sequence of "units" the plan step laid out: for each
+// (sequence, KV head) row its surviving blocks, then its tail.  Every CTA owns an
+// equal, contiguous share of that sequence, so the load is balanced whatever the
+// per-head survivor counts are; a share may cross rows, and a row may be split
+// over CTAs; each (CTA, row) piece produces one partial (m, l, O) per query head.
+//
+// Inside a CTA one producer warp walks the survivor lists and issues tiled TMA
+// copies (128-byte swizzle) of K and V tiles into a ring of shared-memory stages;
+// four consumer warps each take a quarter of the tokens of every tile.  The G
+// query heads of the group are packed on the M side of mma.m16n8k16 (bf16 in,
+// fp32 out), tokens on N, so each K/V byte is read once from HBM and once from
+// shared memory for all heads.  The head_dim and token orders fed to the MMAs are
+// permuted (a dot product does not care) so that every shared-memory read is a
+// conflict-free 16-byte load of the swizzled tile.  Softmax statistics and
+// accumulators are fp32; P is fed to the second MMA as a bf16 high part plus a
+// bf16 residual, so the product keeps fp32-level accuracy.
+#include <cuda.h>
+
+#include "eta_common.cuh"
+
+namespace eta {
+
+struct DecodeArgs {
+    const __nv_bfloat16* q;
+    const int32_t* seq_lens;
+    const float* tau_eff;
+    const int32_t* seg_list;
+    const int32_t* pref;
+    const int4* cta_start;
+    float2* part_ml;
+    float* part_o;
+    uint32_t* status;
+    float beta, scale;
+    int Hq, Hkv, G, b, t_cap, nseg, entries;
+};
+
+constexpr uint32_t UF_FIRST = 1u, UF_LAST = 2u, UF_END = 4u;
+constexpr int N_CONSUMER_WARPS = 4;
+constexpr int DECODE_THREADS = 32 * (N_CONSUMER_WARPS + 1);
+
+// token row inside an 8-row group that MMA column n reads: bits 0 and 2 of n swapped, so that the two
+// rows a quarter-warp touches in one 16-byte load sit in different halves of the swizzle pattern
+__device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
+    return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
+}
+__device__ __forceinline__ int rho(int n) { return (n & 2) | ((n & 1) << 2) | ((n >> 2) & 1); }
+
+template <int D, int TS, int NSTAGE>
+struct DecodeSmem {
+    static constexpr int HALVES = D / 64;
+    static constexpr int TILE_BYTES = TS * 128;                 // one 64-column half tile
+    static constexpr int STAGE_BYTES = 2 * HALVES * TILE_BYTES; // K halves then V halves
+    static constexpr int BAR_OFF = NSTAGE * STAGE_BYTES;        // full[NSTAGE], empty[NSTAGE], flush
+    static constexpr int DESC_OFF = BAR_OFF + 8 * (2 * NSTAGE + 2);
+    static constexpr int ML_OFF = DESC_OFF + 16 * NSTAGE;       // float m[4][8], l[4][8]
+    static constexpr int MO_OFF = ML_OFF + 4 * 2 * N_CONSUMER_WARPS * 8;
+    static size_t bytes(int G) { return 1024 + MO_OFF + sizeof(float) * N_CONSUMER_WARPS * G * D; }
+};
+
+template <int D, int TS, int NSTAGE>
+__global__ void __launch_bounds__(DECODE_THREADS, 1)
+decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DecodeArgs a) {
+    using L = DecodeSmem<D, TS, NSTAGE>;
+    constexpr int HALVES = L::HALVES;
+    constexpr int WT = TS / N_CONSUMER_WARPS;   // tokens per consumer warp per tile (8 or 16)
+    constexpr int NT = WT / 8;                  // 8-token MMA column tiles per warp
+    static_assert(NT == 1 || NT == 2, "tile must give each warp 8 or 16 tokens");
+
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
+    uint64_t* empty = full + NSTAGE;
+    uint64_t* flushbar = empty + NSTAGE;
+    int4* desc = reinterpret_cast<int4*>(smem + L::DESC_OFF);
+    float* sm_m = reinterpret_cast<float*>(smem + L::ML_OFF);
+    float* sm_l = sm_m + N_CONSUMER_WARPS * 8;
+    float* sm_o = reinterpret_cast<float*>(smem + L::MO_OFF);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int4 cs = a.cta_start[blockIdx.x];
+    const int u0 = cs.x, u1 = cs.y;
+    if (u0 >= u1) return;
+
+    if (tid == 0) {
+        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], N_CONSUMER_WARPS); }
+        mbar_init(&flushbar[0], 32 * N_CONSUMER_WARPS);
+        fence_barrier_init();
+        prefetch_tmap(&tmK);
+        prefetch_tmap(&tmV);
+    }
+    __syncthreads();
+
+    if (warp == N_CONSUMER_WARPS) {
+        // ------------------------------------------------------------ producer
+        const int EPR = a.nseg + 1;
+        const int E = a.entries;
+        int e = cs.z;
+        int u = u0;
+        uint32_t fill = 0;
+        bool ok = true;
+        while (u < u1 && ok) {
+            // entry holding unit u: pref[e] <= u < pref[e+1]; skip empty entries 32 at a time
+            while (true) {
+                const int pv = __ldg(a.pref + min(e + 1 + lane, E));
+                const unsigned gt = __ballot_sync(0xffffffffu, pv > u);
+                if (gt) { e += __ffs(gt) - 1; break; }
+                e += 32;
+                if (e >= E) { ok = false; break; }     // inconsistent plan: stop instead of walking off
+            }
+            if (!ok) break;
+            const int pe = __ldg(a.pref + e), pn = __ldg(a.pref + e + 1);
+            const int r = e / EPR, sg = e % EPR;
+            const int row_begin = __ldg(a.pref + r * EPR), row_end = __ldg(a.pref + (r + 1) * EPR);
+            const int i = r / a.Hkv, hk = r % a.Hkv;
+            int T = __ldg(a.seq_lens + i);
+            T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
+            const int NB = T / a.b, tail = T - NB * a.b;
+            const int n_here = min(pn, u1) - u;
+            const int off = u - pe;
+            const bool is_tail = (sg == a.nseg);
+            const int32_t* list = a.seg_list + ((int64_t)r * a.nseg + sg) * LSTRIDE + off;
+            for (int base = 0; base < n_here && ok; base += 32) {
+                int my = 0;
+                if (base + lane < n_here) my = is_tail ? (NB | (0xff << 24)) : __ldg(list + base + lane);
+                const int nb = min(32, n_here - base);
+                for (int k = 0; k < nb && ok; ++k) {
+                    const int ent = __shfl_sync(0xffffffffu, my, k);
+                    const int uu = u + base + k;
+                    const int j = ent & 0xffffff;
+                    const int hmask = (ent >> 24) & 0xff;
+                    const int nrows = is_tail ? tail : a.b;
+                    const bool first = (uu == u0) || (uu == row_begin);
+                    const bool last = (uu == u1 - 1) || (uu == row_end - 1);
+                    for (int sub = 0; sub * TS < nrows && ok; ++sub) {
+                        const int nvalid = min(TS, nrows - sub * TS);
+                        const bool last_sub = (sub + 1) * TS >= nrows;
+                        const int stage = fill % NSTAGE;
+                        const uint32_t round = fill / NSTAGE;
+                        if (lane == 0) {
+                            if (!mbar_wait(&empty[stage], (round & 1) ^ 1)) {
+                                ok = false;
+                            } else {
+                                uint32_t fl = (first && sub == 0 ? UF_FIRST : 0u) | (last && last_sub ? UF_LAST : 0u) |
+                                              (uu == u1 - 1 && last_sub ? UF_END : 0u);
+                                desc[stage] = make_int4(r, (int)fl, hmask, nvalid);
+                                unsigned char* st = smem + stage * L::STAGE_BYTES;
+                                mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
+                                const int y = j * a.b + sub * TS;
+#pragma unroll
+                                for (int hf = 0; hf < HALVES; ++hf) {
+                                    tma_load_4d(st + hf * L::TILE_BYTES, &tmK, hf * 64, y, hk, i, &full[stage]);
+                                    tma_load_4d(st + (HALVES + hf) * L::TILE_BYTES, &tmV, hf * 64, y, hk, i, &full[stage]);
+                                }
+                            }
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                        ++fill;
+                    }
+                }
+            }
+            u += n_here;
+        }
+        if (!ok) {
+            // give up: report, then let copies already issued land before the CTA's shared memory is released
+            if (lane == 0) {
+                if (a.status) atomicOr(a.status, ETA_DEV_TIMEOUT);
+                const uint32_t first_fill = fill > NSTAGE ? fill - NSTAGE : 0;
+                for (uint32_t f = first_fill; f < fill; ++f) mbar_wait(&full[f % NSTAGE], (f / NSTAGE) & 1);
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- consumers
+    const int g = lane >> 2, t = lane & 3;
+    const int rb = warp * WT;                          // first token row of this warp inside a tile
+    const int r0 = rho(2 * t), r1 = rho(2 * t + 1);    // token rows (within an 8-group) of MMA columns 2t, 2t+1
+    const int vchunk = ((g & 1) << 2) | (g >> 1);      // 16-byte chunk of a V half-row this lane reads
+    const float LOG2E = 1.4426950408889634f;
+
+    uint32_t qa[HALVES][2][4];
+    float o[HALVES][4][4];
+    float m_run = -INFINITY, l_run = 0.f, te = 0.f;
+    int row = -1;
+    uint32_t flush_phase = 0;
+    bool ok = true;
+
+    for (uint32_t fill = 0;; ++fill) {
+        const int stage = fill % NSTAGE;
+        if (!mbar_wait(&full[stage], (fill / NSTAGE) & 1)) { ok = false; break; }
+        const int4 ds = desc[stage];
+        const uint32_t fl = (uint32_t)ds.y;
+        const int hmask = ds.z, nvalid = ds.w;
+        const uint32_t kbase = smem_u32(smem + stage * L::STAGE_BYTES);
+        const uint32_t vbase = kbase + HALVES * L::TILE_BYTES;
+
+        if (fl & UF_FIRST) {
+            row = ds.x;
+            const int i = row / a.Hkv, hk = row % a.Hkv;
+            const bool head = g < a.G;
+            const __nv_bfloat16* qp = a.q + ((int64_t)i * a.Hq + hk * a.G + (head ? g : 0)) * D;
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int m = 0; m < 2; ++m) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (head) v = __ldg(reinterpret_cast<const uint4*>(qp + 64 * hf + 32 * m + 8 * t));
+                    qa[hf][m][0] = v.x; qa[hf][m][1] = v.y; qa[hf][m][2] = v.z; qa[hf][m][3] = v.w;
+                }
+            te = head ? __ldg(a.tau_eff + (int64_t)i * a.Hq + hk * a.G + g) : 0.f;
+            m_run = -INFINITY;
+            l_run = 0.f;
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) o[hf][mt][c] = 0.f;
+        }
+
+        // ---- S = q K^T for this warp's WT tokens: heads on M (rows 8..15 are padding), tokens on N
+        float sacc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) sacc[nt][c] = 0.f;
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+            for (int m = 0; m < 2; ++m)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int trow = rb + nt * 8 + rho(g);
+                    const uint4 kv = lds128(kbase + hf * L::TILE_BYTES + trow * 128 + ((((4 * m + t) ^ (trow & 7))) << 4));
+                    mma_bf16_16816(sacc[nt], qa[hf][m][0], 0u, qa[hf][m][1], 0u, kv.x, kv.y);
+                    mma_bf16_16816(sacc[nt], qa[hf][m][2], 0u, qa[hf][m][3], 0u, kv.z, kv.w);
+                }
+
+        // ---- gate, mask, online softmax (lane (g,t) holds head g, tokens r0/r1 of each 8-group)
+        const bool head_on = (g < a.G) && ((hmask >> g) & 1);
+        float sg[NT][2];
+        float bmax = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const int trow = rb + nt * 8 + (c ? r1 : r0);
+                const float S = sacc[nt][c] * a.scale;
+                const float x = (a.beta == 0.f) ? 0.f : a.beta * (S - te);
+                float gated = (te == -INFINITY) ? S : S / (1.f + __expf(-x));
+                gated = (head_on && trow < nvalid) ? gated : -INFINITY;
+                sg[nt][c] = gated;
+                bmax = fmaxf(bmax, gated);
+            }
+        bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+        bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+        const float m_new = fmaxf(m_run, bmax);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        const float alpha = (m_run == m_new) ? 1.f : exp2f((m_run - m_use) * LOG2E);   // m_run = -inf gives 0
+        float p[NT][2], psum = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                p[nt][c] = exp2f((sg[nt][c] - m_use) * LOG2E);   // -inf gives 0
+                psum += p[nt][c];
+            }
+        l_run = l_run * alpha + psum;
+        m_run = m_new;
+
+        // accumulators hold heads 2t, 2t+1 in their columns: fetch those heads' rescale factors
+        const float al0 = __shfl_sync(0xffffffffu, alpha, 8 * t);
+        const float al1 = __shfl_sync(0xffffffffu, alpha, 8 * t + 4);
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) {
+                    o[hf][mt][0] *= al0; o[hf][mt][1] *= al1; o[hf][mt][2] *= al0; o[hf][mt][3] *= al1;
+                }
+        }
+
+        // ---- P as the B operand: bf16 high part and bf16 residual
+        uint32_t pb_hi[2] = {0u, 0u}, pb_lo[2] = {0u, 0u};
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const __nv_bfloat162 hi = __floats2bfloat162_rn(p[nt][0], p[nt][1]);
+            const float2 hf2 = __bfloat1622float2(hi);
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(p[nt][0] - hf2.x, p[nt][1] - hf2.y);
+            pb_hi[nt] = *reinterpret_cast<const uint32_t*>(&hi);
+            pb_lo[nt] = *reinterpret_cast<const uint32_t*>(&lo);
+        }
+
+        // ---- O^T += V^T P : head_dim on M, tokens on K, heads on N
+        const bool partial = nvalid < TS;
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) {
+            uint4 v[2 * NT];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int trow = rb + nt * 8 + (c ? r1 : r0);
+                    uint4 x = lds128(vbase + hf * L::TILE_BYTES + trow * 128 + ((vchunk ^ (trow & 7)) << 4));
+                    if (partial && trow >= nvalid) x = make_uint4(0, 0, 0, 0);   // rows past the sequence end
+                    v[nt * 2 + c] = x;
+                }
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt) {
+                const uint32_t xa = u4_get(v[0], mt), xb = u4_get(v[1], mt);
+                const uint32_t a0 = __byte_perm(xa, xb, 0x5410), a1 = __byte_perm(xa, xb, 0x7632);
+                uint32_t a2 = 0u, a3 = 0u;
+                if (NT == 2) {
+                    const uint32_t xc = u4_get(v[2 * (NT - 1)], mt), xd = u4_get(v[2 * (NT - 1) + 1], mt);
+                    a2 = __byte_perm(xc, xd, 0x5410);
+                    a3 = __byte_perm(xc, xd, 0x7632);
+                }
+                mma_bf16_16816(o[hf][mt], a0, a1, a2, a3, pb_hi[0], pb_hi[1]);
+                mma_bf16_16816(o[hf][mt], a0, a1, a2, a3, pb_lo[0], pb_lo[1]);
+            }
+        }
+
+        // this warp is done with the stage
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[stage]);
+
+        if (fl & UF_LAST) {
+            // ---- piece finished: combine the four warps' partials and store one (m, l, O) per head
+            float lsum = l_run + __shfl_xor_sync(0xffffffffu, l_run, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            if (t == 0) { sm_m[warp * 8 + g] = m_run; sm_l[warp * 8 + g] = lsum; }
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) {
+                    const int dcol = 64 * hf + 8 * vchunk + 2 * mt;
+                    if (2 * t < a.G)
+                        *reinterpret_cast<float2*>(sm_o + ((warp * a.G + 2 * t) * D + dcol)) = make_float2(o[hf][mt][0], o[hf][mt][2]);
+                    if (2 * t + 1 < a.G)
+                        *reinterpret_cast<float2*>(sm_o + ((warp * a.G + 2 * t + 1) * D + dcol)) = make_float2(o[hf][mt][1], o[hf][mt][3]);
+                }
+            mbar_arrive(&flushbar[0]);
+            if (!mbar_wait(&flushbar[0], flush_phase)) { ok = false; break; }
+            flush_phase ^= 1;
+            const int slot = blockIdx.x + row;
+            for (int idx = tid; idx < a.G * D; idx += 32 * N_CONSUMER_WARPS) {
+                const int hh = idx / D, dd = idx % D;
+                float M = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < N_CONSUMER_WARPS; ++w) M = fmaxf(M, sm_m[w * 8 + hh]);
+                float acc = 0.f, lacc = 0.f;
+                if (M != -INFINITY) {
+#pragma unroll
+                    for (int w = 0; w < N_CONSUMER_WARPS; ++w) {
+                        const float sc = exp2f((sm_m[w * 8 + hh] - M) * LOG2E);
+                        acc = fmaf(sm_o[(w * a.G + hh) * D + dd], sc, acc);
+                        lacc = fmaf(sm_l[w * 8 + hh], sc, lacc);
+                    }
+                }
+                a.part_o[((int64_t)slot * a.G + hh) * D + dd] = acc;
+                if (dd == 0) a.part_ml[(int64_t)slot * a.G + hh] = make_float2(M, lacc);
+            }
+            mbar_arrive(&flushbar[0]);
+            if (!mbar_wait(&flushbar[0], flush_phase)) { ok = false; break; }
+            flush_phase ^= 1;
+        }
+        if (fl & UF_END) break;
+    }
+    if (!ok && lane == 0 && a.status) atomicOr(a.status, ETA_DEV_TIMEOUT);
+}
+
+// Associative merge of the pieces of one (sequence, query head): Algorithm 3, global reduction.
+struct MergeArgs {
+    const int32_t* pref;
+    const int32_t* hdr;
+    const float2* part_ml;
+    const float* part_o;
+    float* out;
+    int Hq, Hkv, G, nseg, rows;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128) merge_kernel(const MergeArgs a) {
+    const int wid = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (wid >= a.rows * a.G) return;
+    const int r = wid / a.G, gq = wid % a.G;
+    const int i = r / a.Hkv, hk = r % a.Hkv;
+    const int EPR = a.nseg + 1;
+    const int ra = a.pref[r * EPR], rbd = a.pref[(r + 1) * EPR];
+    const int64_t U = a.hdr[0], P = a.hdr[1];
+    constexpr int VPL = D / 32;
+    float acc[VPL];
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
+    float mg = -INFINITY, lg = 0.f;
+    if (rbd > ra && U > 0) {
+        int c_lo = (int)(((int64_t)ra * P) / U) - 1;
+        int c_hi = (int)(((int64_t)rbd * P + U - 1) / U) + 1;
+        c_lo = c_lo < 0 ? 0 : c_lo;
+        c_hi = c_hi > (int)P - 1 ? (int)P - 1 : c_hi;
+        for (int c = c_lo; c <= c_hi; ++c) {
+            const int cu0 = (int)(((int64_t)c * U) / P), cu1 = (int)(((int64_t)(c + 1) * U) / P);
+            if (max(cu0, ra) >= min(cu1, rbd)) continue;
+            const int64_t slot = (int64_t)c + r;
+            const float2 ml = a.part_ml[slot * a.G + gq];
+            if (ml.x == -INFINITY) continue;
+            const float mn = fmaxf(mg, ml.x);
+            const float ag = __expf(mg - mn), ac = __expf(ml.x - mn);
+            const float* po = a.part_o + (slot * a.G + gq) * D + lane * VPL;
+            lg = lg * ag + ml.y * ac;
+#pragma unroll
+            for (int k = 0; k < VPL; ++k) acc[k] = acc[k] * ag + po[k] * ac;
+            mg = mn;
+        }
+    }
+    float* op = a.out + ((int64_t)i * a.Hq + hk * a.G + gq) * D + lane * VPL;
+    const float inv = lg > 0.f ? 1.f / lg : 0.f;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) op[k] = acc[k] * inv;
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr);
+        if (e != cudaSuccess || qr != cudaDriverEntryPointSuccess || !p) {
+            set_cuda_error(e != cudaSuccess ? e : cudaErrorUnknown, "cuTensorMapEncodeTiled lookup");
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// K or V as a 4-D tensor (c, t, hk, i) of bf16; a box is 64 columns x TS tokens, 128-byte swizzled.
+static int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d, int64_t sb, int64_t sh, int64_t st,
+                     int TS) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return ETA_ERR_CUDA;
+    cuuint64_t dims[4] = {(cuuint64_t)d->head_dim, (cuuint64_t)d->t_cap, (cuuint64_t)d->n_kv_heads, (cuuint64_t)d->batch};
+    cuuint64_t strides[3] = {(cuuint64_t)st * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)TS, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) {
+        set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+        return ETA_ERR_CUDA;
+    }
+    return ETA_OK;
+}
+
+template <int D, int TS, int NSTAGE>
+static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const DecodeArgs& a, int n_ctas,
+                           cudaStream_t s) {
+    const size_t smem = DecodeSmem<D, TS, NSTAGE>::bytes(a.G);
+    static size_t configured = 0;
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, TS, NSTAGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) { set_cuda_error(e, "decode smem attribute"); return ETA_ERR_CUDA; }
+        configured = smem;
+    }
+    decode_kernel<D, TS, NSTAGE><<<n_ctas, DECODE_THREADS, smem, s>>>(tmK, tmV, a);
+    return check_launch("decode");
+}
+
+}  // namespace eta
+
+extern "C" {
+
+int eta_decode_kernel_count(void) { return 4; }
+
+int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q, const void* K, const void* V,
+               const int32_t* seq_lens, const void* musig, const float* mnorm, const float* tau,
+               const float* head_const, float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev,
+               void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace eta;
+    int rc = validate_desc(desc);
+    if (rc != ETA_OK) return rc;
+    if (!params || !q || !K || !V || !seq_lens || !out || !sel_mask) return ETA_ERR_INVALID_ARG;
+    const bool dense = (params->flags & ETA_FLAG_DENSE) != 0;
+    if (!dense && (!musig || !mnorm)) return ETA_ERR_INVALID_ARG;
+    if ((tau != nullptr) == (head_const != nullptr)) return ETA_ERR_INVALID_ARG;
+    if (params->rescue_window < 1 || params->lwb < 0) return ETA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V) | reinterpret_cast<uintptr_t>(q) |
+         reinterpret_cast<uintptr_t>(musig) | reinterpret_cast<uintptr_t>(out)) & 15)
+        return ETA_ERR_UNSUPPORTED;
+    const WsLayout L = ws_layout(desc);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
+        return ETA_ERR_WORKSPACE;
+    if (L.entries > MAX_ENTRIES) return ETA_ERR_UNSUPPORTED;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    const int D = desc->head_dim, b = desc->block_size;
+    const int G = desc->n_q_heads / desc->n_kv_heads;
+    const float scale = params->scale > 0.f ? params->scale : 1.0f / sqrtf((float)D);
+
+    int dev = 0, n_sm = 0;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (ce != cudaSuccess) { set_cuda_error(ce, "device query"); return ETA_ERR_CUDA; }
+    const int TS = b < 64 ? b : 64;
+    int per_sm = params->ctas_per_sm > 0 ? params->ctas_per_sm : 1;
+    if (per_sm > 2) per_sm = 2;
+    if (!(D == 128 && TS == 64) || G == 8) per_sm = 1;
+    int n_ctas = n_sm * per_sm;
+    if (n_ctas > MAX_CTAS) n_ctas = MAX_CTAS;
+
+    ScreenArgs sa;
+    sa.q = static_cast<const __nv_bfloat16*>(q);
+    sa.musig = static_cast<const __half*>(musig);
+    sa.mnorm = mnorm;
+    sa.seq_lens = seq_lens;
+    sa.tau = tau;
+    sa.head_const = head_const;
+    sa.z = params->z; sa.a = params->a; sa.scale = scale;
+    sa.lwb = params->lwb; sa.rescue_window = params->rescue_window; sa.flags = params->flags;
+    sa.Hq = desc->n_q_heads; sa.Hkv = desc->n_kv_heads; sa.b = b; sa.t_cap = desc->t_cap; sa.nb_cap = desc->nb_cap;
+    sa.nseg = L.nseg;
+    sa.seg_count = reinterpret_cast<int32_t*>(ws + L.seg_count);
+    sa.seg_list = reinterpret_cast<int32_t*>(ws + L.seg_list);
+    sa.seg_resc = reinterpret_cast<RescueRec*>(ws + L.seg_resc);
+    sa.tau_eff = reinterpret_cast<float*>(ws + L.tau_eff);
+    sa.sel_mask = sel_mask;
+    rc = launch_screen(sa, L.rows, D, G, s);
+    if (rc != ETA_OK) return rc;
+
+    PlanArgs pa;
+    pa.seq_lens = seq_lens;
+    pa.Hkv = desc->n_kv_heads; pa.G = G; pa.b = b; pa.t_cap = desc->t_cap; pa.nb_cap = desc->nb_cap;
+    pa.nseg = L.nseg; pa.rows = L.rows; pa.entries = L.entries; pa.rescue_window = params->rescue_window;
+    pa.n_ctas = n_ctas;
+    pa.seg_count = sa.seg_count; pa.seg_list = sa.seg_list; pa.seg_resc = sa.seg_resc; pa.sel_mask = sel_mask;
+    pa.pref = reinterpret_cast<int32_t*>(ws + L.pref);
+    pa.cta_start = reinterpret_cast<int4*>(ws + L.cta_start);
+    pa.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
+    pa.stats = stats;
+    pa.status = status_dev;
+    rc = launch_plan(pa, s);
+    if (rc != ETA_OK) return rc;
+
+    CUtensorMap tmK, tmV;
+    rc = make_tmap(&tmK, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t, TS);
+    if (rc != ETA_OK) return rc;
+    rc = make_tmap(&tmV, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_t, TS);
+    if (rc != ETA_OK) return rc;
+
+    DecodeArgs da;
+    da.q = sa.q; da.seq_lens = seq_lens; da.tau_eff = sa.tau_eff; da.seg_list = sa.seg_list; da.pref = pa.pref;
+    da.cta_start = pa.cta_start;
+    da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
+    da.part_o = reinterpret_cast<float*>(ws + L.part_o);
+    da.status = status_dev;
+    da.beta = params->beta; da.scale = scale;
+    da.Hq = desc->n_q_heads; da.Hkv = desc->n_kv_heads; da.G = G; da.b = b; da.t_cap = desc->t_cap;
+    da.nseg = L.nseg; da.entries = L.entries;
+    if (D == 128 && TS == 64) {
+        rc = (per_sm == 2) ? launch_decode_t<128, 64, 3>(tmK, tmV, da, n_ctas, s)
+                           : launch_decode_t<128, 64, 6>(tmK, tmV, da, n_ctas, s);
+    } else if (D == 128 && TS == 32) {
+        rc = launch_decode_t<128, 32, 8>(tmK, tmV, da, n_ctas, s);
+    } else if (D == 64 && TS == 64) {
+        rc = launch_decode_t<64, 64, 8>(tmK, tmV, da, n_ctas, s);
+    } else {
+        rc = launch_decode_t<64, 32, 8>(tmK, tmV, da, n_ctas, s);
+    }
+    if (rc != ETA_OK) return rc;
+
+    MergeArgs ma;
+    ma.pref = pa.pref; ma.hdr = pa.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
+    ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows;
+    const unsigned mgrid = (unsigned)((L.rows * G + 3) / 4);
+    if (D == 128) merge_kernel<128><<<mgrid, 128, 0, s>>>(ma);
+    else merge_kernel<64><<<mgrid, 128, 0, s>>>(ma);
+    return check_launch("merge");
+}
+
+}  // extern "C"

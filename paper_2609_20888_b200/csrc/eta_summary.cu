@@ -1,0 +1,210 @@
+// Block-summary kernels: the dual probabilistic-geometric index of Section 3
+// (centroid, coordinate-wise population standard deviation, largest key norm),
+// built in one pass over K at prefill and extended by one block whenever a
+// decode step completes a block.
+//
+// One warp owns one block of b keys.  A row of d bf16 values is read by d/8
+// lanes as 16-byte vectors, so a warp covers 32/(d/8) rows per load
+// instruction and every 32-byte sector of the block is requested exactly once
+// from HBM; the second pass (deviations about the mean) re-reads the block
+// from L1/L2.  Arithmetic is fp32.
+#include "eta_common.cuh"
+
+namespace eta {
+
+template <int D>
+__device__ __forceinline__ void summarize_block(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
+                                                bool envelope, __half* __restrict__ rec, float* __restrict__ mn) {
+    constexpr int LPR = D / 8;        // lanes per row
+    constexpr int RPP = 32 / LPR;     // rows per pass
+    const int lane = threadIdx.x & 31;
+    const int cc = lane % LPR, ro = lane / LPR;
+    const __nv_bfloat16* base = blk + cc * 8;
+
+    float sum[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) sum[k] = 0.f;
+    float maxn2 = 0.f;
+    // pass 1: coordinate sums and row norms, four rows per lane in flight
+    for (int t0 = ro; t0 < b; t0 += 4 * RPP) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            int t = t0 + u * RPP;
+            v[u] = (t < b) ? __ldg(reinterpret_cast<const uint4*>(base + (int64_t)t * stride_t)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            float n2 = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float lo = bf16_lo(w[k]), hi = bf16_hi(w[k]);
+                sum[2 * k] += lo;
+                sum[2 * k + 1] += hi;
+                n2 = fmaf(lo, lo, n2);
+                n2 = fmaf(hi, hi, n2);
+            }
+#pragma unroll
+            for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+            maxn2 = fmaxf(maxn2, n2);
+        }
+    }
+#pragma unroll
+    for (int s = LPR; s < 32; s <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) sum[k] += __shfl_xor_sync(0xffffffffu, sum[k], s);
+        maxn2 = fmaxf(maxn2, __shfl_xor_sync(0xffffffffu, maxn2, s));
+    }
+    float mean[8];
+    const float inv_b = 1.0f / (float)b;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) mean[k] = sum[k] * inv_b;
+
+    // pass 2: squared deviations about the mean
+    float dev[8], env[8], sub[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { dev[k] = 0.f; env[k] = 0.f; sub[k] = 0.f; }
+    for (int t0 = ro; t0 < b; t0 += 4 * RPP) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            int t = t0 + u * RPP;
+            v[u] = (t < b) ? __ldg(reinterpret_cast<const uint4*>(base + (int64_t)t * stride_t)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            int t = t0 + u * RPP;
+            if (t < b) {
+                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float dl = bf16_lo(w[k]) - mean[2 * k], dh = bf16_hi(w[k]) - mean[2 * k + 1];
+                    dev[2 * k] = fmaf(dl, dl, dev[2 * k]);
+                    dev[2 * k + 1] = fmaf(dh, dh, dev[2 * k + 1]);
+                    sub[2 * k] = fmaf(dl, dl, sub[2 * k]);
+                    sub[2 * k + 1] = fmaf(dh, dh, sub[2 * k + 1]);
+                }
+            }
+            // a 4-token sub-block ends after 4/RPP of this lane's rows (u counts them: t = ro + (4*it+u)*RPP)
+            if (envelope && ((u + 1) % (4 / RPP) == 0)) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    float s4 = sub[k];
+#pragma unroll
+                    for (int s = LPR; s < 32; s <<= 1) s4 += __shfl_xor_sync(0xffffffffu, s4, s);
+                    env[k] = fmaxf(env[k], s4);
+                    sub[k] = 0.f;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int s = LPR; s < 32; s <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) dev[k] += __shfl_xor_sync(0xffffffffu, dev[k], s);
+    }
+    float sg[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) sg[k] = envelope ? sqrtf(env[k] * 0.25f) : sqrtf(dev[k] * inv_b);
+
+    // row group 0 stores the centroid chunk, row group 1 the sigma chunk: one contiguous record
+    if (ro < 2) {
+        const float* src = (ro == 0) ? mean : sg;
+        __half2 h[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) h[k] = __floats2half2_rn(src[2 * k], src[2 * k + 1]);
+        uint4 o;
+        o.x = *reinterpret_cast<uint32_t*>(&h[0]);
+        o.y = *reinterpret_cast<uint32_t*>(&h[1]);
+        o.z = *reinterpret_cast<uint32_t*>(&h[2]);
+        o.w = *reinterpret_cast<uint32_t*>(&h[3]);
+        *reinterpret_cast<uint4*>(rec + ro * D + cc * 8) = o;
+    }
+    if (lane == 0) *mn = sqrtf(maxn2);
+}
+
+template <int D>
+__global__ void __launch_bounds__(128) build_summaries_kernel(
+    const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
+    int nb_max, int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
+    float* __restrict__ mnorm) {
+    const int64_t wid = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (wid >= (int64_t)rows * nb_max) return;
+    const int r = (int)(wid / nb_max), j = (int)(wid % nb_max);
+    const int i = r / Hkv, hk = r % Hkv;
+    int T = seq_lens[i];
+    T = T < 0 ? 0 : (T > t_cap ? t_cap : T);
+    if (j >= T / b || j >= nb_cap) return;
+    const __nv_bfloat16* blk = K + i * sb + hk * sh + (int64_t)j * b * st;
+    const int64_t rec = (int64_t)r * nb_cap + j;
+    summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
+}
+
+template <int D>
+__global__ void __launch_bounds__(128) append_summary_kernel(
+    const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
+    int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
+    float* __restrict__ mnorm) {
+    const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (r >= rows) return;
+    const int i = r / Hkv, hk = r % Hkv;
+    const int T = seq_lens[i];
+    if (T <= 0 || T > t_cap || T % b != 0) return;
+    const int j = T / b - 1;
+    if (j >= nb_cap) return;
+    const __nv_bfloat16* blk = K + i * sb + hk * sh + (int64_t)j * b * st;
+    const int64_t rec = (int64_t)r * nb_cap + j;
+    summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
+}
+
+}  // namespace eta
+
+extern "C" {
+
+int eta_build_block_summaries(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens, void* musig,
+                              float* mnorm, uint32_t flags, void* stream) {
+    int rc = eta::validate_desc(desc);
+    if (rc != ETA_OK) return rc;
+    if (!K || !seq_lens || !musig || !mnorm) return ETA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(musig)) & 15) return ETA_ERR_UNSUPPORTED;
+    const int rows = desc->batch * desc->n_kv_heads;
+    const int nb_max = desc->t_cap / desc->block_size;
+    if (nb_max == 0) return ETA_OK;
+    const int64_t warps = (int64_t)rows * nb_max;
+    const unsigned grid = (unsigned)((warps + 3) / 4);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
+    auto Kp = static_cast<const __nv_bfloat16*>(K);
+    auto mp = static_cast<__half*>(musig);
+    if (desc->head_dim == 128)
+        eta::build_summaries_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, nb_max, rows, seq_lens, env, mp, mnorm);
+    else
+        eta::build_summaries_kernel<64><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, nb_max, rows, seq_lens, env, mp, mnorm);
+    return eta::check_launch("eta_build_block_summaries");
+}
+
+int eta_append_summary(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens_after, void* musig,
+                       float* mnorm, uint32_t flags, void* stream) {
+    int rc = eta::validate_desc(desc);
+    if (rc != ETA_OK) return rc;
+    if (!K || !seq_lens_after || !musig || !mnorm) return ETA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(musig)) & 15) return ETA_ERR_UNSUPPORTED;
+    const int rows = desc->batch * desc->n_kv_heads;
+    const unsigned grid = (unsigned)((rows + 3) / 4);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
+    auto Kp = static_cast<const __nv_bfloat16*>(K);
+    auto mp = static_cast<__half*>(musig);
+    if (desc->head_dim == 128)
+        eta::append_summary_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm);
+    else
+        eta::append_summary_kernel<64><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm);
+    return eta::check_launch("eta_append_summary");
+}
+
+}  // extern "C"

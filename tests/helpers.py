@@ -102,3 +102,70 @@ def calibrate_head_const(bound, seq_lens, b, sparsity_levels):
             k = min(NB - 1, max(0, int(np.floor(sparsity_levels[h] * NB))))
             qs[i, h] = s[h, k]
     return np.median(qs, axis=0).astype(np.float32)
+
+
+# --------------------------------------------------------------------------
+# GPU side (used by the -m gpu tests only)
+# --------------------------------------------------------------------------
+
+def gpu_decode(q_t, K_t, V_t, seq_lens, block_size, musig_bits, mnorm, tau=None, head_const=None, **params):
+    """Run eta_decode on cuda:0 with the given (oracle-built) summaries.
+
+    q_t, K_t, V_t: bf16 CPU tensors; musig_bits uint16 numpy; mnorm float32 numpy; tau/head_const float32 numpy.
+    -> out float32 numpy [B,Hq,d], sel uint8 numpy, stats, status
+    """
+    from paper_2609_20888_b200 import binding as eb
+    dev = torch.device("cuda:0")
+    K, V, q = K_t.to(dev), V_t.to(dev), q_t.to(dev)
+    st = eb.DecodeState(K, V, q_t.shape[1], block_size)
+    st.musig.copy_(torch.from_numpy(musig_bits.view(np.int16)).view(torch.float16).to(dev))
+    st.mnorm.copy_(torch.from_numpy(mnorm).to(dev))
+    lens = torch.from_numpy(np.asarray(seq_lens, np.int32)).to(dev)
+    tau_d = None if tau is None else torch.from_numpy(np.ascontiguousarray(tau, np.float32)).to(dev)
+    hc_d = None if head_const is None else torch.from_numpy(np.ascontiguousarray(head_const, np.float32)).to(dev)
+    p = eb.DecodeParams(**params)
+    st.out.fill_(float("nan"))
+    eb.eta_decode(st.desc, p, q, K, V, lens, st.musig, st.mnorm, tau_d, hc_d, st.out, st.sel_mask, st.workspace,
+                  stats=st.stats, status=st.status)
+    torch.cuda.synchronize()
+    return st.out.cpu().numpy(), st.sel_mask.cpu().numpy(), st.stats.cpu().numpy(), int(st.status.item())
+
+
+def compare_masks(sel_gpu, sel_ref, bound, tau_eff, seq_lens, b, G, band=1e-5, rescued=None):
+    """Selected-block sets must agree bit for bit except (head, block) pairs whose oracle bound lies within
+    `band` of tau_eff, which are returned (logged), and rescue choices made among bounds tied within `band`.
+
+    bound [B,Hq,NBcap] float64, tau_eff [B,Hq] float64.  -> list of near-tie mismatches (i, h, j, bound - tau_eff)
+    """
+    B, Hkv, NBcap = sel_ref.shape
+    near = []
+    diff = sel_gpu ^ sel_ref
+    for i, hk, j in zip(*np.nonzero(diff)):
+        NB = int(seq_lens[i]) // b
+        assert j < NB, f"mask bit set past the last full block: seq {i} kv head {hk} block {j}"
+        for g in range(G):
+            if (diff[i, hk, j] >> g) & 1:
+                h = hk * G + g
+                gap = float(bound[i, h, j] - tau_eff[i, h])
+                scale = max(1.0, abs(float(tau_eff[i, h])))
+                is_rescue_tie = False
+                if rescued is not None and rescued[i, h] >= 0:
+                    # the oracle rescued some block for this head: a different argmax is fine if the bounds tie
+                    is_rescue_tie = abs(float(bound[i, h, j] - bound[i, h, rescued[i, h]])) <= band * scale
+                assert abs(gap) <= band * scale or is_rescue_tie, \
+                    f"selection differs away from the threshold: seq {i} head {h} block {j} bound-tau={gap:.3e}"
+                near.append((int(i), int(h), int(j), gap))
+    return near
+
+
+def fp16_ulp_distance(a_bits, b_bits):
+    """Distance in units in the last place between fp16 bit patterns (sign-magnitude aware)."""
+    def key(x):
+        x = x.astype(np.int32)
+        return np.where(x & 0x8000, -(x & 0x7fff), x & 0x7fff)
+    return np.abs(key(a_bits) - key(b_bits))
+
+
+def output_errors(out_gpu, out_ref):
+    err = np.abs(out_gpu.astype(np.float64) - out_ref)
+    return float(err.max()), float(err.mean())
