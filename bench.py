@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the ETA block-sparse decode path on B200.
+
+One "step" = one decode step of one layer for a whole batch: tail-block summary update, threshold prediction,
+screening, streaming of the surviving K/V blocks, merge - six kernels of the library, all through the C ABI.
+Workload at N=1: the 128K-context configuration (batch 4, 32 query / 8 KV heads, head_dim 128, block 64,
+clustered keys), thresholds calibrated to 90% union block sparsity; the 50% / 97% points of the sweep and the
+dense baseline (same kernels, every block, gate off) are reported beside it.  Metric: decode queries per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched under torchrun) every rank runs an independent replica of the workload: the path is fixed
+to one GPU and has no exchange step, so scaling is weak by construction.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2609_20888_b200 import workloads as wl
+
+METRIC = "eta_decode_queries_per_s"
+UNIT = "queries/s"
+DEFAULT_WORKLOAD = "c3_128k"
+DEFAULT_TARGET = 0.90
+CALIB = os.path.join(ROOT, "tests", "golden", "workload_calibration.json")
+PEAKS = os.path.join(ROOT, "MEASURED_PEAKS.json")
+FALLBACK_HBM_GBS = 6650.0
+
+
+def load_bias(name: str, target: float) -> np.ndarray:
+    data = json.load(open(CALIB))
+    return np.asarray(data[name]["targets"][f"{target:.2f}"]["bias"], np.float32)
+
+
+def hbm_peak():
+    try:
+        return float(json.load(open(PEAKS))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self._stop = index, [], threading.Event()
+
+    def run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                parts = [p.strip() for p in out.strip().split(",")]
+                if len(parts) >= 6:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def stop(self) -> dict:
+        self._stop.set()
+        self.join(timeout=6)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        mhz = sorted(float(s[0]) for s in self.samples)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names) if any(s[2 + k].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": float(self.samples[0][1]), "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+def algorithmic_bytes(sp, lens, union_blocks: float):
+    """Bytes one step must move ('algorithmic bytes'): summaries of every full block, K and V of the
+    union of surviving blocks and of the tails, queries, thresholds, mask, output.  Split by kernel."""
+    d, b, G = sp.head_dim, sp.block_size, sp.gqa
+    nb = sum(int(t) // b for t in lens) * sp.n_kv_heads
+    tails = sum(int(t) % b for t in lens) * sp.n_kv_heads
+    screen = nb * (4 * d + 4) + nb + sp.batch * sp.n_q_heads * (2 * d + 4)
+    decode = union_blocks * 4 * b * d + tails * 4 * d + sp.batch * sp.n_q_heads * 2 * d
+    other = sp.batch * sp.n_q_heads * (2 * d + 4 * d) + sp.n_q_heads * d * sp.n_q_heads * 4
+    return {"screen": float(screen), "decode": float(decode), "total": float(screen + decode + other)}
+
+
+def run_ours(args):
+    from paper_2609_20888_b200 import binding as eb
+    from paper_2609_20888_b200 import build as ebuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        ebuild.build()
+    if world > 1:
+        dist.barrier()
+    eb.load()
+
+    sp = wl.CONFIGS[args.workload]
+    t0 = time.time()
+    w = wl.make_workload(sp, threads=min(16, len(os.sched_getaffinity(0))))
+    gen_s = time.time() - t0
+    Kd, Vd = w.K.to(dev), w.V.to(dev)
+    st = eb.DecodeState(Kd, Vd, sp.n_q_heads, sp.block_size)
+    lens = w.seq_lens.numpy().astype(np.int32)
+    lens_d = w.seq_lens.to(dev)
+    Wd = w.W.to(dev)
+
+    # prefill-side index build (once per sequence; timed on its own, not part of a decode step)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    eb.eta_build_block_summaries(st.desc, Kd, lens_d, st.musig, st.mnorm)
+    torch.cuda.synchronize()
+    ev0.record()
+    eb.eta_build_block_summaries(st.desc, Kd, lens_d, st.musig, st.mnorm)
+    ev1.record()
+    torch.cuda.synchronize()
+    build_ms = ev0.elapsed_time(ev1)
+    k_bytes = sum(int(t) // sp.block_size for t in lens) * sp.n_kv_heads * sp.block_size * sp.head_dim * 2
+
+    n_q = args.steps + args.warmup
+    q_host = [w.queries(s).pin_memory() for s in range(n_q)]
+    q_dev = [q.to(dev) for q in q_host]
+    out_host = torch.empty((sp.batch, sp.n_q_heads, sp.head_dim), dtype=torch.float32).pin_memory()
+    flush = torch.empty(384 << 20, dtype=torch.uint8, device=dev)     # > 126 MB of L2
+
+    def make_step(bias_np, flags=0):
+        bias_d = torch.from_numpy(bias_np).to(dev)
+        params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags,
+                                 ctas_per_sm=args.ctas_per_sm)
+
+        def step(qd):
+            eb.eta_append_summary(st.desc, Kd, lens_d, st.musig, st.mnorm)
+            eb.eta_predict_threshold(qd, Wd, bias_d, st.tau)
+            eb.eta_decode(st.desc, params, qd, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau, None, st.out,
+                          st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+        return step
+
+    def timed(step, sampler=None):
+        """W warm-up steps, then K steps each bracketed by CUDA events with an L2 flush in between."""
+        for s in range(args.warmup):
+            step(q_dev[s])
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.start()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        union = 0
+        wall0 = time.perf_counter()
+        for k in range(args.steps):
+            flush.fill_(k & 0xff)
+            evs[k][0].record()
+            step(q_dev[args.warmup + k])
+            evs[k][1].record()
+            union += 0        # stats are read after the region
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - wall0
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ms = [a.elapsed_time(b) for a, b in evs]
+        assert int(st.status.item()) == 0, "device status flagged a problem"
+        return ms, wall
+
+    def union_blocks_of(step):
+        tot = 0
+        for k in range(args.steps):
+            step(q_dev[args.warmup + k])
+            tot += int(st.stats.sum().item())
+        return tot / args.steps
+
+    def kernel_times(step):
+        eb.eta_profile_enable(True)
+        acc = {}
+        for k in range(args.steps):
+            flush.fill_(k & 0xff)
+            step(q_dev[args.warmup + k])
+            for name, v in eb.eta_profile_read().items():
+                acc[name] = acc.get(name, 0.0) + v
+        eb.eta_profile_enable(False)
+        return {k: v / args.steps for k, v in acc.items()}
+
+    targets = list(sp.target_sparsity)
+    main_target = DEFAULT_TARGET if DEFAULT_TARGET in targets else targets[0]
+    sampler = ClockSampler(local)
+    step_main = make_step(load_bias(sp.name, main_target))
+    ms_main, wall_main = timed(step_main, sampler)
+    clocks = sampler.stop()
+    ms_step = sum(ms_main) / len(ms_main)
+    if world > 1:
+        tt = torch.tensor([ms_step], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_step = float(tt.item())
+    union_main = union_blocks_of(step_main)
+    kt = kernel_times(step_main)
+    nb_total = sum(int(t) // sp.block_size for t in lens) * sp.n_kv_heads
+    ab = algorithmic_bytes(sp, lens, union_main)
+    peak, peak_kind = hbm_peak()
+    dec_s = kt["decode_kernel"] * 1e-3
+    achieved = ab["decode"] / dec_s / 1e9
+
+    # end to end: the query comes from pinned host memory and the output goes back to it, every step;
+    # each step is bracketed by events on the launching stream and followed by a host synchronise
+    dq = torch.empty_like(q_dev[0])
+    e2e_ms = 0.0
+    for k in range(args.steps):
+        flush.fill_(k & 0xff)
+        a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_ev.record()
+        dq.copy_(q_host[args.warmup + k], non_blocking=True)
+        step_main(dq)
+        out_host.copy_(st.out, non_blocking=True)
+        b_ev.record()
+        torch.cuda.synchronize()
+        e2e_ms += a_ev.elapsed_time(b_ev)
+    e2e_s = e2e_ms * 1e-3 / args.steps
+    if world > 1:
+        tt = torch.tensor([e2e_s], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_s = float(tt.item())
+
+    sweep = {}
+    if rank == 0 and world == 1 and not args.no_sweep:
+        for tgt in targets:
+            if tgt == main_target:
+                continue
+            stp = make_step(load_bias(sp.name, tgt))
+            ms, _ = timed(stp)
+            ub = union_blocks_of(stp)
+            abt = algorithmic_bytes(sp, lens, ub)
+            m = sum(ms) / len(ms)
+            sweep[f"{tgt:.2f}"] = {"ms_per_step": m, "union_sparsity": 1 - ub / nb_total,
+                                   "gbs_on_algorithmic_bytes": abt["total"] / (m * 1e-3) / 1e9}
+        stp = make_step(np.zeros(sp.n_q_heads, np.float32), flags=eb.ETA_FLAG_DENSE)
+        ms, _ = timed(stp)
+        m = sum(ms) / len(ms)
+        abt = algorithmic_bytes(sp, lens, nb_total)
+        sweep["dense_baseline"] = {"ms_per_step": m, "gbs_on_algorithmic_bytes": (abt["decode"]) / (m * 1e-3) / 1e9,
+                                   "speedup_of_main": m / ms_step}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(sp, w, load_bias(sp.name, main_target), budget_s=20.0)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": world * sp.batch / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": sp.name, "batch": sp.batch, "n_q_heads": sp.n_q_heads, "n_kv_heads": sp.n_kv_heads,
+                       "head_dim": sp.head_dim, "context": sp.context, "block_size": sp.block_size,
+                       "target_union_sparsity": main_target, "measured_union_sparsity": 1 - union_main / nb_total,
+                       "z": sp.z, "beta": sp.beta, "l2": "flushed between timed steps (384 MiB write)",
+                       "fresh_query_every_step": True, "replicas": world},
+            "attention_us_per_token": ms_step * 1e3,
+            "achieved_gbs_all_kernels": ab["total"] / (ms_step * 1e-3) / 1e9,
+            "frac_of_8tbs_nominal": ab["total"] / (ms_step * 1e-3) / 8e12,
+            "kernel_ms": kt,
+            "clocks": clocks,
+            "e2e": {"value": world * sp.batch / e2e_s, "unit": UNIT, "h2d_bytes_per_step": q_host[0].numel() * 2,
+                    "d2h_bytes_per_step": out_host.numel() * 4},
+            "gpu_launches": args.steps * (2 + eb.eta_decode_kernel_count()),
+            "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                         "algorithmic_bytes_per_launch": ab["decode"]},
+            "prefill_build": {"ms": build_ms, "gbs": k_bytes / (build_ms * 1e-3) / 1e9},
+            "sweep": sweep,
+            "cpu_baseline": cpu,
+            "setup_s": {"generate": round(gen_s, 1)},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(sp, w, bias, budget_s: float, steps: int | None = None):
+    """The oracle, as it stands, on this machine's host cores: whole decode steps (threshold prediction, bounds,
+    selection, gated attention over the admitted blocks) on the first sequence of the workload."""
+    from oracle import eta_oracle as orc
+    from tests.helpers import bits
+    orc.build()
+    nseq = 1
+    K, V = bits(w.K[:nseq]), bits(w.V[:nseq])
+    lens = w.seq_lens.numpy().astype(np.int32)[:nseq].copy()
+    c = orc.Cache(K, V, lens, sp.block_size)
+    musig, mnorm = orc.block_summaries(c)           # prefill-side, not timed (as on the GPU side)
+    times = []
+    t_all = time.perf_counter()
+    s = 0
+    while True:
+        q = bits(w.queries(s))[:nseq].copy()
+        t0 = time.perf_counter()
+        tau = orc.predict_threshold(q, w.W.numpy(), bias)
+        orc.decode_step(q, c, musig, mnorm, tau=tau.astype(np.float32), z=sp.z, beta=sp.beta, lwb=sp.lwb,
+                        rescue_window=sp.rescue_window)
+        times.append(time.perf_counter() - t0)
+        s += 1
+        if steps is not None:
+            if s >= steps:
+                break
+        elif time.perf_counter() - t_all > budget_s or s >= 64:
+            break
+    per = sum(times) / len(times)
+    return {"value": nseq / per, "unit": UNIT, "cores": orc.n_threads(), "kind": "oracle",
+            "sample": f"{len(times)} decode steps of sequence 0 of {sp.name} (1 of {sp.batch} sequences, all "
+                      f"{sp.n_q_heads} heads, full context)", "s_per_step": per}
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle on the host cores, same metric and configuration."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sp = wl.CONFIGS[args.workload]
+    w = wl.make_workload(sp, threads=min(16, len(os.sched_getaffinity(0))))
+    targets = list(sp.target_sparsity)
+    main_target = DEFAULT_TARGET if DEFAULT_TARGET in targets else targets[0]
+    bias = load_bias(sp.name, main_target)
+    cpu_baseline(sp, w, bias, 0.0, steps=max(1, args.warmup))
+    cpu = cpu_baseline(sp, w, bias, 0.0, steps=args.steps)
+    line = {"impl": "reference", "metric": METRIC, "value": cpu["value"], "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": cpu["s_per_step"] * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": sp.name, "batch": sp.batch, "n_q_heads": sp.n_q_heads, "n_kv_heads": sp.n_kv_heads,
+                       "head_dim": sp.head_dim, "context": sp.context, "block_size": sp.block_size,
+                       "target_union_sparsity": main_target},
+            "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": cpu["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.CONFIGS))
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

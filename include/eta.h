@@ -163,6 +163,17 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
 /* Number of kernels one eta_decode call launches (for launch accounting). */
 int eta_decode_kernel_count(void);
 
+/*
+ * Per-kernel timing of eta_decode (measurement aid; the paper has no counterpart).  While enabled, every
+ * eta_decode call records host-side CUDA events between its kernel launches on the call's stream;
+ * eta_profile_read waits for the most recent call to finish and writes the device time of each kernel in
+ * milliseconds to ms[0 .. count-1] (n >= eta_decode_kernel_count()), returning the count, or a negative status
+ * when no profiled call has been made.  Not thread-safe; leave disabled in production.
+ */
+int eta_profile_enable(int on);
+int eta_profile_read(float* ms, int n);
+const char* eta_profile_kernel_name(int k);
+
 /* Text for an eta_status. */
 const char* eta_strerror(int code);
 

@@ -20,7 +20,8 @@ ETA_BUILD_SIGMA_ENVELOPE = 1
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
 EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
-           "eta_score_dual", "eta_decode", "eta_decode_kernel_count", "eta_strerror", "eta_last_cuda_error")
+           "eta_score_dual", "eta_decode", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
+           "eta_profile_kernel_name", "eta_strerror", "eta_last_cuda_error")
 
 
 class CacheDesc(ctypes.Structure):
@@ -65,8 +66,13 @@ def load() -> ctypes.CDLL:
         lib.eta_strerror.restype = ctypes.c_char_p
         lib.eta_strerror.argtypes = [ctypes.c_int]
         lib.eta_last_cuda_error.restype = ctypes.c_char_p
+        lib.eta_profile_enable.argtypes = [ctypes.c_int]
+        lib.eta_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int]
+        lib.eta_profile_kernel_name.restype = ctypes.c_char_p
+        lib.eta_profile_kernel_name.argtypes = [ctypes.c_int]
         for name in EXPORTS:
-            if name not in ("eta_strerror", "eta_last_cuda_error", "eta_decode_kernel_count"):
+            if name not in ("eta_strerror", "eta_last_cuda_error", "eta_decode_kernel_count",
+                            "eta_profile_kernel_name"):
                 getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -176,6 +182,20 @@ def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau,
 
 def eta_decode_kernel_count() -> int:
     return load().eta_decode_kernel_count()
+
+
+def eta_profile_enable(on: bool) -> None:
+    _check(load().eta_profile_enable(1 if on else 0), "eta_profile_enable")
+
+
+def eta_profile_read() -> dict:
+    """Device time (ms) of each kernel of the most recent profiled eta_decode call, by kernel name."""
+    lib = load()
+    ms = (ctypes.c_float * 8)()
+    n = lib.eta_profile_read(ms, 8)
+    if n < 0:
+        _check(n, "eta_profile_read")
+    return {lib.eta_profile_kernel_name(k).decode(): float(ms[k]) for k in range(n)}
 
 
 class DecodeState:

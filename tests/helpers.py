@@ -75,8 +75,8 @@ def calibrate_bias(bound, tau_raw, seq_lens, b, G, target_union_sparsity):
         qs = np.empty((B, Hq))
         for i in range(B):
             NB = srt[i].shape[1]
-            k = min(NB - 1, max(0, int(np.floor((1.0 - rho) * NB))))
-            qs[i] = srt[i][:, k]
+            k = min(NB - 1, max(1, int(np.floor((1.0 - rho) * NB))))
+            qs[i] = 0.5 * (srt[i][:, k] + srt[i][:, k - 1])     # between two bounds, never exactly on one
         return np.median(qs - tau_raw, axis=0)
 
     lo, hi = 0.0, 1.0
@@ -99,8 +99,8 @@ def calibrate_head_const(bound, seq_lens, b, sparsity_levels):
         NB = int(seq_lens[i]) // b
         s = np.sort(bound[i, :, :NB], axis=1)
         for h in range(Hq):
-            k = min(NB - 1, max(0, int(np.floor(sparsity_levels[h] * NB))))
-            qs[i, h] = s[h, k]
+            k = min(NB - 1, max(1, int(np.floor(sparsity_levels[h] * NB))))
+            qs[i, h] = 0.5 * (s[h, k] + s[h, k - 1])
     return np.median(qs, axis=0).astype(np.float32)
 
 
