@@ -144,16 +144,48 @@ def run_ours(args):
     out_host = torch.empty((sp.batch, sp.n_q_heads, sp.head_dim), dtype=torch.float32).pin_memory()
     flush = torch.empty(384 << 20, dtype=torch.uint8, device=dev)     # > 126 MB of L2
 
+    static_q = torch.empty_like(q_dev[0])
+
     def make_step(bias_np, flags=0):
+        """One decode step on the query in `static_q`.  With --graph (default) the six launches are captured once
+        into a CUDA graph and replayed, so the host costs one graph launch per step instead of six kernel launches
+        through ctypes; the library calls are the same either way."""
         bias_d = torch.from_numpy(bias_np).to(dev)
         params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags,
                                  ctas_per_sm=args.ctas_per_sm)
 
-        def step(qd):
+        def launch(evs=None):
+            if evs:
+                evs[0].record()
             eb.eta_append_summary(st.desc, Kd, lens_d, st.musig, st.mnorm)
-            eb.eta_predict_threshold(qd, Wd, bias_d, st.tau)
-            eb.eta_decode(st.desc, params, qd, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau, None, st.out,
+            if evs:
+                evs[1].record()
+            eb.eta_predict_threshold(static_q, Wd, bias_d, st.tau)
+            if evs:
+                evs[2].record()
+            eb.eta_decode(st.desc, params, static_q, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau, None, st.out,
                           st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+
+        graph = None
+        if args.graph:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                static_q.copy_(q_dev[0])
+                for _ in range(2):
+                    launch()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                launch()
+
+        def step(qd, evs=None):
+            static_q.copy_(qd, non_blocking=True)
+            if graph is not None and evs is None:
+                graph.replay()
+            else:
+                launch(evs)
         return step
 
     def timed(step):
@@ -192,11 +224,14 @@ def run_ours(args):
     def kernel_times(step):
         eb.eta_profile_enable(True)
         acc = {}
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         for k in range(args.steps):
             flush.fill_(k & 0xff)
-            step(q_dev[args.warmup + k])
+            step(q_dev[args.warmup + k], evs=evs)
             for name, v in eb.eta_profile_read().items():
                 acc[name] = acc.get(name, 0.0) + v
+            acc["append_summary_kernel"] = acc.get("append_summary_kernel", 0.0) + evs[0].elapsed_time(evs[1])
+            acc["predict_threshold_kernel"] = acc.get("predict_threshold_kernel", 0.0) + evs[1].elapsed_time(evs[2])
         eb.eta_profile_enable(False)
         return {k: v / args.steps for k, v in acc.items()}
 
@@ -228,7 +263,7 @@ def run_ours(args):
         flush.fill_(k & 0xff)
         a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a_ev.record()
-        dq.copy_(q_host[args.warmup + k], non_blocking=True)
+        dq.copy_(q_host[args.warmup + k], non_blocking=True)      # host -> device, then the step reads it
         step_main(dq)
         out_host.copy_(st.out, non_blocking=True)
         b_ev.record()
@@ -252,14 +287,18 @@ def run_ours(args):
             ub = union_blocks_of(stp)
             abt = algorithmic_bytes(sp, lens, ub)
             m = sum(ms) / len(ms)
+            ktt = kernel_times(stp)
             sweep[f"{tgt:.2f}"] = {"ms_per_step": m, "union_sparsity": 1 - ub / nb_total,
-                                   "gbs_on_algorithmic_bytes": abt["total"] / (m * 1e-3) / 1e9}
+                                   "gbs_on_algorithmic_bytes": abt["total"] / (m * 1e-3) / 1e9, "kernel_ms": ktt,
+                                   "decode_kernel_gbs": abt["decode"] / (ktt["decode_kernel"] * 1e-3) / 1e9}
         stp = make_step(np.zeros(sp.n_q_heads, np.float32), flags=eb.ETA_FLAG_DENSE)
         ms, _ = timed(stp)
         m = sum(ms) / len(ms)
         abt = algorithmic_bytes(sp, lens, nb_total)
+        ktt = kernel_times(stp)
         sweep["dense_baseline"] = {"ms_per_step": m, "gbs_on_algorithmic_bytes": (abt["decode"]) / (m * 1e-3) / 1e9,
-                                   "speedup_of_main": m / ms_step}
+                                   "speedup_of_main": m / ms_step, "kernel_ms": ktt,
+                                   "decode_kernel_gbs": abt["decode"] / (ktt["decode_kernel"] * 1e-3) / 1e9}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -274,7 +313,7 @@ def run_ours(args):
                        "head_dim": sp.head_dim, "context": sp.context, "block_size": sp.block_size,
                        "target_union_sparsity": main_target, "measured_union_sparsity": 1 - union_main / nb_total,
                        "z": sp.z, "beta": sp.beta, "l2": "flushed between timed steps (384 MiB write)",
-                       "fresh_query_every_step": True, "replicas": world},
+                       "fresh_query_every_step": True, "replicas": world, "cuda_graph": bool(args.graph)},
             "attention_us_per_token": ms_step * 1e3,
             "achieved_gbs_all_kernels": ab["total"] / (ms_step * 1e-3) / 1e9,
             "frac_of_8tbs_nominal": ab["total"] / (ms_step * 1e-3) / 8e12,
@@ -361,6 +400,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.CONFIGS))
     ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch the kernels directly every step")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -46,7 +46,7 @@ WsLayout ws_layout(const eta_cache_desc* d) {
     L.pref = off;       off = align_up(off + sizeof(int32_t) * ((size_t)L.entries + 1), 256);
     L.cta_start = off;  off = align_up(off + sizeof(int4) * (size_t)MAX_CTAS, 256);
     L.tau_eff = off;    off = align_up(off + sizeof(float) * (size_t)d->batch * d->n_q_heads, 256);
-    size_t slots = (size_t)MAX_CTAS + L.rows;
+    size_t slots = ((size_t)MAX_CTAS + L.rows) * DECODE_GROUPS;
     L.part_ml = off;    off = align_up(off + sizeof(float2) * slots * G, 256);
     L.part_o = off;     off = align_up(off + sizeof(float) * slots * G * d->head_dim, 256);
     L.total = off;

@@ -26,8 +26,9 @@ int validate_desc(const eta_cache_desc* d);
 // LSTRIDE slots (SEG plus room for one rescued block per query head).
 constexpr int SEG = 64;
 constexpr int LSTRIDE = SEG + 8;
-constexpr int MAX_CTAS = 1024;       // upper bound on streaming CTAs (sizes the scratch)
+constexpr int MAX_CTAS = 256;        // upper bound on streaming CTAs (sizes the scratch; a B200 has 148 SMs)
 constexpr int MAX_ENTRIES = 49152;   // plan kernel keeps the unit prefix in shared memory
+constexpr int DECODE_GROUPS = 3;     // consumer groups per streaming CTA, each with its own partial per piece
 
 // Scratch layout (byte offsets from a 256-byte aligned base).
 struct WsLayout {
@@ -41,8 +42,8 @@ struct WsLayout {
     size_t pref;        // int32 [entries + 1] exclusive prefix of units per entry
     size_t cta_start;   // int4 [MAX_CTAS]: {u0, u1, first entry, 0}
     size_t tau_eff;     // float [batch * n_q_heads]
-    size_t part_ml;     // float2 [(MAX_CTAS + rows) * G]
-    size_t part_o;      // float [(MAX_CTAS + rows) * G * d]
+    size_t part_ml;     // float2 [(MAX_CTAS + rows) * DECODE_GROUPS * G]
+    size_t part_o;      // float [(MAX_CTAS + rows) * DECODE_GROUPS * G * d]
     size_t total;
 };
 WsLayout ws_layout(const eta_cache_desc* d);
@@ -79,6 +80,8 @@ struct PlanArgs {
     int32_t* hdr;
     int32_t* stats;
     uint32_t* status;
+    float2* part_ml;   // partial (m, l) slots, reset to "absent" before the streaming kernel runs
+    int n_part;
 };
 int launch_screen(const ScreenArgs& a, int rows, int D, int G, cudaStream_t s);
 int launch_plan(const PlanArgs& a, cudaStream_t s);

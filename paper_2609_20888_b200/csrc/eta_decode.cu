@@ -39,36 +39,45 @@ struct DecodeArgs {
     int Hq, Hkv, G, b, t_cap, nseg, entries;
 };
 
-constexpr uint32_t UF_FIRST = 1u, UF_LAST = 2u, UF_END = 4u;
-constexpr int N_CONSUMER_WARPS = 4;
-constexpr int DECODE_THREADS = 32 * (N_CONSUMER_WARPS + 1);
+constexpr uint32_t UF_END = 1u;
+constexpr int WARPS_PER_GROUP = 4;     // the four warps of a group each take a quarter of a tile's tokens
 
-// token row inside an 8-row group that MMA column n reads: bits 0 and 2 of n swapped, so that the two
-// rows a quarter-warp touches in one 16-byte load sit in different halves of the swizzle pattern
 __device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
     return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
 }
+// token row inside an 8-row group that MMA column n reads: bits 0 and 2 of n swapped, so that the two
+// rows a quarter-warp touches in one 16-byte load sit in different halves of the swizzle pattern
 __device__ __forceinline__ int rho(int n) { return (n & 2) | ((n & 1) << 2) | ((n >> 2) & 1); }
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
-template <int D, int TS, int NSTAGE>
+template <int D, int TS, int NSTAGE, int NGROUPS>
 struct DecodeSmem {
     static constexpr int HALVES = D / 64;
     static constexpr int TILE_BYTES = TS * 128;                 // one 64-column half tile
     static constexpr int STAGE_BYTES = 2 * HALVES * TILE_BYTES; // K halves then V halves
-    static constexpr int BAR_OFF = NSTAGE * STAGE_BYTES;        // full[NSTAGE], empty[NSTAGE], flush
-    static constexpr int DESC_OFF = BAR_OFF + 8 * (2 * NSTAGE + 2);
-    static constexpr int ML_OFF = DESC_OFF + 16 * NSTAGE;       // float m[4][8], l[4][8]
-    static constexpr int MO_OFF = ML_OFF + 4 * 2 * N_CONSUMER_WARPS * 8;
-    static size_t bytes(int G) { return 1024 + MO_OFF + sizeof(float) * N_CONSUMER_WARPS * G * D; }
+    static constexpr int BAR_OFF = NSTAGE * STAGE_BYTES;        // full[NSTAGE], empty[NSTAGE], flush[NGROUPS]
+    static constexpr int DESC_OFF = BAR_OFF + 8 * (2 * NSTAGE + NGROUPS + (NGROUPS & 1));
+    static constexpr int ML_OFF = DESC_OFF + 16 * NSTAGE;       // float m[NGROUPS][4][8], l[NGROUPS][4][8]
+    static constexpr int MO_OFF = ML_OFF + 4 * 2 * NGROUPS * WARPS_PER_GROUP * 8;
+    static size_t bytes(int G) { return 1024 + MO_OFF + sizeof(float) * NGROUPS * WARPS_PER_GROUP * G * D; }
 };
 
-template <int D, int TS, int NSTAGE>
-__global__ void __launch_bounds__(DECODE_THREADS, 1)
+// The streaming kernel.  Warp roles: NGROUPS consumer groups of four warps, then one producer warp.  Group k
+// consumes the stage fills k, k + NGROUPS, ...; with two or three groups every scheduler holds several warps in
+// different phases of a tile, which hides the fixed latencies of the MMA / shuffle / exp chains.  Each group
+// keeps its own running (m, l, O) and writes its own partial per (CTA, row) piece.
+template <int D, int TS, int NSTAGE, int NGROUPS>
+__global__ void __launch_bounds__(32 * (WARPS_PER_GROUP * NGROUPS + 1), 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DecodeArgs a) {
-    using L = DecodeSmem<D, TS, NSTAGE>;
+    using L = DecodeSmem<D, TS, NSTAGE, NGROUPS>;
     constexpr int HALVES = L::HALVES;
-    constexpr int WT = TS / N_CONSUMER_WARPS;   // tokens per consumer warp per tile (8 or 16)
+    constexpr int WT = TS / WARPS_PER_GROUP;    // tokens per consumer warp per tile (8 or 16)
     constexpr int NT = WT / 8;                  // 8-token MMA column tiles per warp
+    constexpr int PRODUCER_WARP = WARPS_PER_GROUP * NGROUPS;
     static_assert(NT == 1 || NT == 2, "tile must give each warp 8 or 16 tokens");
 
     extern __shared__ unsigned char smem_raw[];
@@ -77,9 +86,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     uint64_t* empty = full + NSTAGE;
     uint64_t* flushbar = empty + NSTAGE;
     int4* desc = reinterpret_cast<int4*>(smem + L::DESC_OFF);
-    float* sm_m = reinterpret_cast<float*>(smem + L::ML_OFF);
-    float* sm_l = sm_m + N_CONSUMER_WARPS * 8;
-    float* sm_o = reinterpret_cast<float*>(smem + L::MO_OFF);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int4 cs = a.cta_start[blockIdx.x];
@@ -87,21 +93,22 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     if (u0 >= u1) return;
 
     if (tid == 0) {
-        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], N_CONSUMER_WARPS); }
-        mbar_init(&flushbar[0], 32 * N_CONSUMER_WARPS);
+        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], WARPS_PER_GROUP); }
+        for (int k = 0; k < NGROUPS; ++k) mbar_init(&flushbar[k], 32 * WARPS_PER_GROUP);
         fence_barrier_init();
         prefetch_tmap(&tmK);
         prefetch_tmap(&tmV);
     }
     __syncthreads();
 
-    if (warp == N_CONSUMER_WARPS) {
+    if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
         const int EPR = a.nseg + 1;
         const int E = a.entries;
         int e = cs.z;
         int u = u0;
         uint32_t fill = 0;
+        int piece = -1;
         bool ok = true;
         while (u < u1 && ok) {
             // entry holding unit u: pref[e] <= u < pref[e+1]; skip empty entries 32 at a time
@@ -113,10 +120,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 if (e >= E) { ok = false; break; }     // inconsistent plan: stop instead of walking off
             }
             if (!ok) break;
-            const int pe = __ldg(a.pref + e), pn = __ldg(a.pref + e + 1);
             const int r = e / EPR, sg = e % EPR;
-            const int row_begin = __ldg(a.pref + r * EPR), row_end = __ldg(a.pref + (r + 1) * EPR);
             const int i = r / a.Hkv, hk = r % a.Hkv;
+            const int pe = __ldg(a.pref + e), pn = __ldg(a.pref + e + 1);
+            const int row_begin = __ldg(a.pref + r * EPR);
             int T = __ldg(a.seq_lens + i);
             T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
             const int NB = T / a.b, tail = T - NB * a.b;
@@ -134,20 +141,16 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     const int j = ent & 0xffffff;
                     const int hmask = (ent >> 24) & 0xff;
                     const int nrows = is_tail ? tail : a.b;
-                    const bool first = (uu == u0) || (uu == row_begin);
-                    const bool last = (uu == u1 - 1) || (uu == row_end - 1);
+                    if (uu == u0 || uu == row_begin) ++piece;      // a new (CTA, row) piece starts here
                     for (int sub = 0; sub * TS < nrows && ok; ++sub) {
                         const int nvalid = min(TS, nrows - sub * TS);
-                        const bool last_sub = (sub + 1) * TS >= nrows;
                         const int stage = fill % NSTAGE;
                         const uint32_t round = fill / NSTAGE;
                         if (lane == 0) {
                             if (!mbar_wait(&empty[stage], (round & 1) ^ 1)) {
                                 ok = false;
                             } else {
-                                uint32_t fl = (first && sub == 0 ? UF_FIRST : 0u) | (last && last_sub ? UF_LAST : 0u) |
-                                              (uu == u1 - 1 && last_sub ? UF_END : 0u);
-                                desc[stage] = make_int4(r, (int)fl, hmask, nvalid);
+                                desc[stage] = make_int4(r, piece << 1, hmask, nvalid);
                                 unsigned char* st = smem + stage * L::STAGE_BYTES;
                                 mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
                                 const int y = j * a.b + sub * TS;
@@ -165,6 +168,20 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
             u += n_here;
         }
+        // one end marker per group (no data): the next NGROUPS fills reach every group exactly once
+        for (int k = 0; k < NGROUPS && ok; ++k) {
+            const int stage = fill % NSTAGE;
+            if (lane == 0) {
+                if (!mbar_wait(&empty[stage], ((fill / NSTAGE) & 1) ^ 1)) {
+                    ok = false;
+                } else {
+                    desc[stage] = make_int4(0, (int)UF_END, 0, 0);
+                    mbar_arrive(&full[stage]);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            ++fill;
+        }
         if (!ok) {
             // give up: report, then let copies already issued land before the CTA's shared memory is released
             if (lane == 0) {
@@ -177,32 +194,96 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
 
     // ---------------------------------------------------------------- consumers
+    const int group = warp / WARPS_PER_GROUP, wq = warp % WARPS_PER_GROUP;
+    float* sm_m = reinterpret_cast<float*>(smem + L::ML_OFF) + group * 2 * WARPS_PER_GROUP * 8;
+    float* sm_l = sm_m + WARPS_PER_GROUP * 8;
+    float* sm_o = reinterpret_cast<float*>(smem + L::MO_OFF) + group * WARPS_PER_GROUP * a.G * D;
+    const int gtid = tid - group * 32 * WARPS_PER_GROUP;    // thread index inside the group
     const int g = lane >> 2, t = lane & 3;
-    const int rb = warp * WT;                          // first token row of this warp inside a tile
+    const int rb = wq * WT;                            // first token row of this warp inside a tile
     const int r0 = rho(2 * t), r1 = rho(2 * t + 1);    // token rows (within an 8-group) of MMA columns 2t, 2t+1
     const int vchunk = ((g & 1) << 2) | (g >> 1);      // 16-byte chunk of a V half-row this lane reads
     const float LOG2E = 1.4426950408889634f;
+    const bool head = g < a.G;
+
+    // byte offsets inside a half tile of the 16-byte pieces this lane reads (fixed for the whole kernel)
+    uint32_t koff[NT][2], voff[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int krow = rb + nt * 8 + rho(g);
+#pragma unroll
+        for (int m = 0; m < 2; ++m) koff[nt][m] = krow * 128 + (((4 * m + t) ^ (krow & 7)) << 4);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            const int vrow = rb + nt * 8 + (c ? r1 : r0);
+            voff[nt][c] = vrow * 128 + ((vchunk ^ (vrow & 7)) << 4);
+        }
+    }
 
     uint32_t qa[HALVES][2][4];
     float o[HALVES][4][4];
     float m_run = -INFINITY, l_run = 0.f, te = 0.f;
-    int row = -1;
+    int row = -1, piece = -1;
     uint32_t flush_phase = 0;
     bool ok = true;
 
-    for (uint32_t fill = 0;; ++fill) {
+    for (uint32_t fill = group;; fill += NGROUPS) {
         const int stage = fill % NSTAGE;
         if (!mbar_wait(&full[stage], (fill / NSTAGE) & 1)) { ok = false; break; }
         const int4 ds = desc[stage];
-        const uint32_t fl = (uint32_t)ds.y;
+        const bool end = (ds.y & (int)UF_END) != 0;
+        const int new_piece = ds.y >> 1;
+
+        if ((end || new_piece != piece) && piece >= 0) {
+            // ---- this group's part of a piece is complete: combine its four warps and store (m, l, O) per head
+            float lsum = l_run + __shfl_xor_sync(0xffffffffu, l_run, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            if (t == 0) { sm_m[wq * 8 + g] = m_run; sm_l[wq * 8 + g] = lsum; }
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) {
+                    const int dcol = 64 * hf + 8 * vchunk + 2 * mt;
+                    if (2 * t < a.G)
+                        *reinterpret_cast<float2*>(sm_o + ((wq * a.G + 2 * t) * D + dcol)) = make_float2(o[hf][mt][0], o[hf][mt][2]);
+                    if (2 * t + 1 < a.G)
+                        *reinterpret_cast<float2*>(sm_o + ((wq * a.G + 2 * t + 1) * D + dcol)) = make_float2(o[hf][mt][1], o[hf][mt][3]);
+                }
+            mbar_arrive(&flushbar[group]);
+            if (!mbar_wait(&flushbar[group], flush_phase)) { ok = false; break; }
+            flush_phase ^= 1;
+            const int64_t slot = ((int64_t)blockIdx.x + row) * NGROUPS + group;
+            for (int idx = gtid; idx < a.G * D; idx += 32 * WARPS_PER_GROUP) {
+                const int hh = idx / D, dd = idx % D;
+                float M = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < WARPS_PER_GROUP; ++w) M = fmaxf(M, sm_m[w * 8 + hh]);
+                float acc = 0.f, lacc = 0.f;
+                if (M != -INFINITY) {
+#pragma unroll
+                    for (int w = 0; w < WARPS_PER_GROUP; ++w) {
+                        const float sc = exp2f((sm_m[w * 8 + hh] - M) * LOG2E);
+                        acc = fmaf(sm_o[(w * a.G + hh) * D + dd], sc, acc);
+                        lacc = fmaf(sm_l[w * 8 + hh], sc, lacc);
+                    }
+                }
+                a.part_o[(slot * a.G + hh) * D + dd] = acc;
+                if (dd == 0) a.part_ml[slot * a.G + hh] = make_float2(M, lacc);
+            }
+            mbar_arrive(&flushbar[group]);
+            if (!mbar_wait(&flushbar[group], flush_phase)) { ok = false; break; }
+            flush_phase ^= 1;
+        }
+        if (end) break;
+
         const int hmask = ds.z, nvalid = ds.w;
         const uint32_t kbase = smem_u32(smem + stage * L::STAGE_BYTES);
         const uint32_t vbase = kbase + HALVES * L::TILE_BYTES;
 
-        if (fl & UF_FIRST) {
+        if (new_piece != piece) {
+            piece = new_piece;
             row = ds.x;
             const int i = row / a.Hkv, hk = row % a.Hkv;
-            const bool head = g < a.G;
             const __nv_bfloat16* qp = a.q + ((int64_t)i * a.Hq + hk * a.G + (head ? g : 0)) * D;
 #pragma unroll
             for (int hf = 0; hf < HALVES; ++hf)
@@ -229,30 +310,49 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int c = 0; c < 4; ++c) sacc[nt][c] = 0.f;
+        {
+            uint4 kv[HALVES][2][NT];
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int m = 0; m < 2; ++m)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) kv[hf][m][nt] = lds128(kbase + hf * L::TILE_BYTES + koff[nt][m]);
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int m = 0; m < 2; ++m)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        mma_bf16_16816(sacc[nt], qa[hf][m][0], 0u, qa[hf][m][1], 0u, kv[hf][m][nt].x, kv[hf][m][nt].y);
+                        mma_bf16_16816(sacc[nt], qa[hf][m][2], 0u, qa[hf][m][3], 0u, kv[hf][m][nt].z, kv[hf][m][nt].w);
+                    }
+        }
+        // V pieces are requested now so that their latency hides behind the softmax arithmetic
+        uint4 v[HALVES][2 * NT];
 #pragma unroll
         for (int hf = 0; hf < HALVES; ++hf)
 #pragma unroll
-            for (int m = 0; m < 2; ++m)
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int trow = rb + nt * 8 + rho(g);
-                    const uint4 kv = lds128(kbase + hf * L::TILE_BYTES + trow * 128 + ((((4 * m + t) ^ (trow & 7))) << 4));
-                    mma_bf16_16816(sacc[nt], qa[hf][m][0], 0u, qa[hf][m][1], 0u, kv.x, kv.y);
-                    mma_bf16_16816(sacc[nt], qa[hf][m][2], 0u, qa[hf][m][3], 0u, kv.z, kv.w);
-                }
+                for (int c = 0; c < 2; ++c) v[hf][nt * 2 + c] = lds128(vbase + hf * L::TILE_BYTES + voff[nt][c]);
 
         // ---- gate, mask, online softmax (lane (g,t) holds head g, tokens r0/r1 of each 8-group)
-        const bool head_on = (g < a.G) && ((hmask >> g) & 1);
+        const bool head_on = head && ((hmask >> g) & 1);
         float sg[NT][2];
         float bmax = -INFINITY;
+        const bool gate_on = (te != -INFINITY);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int trow = rb + nt * 8 + (c ? r1 : r0);
                 const float S = sacc[nt][c] * a.scale;
-                const float x = (a.beta == 0.f) ? 0.f : a.beta * (S - te);
-                float gated = (te == -INFINITY) ? S : S / (1.f + __expf(-x));
+                float gated = S;
+                if (gate_on) {
+                    const float x = (a.beta == 0.f) ? 0.f : a.beta * (S - te);
+                    gated = S * rcp_approx(1.f + exp2f(-x * LOG2E));      // S * sigmoid(x); exp2(+inf) -> rcp -> 0
+                }
                 gated = (head_on && trow < nvalid) ? gated : -INFINITY;
                 sg[nt][c] = gated;
                 bmax = fmaxf(bmax, gated);
@@ -274,9 +374,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         m_run = m_new;
 
         // accumulators hold heads 2t, 2t+1 in their columns: fetch those heads' rescale factors
-        const float al0 = __shfl_sync(0xffffffffu, alpha, 8 * t);
-        const float al1 = __shfl_sync(0xffffffffu, alpha, 8 * t + 4);
         if (__any_sync(0xffffffffu, alpha != 1.f)) {
+            const float al0 = __shfl_sync(0xffffffffu, alpha, 8 * t);
+            const float al1 = __shfl_sync(0xffffffffu, alpha, 8 * t + 4);
 #pragma unroll
             for (int hf = 0; hf < HALVES; ++hf)
 #pragma unroll
@@ -297,26 +397,29 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
 
         // ---- O^T += V^T P : head_dim on M, tokens on K, heads on N
-        const bool partial = nvalid < TS;
+        if (nvalid < TS) {
+            // rows past the end of the sequence hold whatever the cache holds: keep them out of the product
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+                        if (rb + nt * 8 + (c ? r1 : r0) >= nvalid) v[hf][nt * 2 + c] = make_uint4(0, 0, 0, 0);
+        }
+        // every shared-memory read of this stage has been issued before this point; the arrive (release) orders
+        // them before the producer's next copy into the stage
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[stage]);
 #pragma unroll
         for (int hf = 0; hf < HALVES; ++hf) {
-            uint4 v[2 * NT];
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    const int trow = rb + nt * 8 + (c ? r1 : r0);
-                    uint4 x = lds128(vbase + hf * L::TILE_BYTES + trow * 128 + ((vchunk ^ (trow & 7)) << 4));
-                    if (partial && trow >= nvalid) x = make_uint4(0, 0, 0, 0);   // rows past the sequence end
-                    v[nt * 2 + c] = x;
-                }
 #pragma unroll
             for (int mt = 0; mt < 4; ++mt) {
-                const uint32_t xa = u4_get(v[0], mt), xb = u4_get(v[1], mt);
+                const uint32_t xa = u4_get(v[hf][0], mt), xb = u4_get(v[hf][1], mt);
                 const uint32_t a0 = __byte_perm(xa, xb, 0x5410), a1 = __byte_perm(xa, xb, 0x7632);
                 uint32_t a2 = 0u, a3 = 0u;
                 if (NT == 2) {
-                    const uint32_t xc = u4_get(v[2 * (NT - 1)], mt), xd = u4_get(v[2 * (NT - 1) + 1], mt);
+                    const uint32_t xc = u4_get(v[hf][2 * (NT - 1)], mt), xd = u4_get(v[hf][2 * (NT - 1) + 1], mt);
                     a2 = __byte_perm(xc, xd, 0x5410);
                     a3 = __byte_perm(xc, xd, 0x7632);
                 }
@@ -325,51 +428,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
         }
 
-        // this warp is done with the stage
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[stage]);
-
-        if (fl & UF_LAST) {
-            // ---- piece finished: combine the four warps' partials and store one (m, l, O) per head
-            float lsum = l_run + __shfl_xor_sync(0xffffffffu, l_run, 1);
-            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
-            if (t == 0) { sm_m[warp * 8 + g] = m_run; sm_l[warp * 8 + g] = lsum; }
-#pragma unroll
-            for (int hf = 0; hf < HALVES; ++hf)
-#pragma unroll
-                for (int mt = 0; mt < 4; ++mt) {
-                    const int dcol = 64 * hf + 8 * vchunk + 2 * mt;
-                    if (2 * t < a.G)
-                        *reinterpret_cast<float2*>(sm_o + ((warp * a.G + 2 * t) * D + dcol)) = make_float2(o[hf][mt][0], o[hf][mt][2]);
-                    if (2 * t + 1 < a.G)
-                        *reinterpret_cast<float2*>(sm_o + ((warp * a.G + 2 * t + 1) * D + dcol)) = make_float2(o[hf][mt][1], o[hf][mt][3]);
-                }
-            mbar_arrive(&flushbar[0]);
-            if (!mbar_wait(&flushbar[0], flush_phase)) { ok = false; break; }
-            flush_phase ^= 1;
-            const int slot = blockIdx.x + row;
-            for (int idx = tid; idx < a.G * D; idx += 32 * N_CONSUMER_WARPS) {
-                const int hh = idx / D, dd = idx % D;
-                float M = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < N_CONSUMER_WARPS; ++w) M = fmaxf(M, sm_m[w * 8 + hh]);
-                float acc = 0.f, lacc = 0.f;
-                if (M != -INFINITY) {
-#pragma unroll
-                    for (int w = 0; w < N_CONSUMER_WARPS; ++w) {
-                        const float sc = exp2f((sm_m[w * 8 + hh] - M) * LOG2E);
-                        acc = fmaf(sm_o[(w * a.G + hh) * D + dd], sc, acc);
-                        lacc = fmaf(sm_l[w * 8 + hh], sc, lacc);
-                    }
-                }
-                a.part_o[((int64_t)slot * a.G + hh) * D + dd] = acc;
-                if (dd == 0) a.part_ml[(int64_t)slot * a.G + hh] = make_float2(M, lacc);
-            }
-            mbar_arrive(&flushbar[0]);
-            if (!mbar_wait(&flushbar[0], flush_phase)) { ok = false; break; }
-            flush_phase ^= 1;
-        }
-        if (fl & UF_END) break;
     }
     if (!ok && lane == 0 && a.status) atomicOr(a.status, ETA_DEV_TIMEOUT);
 }
@@ -381,48 +439,100 @@ struct MergeArgs {
     const float2* part_ml;
     const float* part_o;
     float* out;
-    int Hq, Hkv, G, nseg, rows;
+    int Hq, Hkv, G, nseg, rows, ngroups;
 };
 
+constexpr int MERGE_WARPS = 8;
+
+// One CTA per (row, query head).  Every warp reads the (m, l) of all candidate parts (lanes in parallel) and
+// takes the largest m; warp w then weighs and adds the O of parts w, w + 8, ... (all of its loads in flight at
+// once), and the eight warp sums are added in a fixed order:
+//   o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
 template <int D>
-__global__ void __launch_bounds__(128) merge_kernel(const MergeArgs a) {
-    const int wid = blockIdx.x * 4 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (wid >= a.rows * a.G) return;
-    const int r = wid / a.G, gq = wid % a.G;
+__global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs a) {
+    constexpr int VPL = D / 32;
+    __shared__ float s_acc[MERGE_WARPS][D];
+    __shared__ float s_l[MERGE_WARPS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
     const int EPR = a.nseg + 1;
     const int ra = a.pref[r * EPR], rbd = a.pref[(r + 1) * EPR];
     const int64_t U = a.hdr[0], P = a.hdr[1];
-    constexpr int VPL = D / 32;
     float acc[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
-    float mg = -INFINITY, lg = 0.f;
+    float lw_sum = 0.f;
     if (rbd > ra && U > 0) {
+        // streaming CTAs whose unit range meets this row's range [ra, rbd): a superset, then tested exactly
         int c_lo = (int)(((int64_t)ra * P) / U) - 1;
         int c_hi = (int)(((int64_t)rbd * P + U - 1) / U) + 1;
         c_lo = c_lo < 0 ? 0 : c_lo;
         c_hi = c_hi > (int)P - 1 ? (int)P - 1 : c_hi;
-        for (int c = c_lo; c <= c_hi; ++c) {
-            const int cu0 = (int)(((int64_t)c * U) / P), cu1 = (int)(((int64_t)(c + 1) * U) / P);
-            if (max(cu0, ra) >= min(cu1, rbd)) continue;
-            const int64_t slot = (int64_t)c + r;
-            const float2 ml = a.part_ml[slot * a.G + gq];
-            if (ml.x == -INFINITY) continue;
-            const float mn = fmaxf(mg, ml.x);
-            const float ag = __expf(mg - mn), ac = __expf(ml.x - mn);
-            const float* po = a.part_o + (slot * a.G + gq) * D + lane * VPL;
-            lg = lg * ag + ml.y * ac;
+        const int n_cand = (c_hi - c_lo + 1) * a.ngroups;
+        float mg = -INFINITY;
+        for (int k0 = 0; k0 < n_cand; k0 += 32) {
+            const int k = k0 + lane;
+            if (k < n_cand) {
+                const int c = c_lo + k / a.ngroups;
+                const int cu0 = (int)(((int64_t)c * U) / P), cu1 = (int)(((int64_t)(c + 1) * U) / P);
+                if (max(cu0, ra) < min(cu1, rbd)) {
+                    const int64_t slot = ((int64_t)c + r) * a.ngroups + k % a.ngroups;
+                    mg = fmaxf(mg, a.part_ml[slot * a.G + gq].x);
+                }
+            }
+        }
 #pragma unroll
-            for (int k = 0; k < VPL; ++k) acc[k] = acc[k] * ag + po[k] * ac;
-            mg = mn;
+        for (int s = 16; s >= 1; s >>= 1) mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, s));
+        if (mg != -INFINITY) {
+            // this warp's parts, four at a time
+            for (int k0 = warp; k0 < n_cand; k0 += 4 * MERGE_WARPS) {
+                float wv[4];
+                float xv[4][VPL];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int k = k0 + u * MERGE_WARPS;
+                    wv[u] = 0.f;
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) xv[u][v] = 0.f;
+                    if (k < n_cand) {
+                        const int c = c_lo + k / a.ngroups;
+                        const int cu0 = (int)(((int64_t)c * U) / P), cu1 = (int)(((int64_t)(c + 1) * U) / P);
+                        if (max(cu0, ra) < min(cu1, rbd)) {
+                            const int64_t slot = ((int64_t)c + r) * a.ngroups + k % a.ngroups;
+                            const float2 ml = a.part_ml[slot * a.G + gq];
+                            if (ml.x != -INFINITY) {     // cleared by the plan step and never written: no such part
+                                wv[u] = __expf(ml.x - mg);
+                                lw_sum = fmaf(ml.y, wv[u], lw_sum);
+                                const float* po = a.part_o + (slot * a.G + gq) * D + lane * VPL;
+                                if (VPL == 4) {
+                                    const float4 x = __ldg(reinterpret_cast<const float4*>(po));
+                                    xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
+                                } else {
+                                    const float2 x = __ldg(reinterpret_cast<const float2*>(po));
+                                    xv[u][0] = x.x; xv[u][1] = x.y;
+                                }
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) acc[v] = fmaf(xv[u][v], wv[u], acc[v]);
+            }
         }
     }
-    float* op = a.out + ((int64_t)i * a.Hq + hk * a.G + gq) * D + lane * VPL;
-    const float inv = lg > 0.f ? 1.f / lg : 0.f;
 #pragma unroll
-    for (int k = 0; k < VPL; ++k) op[k] = acc[k] * inv;
+    for (int v = 0; v < VPL; ++v) s_acc[warp][lane * VPL + v] = acc[v];
+    if (lane == 0) s_l[warp] = lw_sum;      // every lane of a warp holds the same sum
+    __syncthreads();
+    if (threadIdx.x < D) {
+        float o = 0.f, l = 0.f;
+#pragma unroll
+        for (int w = 0; w < MERGE_WARPS; ++w) { o += s_acc[w][threadIdx.x]; l += s_l[w]; }
+        a.out[((int64_t)i * a.Hq + hk * a.G + gq) * D + threadIdx.x] = l > 0.f ? o / l : 0.f;
+    }
 }
 
 // ------------------------------------------------------------------ host side
@@ -465,18 +575,18 @@ static int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d,
     return ETA_OK;
 }
 
-template <int D, int TS, int NSTAGE>
+template <int D, int TS, int NSTAGE, int NGROUPS>
 static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const DecodeArgs& a, int n_ctas,
                            cudaStream_t s) {
-    const size_t smem = DecodeSmem<D, TS, NSTAGE>::bytes(a.G);
+    const size_t smem = DecodeSmem<D, TS, NSTAGE, NGROUPS>::bytes(a.G);
     static size_t configured = 0;
     if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, TS, NSTAGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, TS, NSTAGE, NGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
         if (e != cudaSuccess) { set_cuda_error(e, "decode smem attribute"); return ETA_ERR_CUDA; }
         configured = smem;
     }
-    decode_kernel<D, TS, NSTAGE><<<n_ctas, DECODE_THREADS, smem, s>>>(tmK, tmV, a);
+    decode_kernel<D, TS, NSTAGE, NGROUPS><<<n_ctas, 32 * (WARPS_PER_GROUP * NGROUPS + 1), smem, s>>>(tmK, tmV, a);
     return check_launch("decode");
 }
 
@@ -553,10 +663,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     if (ce != cudaSuccess) { set_cuda_error(ce, "device query"); return ETA_ERR_CUDA; }
     const int TS = b < 64 ? b : 64;
-    int per_sm = params->ctas_per_sm > 0 ? params->ctas_per_sm : 1;
-    if (per_sm > 2) per_sm = 2;
-    if (!(D == 128 && TS == 64) || G == 8) per_sm = 1;
-    int n_ctas = n_sm * per_sm;
+    int n_ctas = n_sm;                  // one persistent CTA per SM; the shared-memory ring fills the SM
     if (n_ctas > MAX_CTAS) n_ctas = MAX_CTAS;
 
     ScreenArgs sa;
@@ -591,6 +698,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     pa.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
     pa.stats = stats;
     pa.status = status_dev;
+    pa.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
+    pa.n_part = (n_ctas + L.rows) * DECODE_GROUPS * G;
     rc = launch_plan(pa, s);
     if (rc != ETA_OK) return rc;
     profile_mark(2, s);
@@ -611,24 +720,24 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.Hq = desc->n_q_heads; da.Hkv = desc->n_kv_heads; da.G = G; da.b = b; da.t_cap = desc->t_cap;
     da.nseg = L.nseg; da.entries = L.entries;
     if (D == 128 && TS == 64) {
-        rc = (per_sm == 2) ? launch_decode_t<128, 64, 3>(tmK, tmV, da, n_ctas, s)
-                           : launch_decode_t<128, 64, 6>(tmK, tmV, da, n_ctas, s);
+        rc = (G == 8) ? launch_decode_t<128, 64, 5, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s)
+                      : launch_decode_t<128, 64, 6, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s);
     } else if (D == 128 && TS == 32) {
-        rc = launch_decode_t<128, 32, 8>(tmK, tmV, da, n_ctas, s);
+        rc = launch_decode_t<128, 32, 8, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s);
     } else if (D == 64 && TS == 64) {
-        rc = launch_decode_t<64, 64, 8>(tmK, tmV, da, n_ctas, s);
+        rc = launch_decode_t<64, 64, 8, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s);
     } else {
-        rc = launch_decode_t<64, 32, 8>(tmK, tmV, da, n_ctas, s);
+        rc = launch_decode_t<64, 32, 8, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s);
     }
     if (rc != ETA_OK) return rc;
     profile_mark(3, s);
 
     MergeArgs ma;
     ma.pref = pa.pref; ma.hdr = pa.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
-    ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows;
-    const unsigned mgrid = (unsigned)((L.rows * G + 3) / 4);
-    if (D == 128) merge_kernel<128><<<mgrid, 128, 0, s>>>(ma);
-    else merge_kernel<64><<<mgrid, 128, 0, s>>>(ma);
+    ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS;
+    const unsigned mgrid = (unsigned)(L.rows * G);
+    if (D == 128) merge_kernel<128><<<mgrid, 32 * MERGE_WARPS, 0, s>>>(ma);
+    else merge_kernel<64><<<mgrid, 32 * MERGE_WARPS, 0, s>>>(ma);
     profile_mark(4, s);
     return check_launch("merge");
 }

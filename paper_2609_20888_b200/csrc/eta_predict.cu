@@ -1,48 +1,68 @@
 // Threshold predictor, Eq. tau_pred: tau = qbar W + bias with qbar the
 // head-major concatenation of the post-RoPE query heads of one sequence.
 //
-// One CTA per sequence.  Thread (rg, h) accumulates column h of W over the rows
-// r = rg, rg + NRG, ... so that a warp reads whole rows of W (coalesced), then
-// the NRG partial sums of a column are added in a fixed order: the result does
-// not depend on scheduling.
+// W is small (n_q_heads^2 * head_dim floats) but a decode step waits for tau, so
+// the kernel is built for latency, not bandwidth: the rows of W are split over
+// the CTAs of a thread-block cluster (one cluster per sequence) so that no SM
+// reads more than 1/8 of W and every thread has all of its loads in flight at
+// once; the per-CTA partial sums meet in the shared memory of the cluster's
+// first CTA and are added there in a fixed order, so the result does not depend
+// on scheduling.
+#include <cooperative_groups.h>
+
 #include "eta_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace eta {
 
-constexpr int PRED_THREADS = 1024;
+constexpr int PRED_THREADS = 512;
+constexpr int PRED_CLUSTER = 8;
 
 __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     const __nv_bfloat16* __restrict__ q, const float* __restrict__ W, const float* __restrict__ bias,
     float* __restrict__ tau, int Hq, int rows) {
     extern __shared__ float sm[];
-    float* qs = sm;                 // [rows] the concatenated query in fp32
-    float* part = sm + rows;        // [NRG][Hq]
-    const int i = blockIdx.x;
+    const int NRG = PRED_THREADS / Hq;           // row groups inside a CTA
+    float* part = sm;                            // [NRG][Hq] partial sums of this CTA
+    float* cpart = sm + NRG * Hq;                // [PRED_CLUSTER][Hq], used in the cluster's first CTA
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank();
+    const int i = blockIdx.y;
+    const int per_cta = (rows + PRED_CLUSTER - 1) / PRED_CLUSTER;
+    const int r_begin = crank * per_cta, r_end = min(rows, r_begin + per_cta);
     const __nv_bfloat16* qi = q + (int64_t)i * rows;
-    for (int r = threadIdx.x; r < rows; r += PRED_THREADS) qs[r] = __bfloat162float(qi[r]);
-    __syncthreads();
-    const int NRG = PRED_THREADS / Hq;
     const int h = threadIdx.x % Hq, rg = threadIdx.x / Hq;
-    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+
+    float acc = 0.f;
     if (rg < NRG) {
-        int r = rg;
-        for (; r + 3 * NRG < rows; r += 4 * NRG) {
-            float w0 = __ldg(W + (int64_t)r * Hq + h);
-            float w1 = __ldg(W + (int64_t)(r + NRG) * Hq + h);
-            float w2 = __ldg(W + (int64_t)(r + 2 * NRG) * Hq + h);
-            float w3 = __ldg(W + (int64_t)(r + 3 * NRG) * Hq + h);
-            acc0 = fmaf(qs[r], w0, acc0);
-            acc1 = fmaf(qs[r + NRG], w1, acc1);
-            acc2 = fmaf(qs[r + 2 * NRG], w2, acc2);
-            acc3 = fmaf(qs[r + 3 * NRG], w3, acc3);
+        // rows r_begin + rg, + NRG, ...: sixteen independent loads in flight per pass
+        for (int r0 = r_begin + rg; r0 < r_end; r0 += 16 * NRG) {
+            float w[16], x[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const int r = r0 + k * NRG;
+                const bool in = r < r_end;
+                w[k] = in ? __ldg(W + (int64_t)r * Hq + h) : 0.f;
+                x[k] = in ? __bfloat162float(qi[r]) : 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < 16; ++k) acc = fmaf(x[k], w[k], acc);
         }
-        for (; r < rows; r += NRG) acc0 = fmaf(qs[r], __ldg(W + (int64_t)r * Hq + h), acc0);
-        part[rg * Hq + h] = (acc0 + acc1) + (acc2 + acc3);
+        part[rg * Hq + h] = acc;
     }
     __syncthreads();
     if (threadIdx.x < Hq) {
         float s = 0.f;
-        for (int g = 0; g < NRG; ++g) s += part[g * Hq + threadIdx.x];
+        for (int k = 0; k < NRG; ++k) s += part[k * Hq + threadIdx.x];
+        float* dst = cluster.map_shared_rank(cpart, 0);
+        dst[crank * Hq + threadIdx.x] = s;
+    }
+    cluster.sync();
+    if (crank == 0 && threadIdx.x < Hq) {
+        float s = 0.f;
+#pragma unroll
+        for (int c = 0; c < PRED_CLUSTER; ++c) s += cpart[c * Hq + threadIdx.x];
         tau[(int64_t)i * Hq + threadIdx.x] = s + bias[threadIdx.x];
     }
 }
@@ -53,12 +73,26 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
                                      const float* W, const float* bias, float* tau, void* stream) {
     if (!q || !W || !bias || !tau) return ETA_ERR_INVALID_ARG;
     if (batch <= 0 || n_q_heads <= 0 || head_dim <= 0) return ETA_ERR_INVALID_ARG;
-    if (n_q_heads > eta::PRED_THREADS) return ETA_ERR_UNSUPPORTED;
+    if (n_q_heads > eta::PRED_THREADS || batch > 65535) return ETA_ERR_UNSUPPORTED;
     const int rows = n_q_heads * head_dim;
     const int NRG = eta::PRED_THREADS / n_q_heads;
-    const size_t smem = sizeof(float) * ((size_t)rows + (size_t)NRG * n_q_heads);
+    const size_t smem = sizeof(float) * ((size_t)NRG * n_q_heads + (size_t)eta::PRED_CLUSTER * n_q_heads);
     if (smem > 48 * 1024) return ETA_ERR_UNSUPPORTED;
-    eta::predict_threshold_kernel<<<batch, eta::PRED_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __nv_bfloat16*>(q), W, bias, tau, n_q_heads, rows);
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(eta::PRED_CLUSTER, batch, 1);
+    cfg.blockDim = dim3(eta::PRED_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = eta::PRED_CLUSTER;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, eta::predict_threshold_kernel, static_cast<const __nv_bfloat16*>(q), W,
+                                       bias, tau, (int)n_q_heads, rows);
+    if (e != cudaSuccess) { eta::set_cuda_error(e, "eta_predict_threshold"); return ETA_ERR_CUDA; }
     return eta::check_launch("eta_predict_threshold");
 }

@@ -245,7 +245,11 @@ __global__ void __launch_bounds__(1024) plan_kernel(const PlanArgs a) {
     __shared__ int32_t warp_sum[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    // ---- top-1 rescue, one warp per row, heads in turn (Algorithm 3: rescue phase of the first chunk)
+    // partial slots a streaming group never writes must read as "absent" in the merge
+    for (int k = tid; k < a.n_part; k += 1024) a.part_ml[k] = make_float2(-INFINITY, 0.f);
+
+    // ---- top-1 rescue, one warp per row (Algorithm 3: rescue phase of the first chunk).  Lane (g, s) reads the
+    // window statistics of head g in window segment s, all at once; four segments (256 blocks) per pass.
     for (int r = warp; r < a.rows; r += 32) {
         const int i = r / a.Hkv;
         int T = a.seq_lens[i];
@@ -258,39 +262,46 @@ __global__ void __launch_bounds__(1024) plan_kernel(const PlanArgs a) {
         const int Wr = min(a.rescue_window, NB);
         const int nsw = (Wr + SEG - 1) / SEG;
         if (Wr <= 0) continue;
-        for (int g = 0; g < a.G; ++g) {
-            int cnt = 0, arg = 0x7fffffff;
-            float best = -INFINITY;
-            for (int s = lane; s < nsw; s += 32) {
+        const int g = lane >> 2, s4 = lane & 3;
+        int cnt = 0, arg = 0x7fffffff;
+        float best = -INFINITY;
+        if (g < a.G) {
+            for (int s = s4; s < nsw; s += 4) {
                 const RescueRec rr = a.seg_resc[((int64_t)r * a.nseg + s) * a.G + g];
                 cnt += rr.cnt;
                 if (rr.arg >= 0 && rr.maxb > best) { best = rr.maxb; arg = rr.arg; }
             }
-            for (int s = 16; s >= 1; s >>= 1) {
-                cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
-                const float ob = __shfl_xor_sync(0xffffffffu, best, s);
-                const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
-                if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+        }
+#pragma unroll
+        for (int s = 1; s <= 2; s <<= 1) {
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
+            const float ob = __shfl_xor_sync(0xffffffffu, best, s);
+            const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
+            if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+        }
+        unsigned need = __ballot_sync(0xffffffffu, g < a.G && s4 == 0 && cnt == 0);
+        while (need) {
+            const int src = __ffs(need) - 1;
+            need &= need - 1;
+            const int gg = src >> 2;
+            const int ja = __shfl_sync(0xffffffffu, arg, src);
+            const int j = (ja == 0x7fffffff) ? 0 : ja;
+            const int s = j / SEG;
+            int32_t* list = a.seg_list + ((int64_t)r * a.nseg + s) * LSTRIDE;
+            const int n = a.seg_count[r * a.nseg + s];
+            int found = -1;
+            for (int k = lane; k < n; k += 32)
+                if ((list[k] & 0xffffff) == j) found = k;
+            const unsigned fb = __ballot_sync(0xffffffffu, found >= 0);
+            if (fb) {
+                if (found >= 0) list[found] |= 1 << (24 + gg);
+            } else if (lane == 0) {
+                list[n] = j | (1 << (24 + gg));
+                a.seg_count[r * a.nseg + s] = n + 1;
             }
-            if (cnt == 0) {
-                const int j = (arg == 0x7fffffff) ? 0 : arg;
-                const int s = j / SEG;
-                int32_t* list = a.seg_list + ((int64_t)r * a.nseg + s) * LSTRIDE;
-                const int n = a.seg_count[r * a.nseg + s];
-                int found = -1;
-                for (int k = lane; k < n; k += 32)
-                    if ((list[k] & 0xffffff) == j) found = k;
-                const unsigned fb = __ballot_sync(0xffffffffu, found >= 0);
-                if (fb) {
-                    if (found >= 0) list[found] |= 1 << (24 + g);
-                } else if (lane == 0) {
-                    list[n] = j | (1 << (24 + g));
-                    a.seg_count[r * a.nseg + s] = n + 1;
-                }
-                if (lane == 0) a.sel_mask[(int64_t)r * a.nb_cap + j] |= (uint8_t)(1u << g);
-                __threadfence_block();
-                __syncwarp();
-            }
+            if (lane == 0) a.sel_mask[(int64_t)r * a.nb_cap + j] |= (uint8_t)(1u << gg);
+            __threadfence_block();
+            __syncwarp();
         }
     }
     __syncthreads();
