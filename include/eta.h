@@ -160,6 +160,35 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
                float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev,
                void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * eta_decode for callers that cannot provide scratch memory (the paper has no counterpart: this is a
+ * deployment convenience, not part of the method).  Who needs it: a serving process that handed all of its HBM to
+ * a KV-cache pool at start-up and has nothing left to carve a workspace from; a plug-in that receives tensors
+ * but no allocator; a decode loop that must stay out of the CUDA allocator because cudaMalloc synchronises the
+ * device and may fail once memory is fragmented.
+ *
+ * Same arguments, results and status codes as eta_decode, minus workspace / workspace_bytes.  The scratch is a
+ * fixed array of ETA_STATIC_SCRATCH_BYTES (8 MiB) inside the library's CUDA module: every GPU that loads the
+ * library holds it from load until the process exits.  The call allocates and frees nothing.
+ *   - Limit: shapes for which eta_workspace_bytes() exceeds ETA_STATIC_SCRATCH_BYTES are refused with
+ *     ETA_ERR_WORKSPACE before anything is launched (the five benchmark configurations need 0.8 - 3 MiB).
+ *   - Set-up: the first call on each device looks up the array's device address (with that device current).
+ *     Make that first call ahead of any stream capture.
+ *   - Sharing: all calls on a device use the same array, and it keeps the previous call's contents.  Nothing in
+ *     it has to be cleared by the caller: each call writes every word before reading it.  For the same reason
+ *     two calls whose kernels can overlap on the GPU (different streams, no dependency between them) race on
+ *     the array and corrupt each other; calls on one stream, or otherwise ordered, are fine.
+ */
+#define ETA_STATIC_SCRATCH_BYTES (8u << 20)
+int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, const void* q,
+                      const void* K, const void* V, const int32_t* seq_lens,
+                      const void* musig, const float* mnorm,
+                      const float* tau, const float* head_const,
+                      float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev, void* stream);
+
+/* Size of the built-in scratch of eta_decode_static, in bytes. */
+size_t eta_static_scratch_bytes(void);
+
 /* Number of kernels one eta_decode call launches (for launch accounting). */
 int eta_decode_kernel_count(void);
 

@@ -20,7 +20,7 @@ ETA_BUILD_SIGMA_ENVELOPE = 1
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
 EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
-           "eta_score_dual", "eta_decode", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
+           "eta_score_dual", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
            "eta_profile_kernel_name", "eta_strerror", "eta_last_cuda_error")
 
 
@@ -62,6 +62,8 @@ def load() -> ctypes.CDLL:
         lib.eta_score_dual.argtypes = [D, P, vp, i32p, vp, f32p, f32p, vp]
         lib.eta_decode.argtypes = [D, P, vp, vp, vp, i32p, vp, f32p, f32p, f32p, f32p, vp, i32p, vp, vp,
                                    ctypes.c_size_t, vp]
+        lib.eta_decode_static.argtypes = [D, P, vp, vp, vp, i32p, vp, f32p, f32p, f32p, f32p, vp, i32p, vp, vp]
+        lib.eta_static_scratch_bytes.restype = ctypes.c_size_t
         lib.eta_decode_kernel_count.restype = ctypes.c_int
         lib.eta_strerror.restype = ctypes.c_char_p
         lib.eta_strerror.argtypes = [ctypes.c_int]
@@ -72,7 +74,7 @@ def load() -> ctypes.CDLL:
         lib.eta_profile_kernel_name.argtypes = [ctypes.c_int]
         for name in EXPORTS:
             if name not in ("eta_strerror", "eta_last_cuda_error", "eta_decode_kernel_count",
-                            "eta_profile_kernel_name"):
+                            "eta_profile_kernel_name", "eta_static_scratch_bytes"):
                 getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -178,6 +180,25 @@ def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau,
                              _dev(status, torch.int32, "status"), _dev(workspace, torch.uint8, "workspace"),
                              workspace.numel(), _stream()),
            "eta_decode")
+
+
+def eta_decode_static(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,
+                      stats=None, status=None) -> None:
+    """eta_decode without a workspace argument, for callers that have no device memory to give: the scratch is
+    an 8 MiB array built into the library (see include/eta.h for its limit and sharing rules)."""
+    p = params.c()
+    _check(load().eta_decode_static(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
+                                    _dev(K, torch.bfloat16, "K"), _dev(V, torch.bfloat16, "V"),
+                                    _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                    _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
+                                    _dev(head_const, torch.float32, "head_const"), _dev(out, torch.float32, "out"),
+                                    _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),
+                                    _dev(status, torch.int32, "status"), _stream()),
+           "eta_decode_static")
+
+
+def eta_static_scratch_bytes() -> int:
+    return int(load().eta_static_scratch_bytes())
 
 
 def eta_decode_kernel_count() -> int:

@@ -20,7 +20,7 @@ def lib():
 
 def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "eta.h")).read()
-    declared = set(re.findall(r"^(?:int|const char\*)\s+(eta_\w+)\s*\(", header, flags=re.M))
+    declared = set(re.findall(r"^(?:int|size_t|const char\*)\s+(eta_\w+)\s*\(", header, flags=re.M))
     assert declared, "no declarations found in include/eta.h"
     assert declared == set(eb.EXPORTS)
     for name in declared:
