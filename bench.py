@@ -146,7 +146,7 @@ def run_ours(args):
 
     static_q = torch.empty_like(q_dev[0])
 
-    def make_step(bias_np, flags=0):
+    def make_step(bias_np, flags=0, profiled=False):
         """One decode step on the query in `static_q`.  With --graph (default) the six launches are captured once
         into a CUDA graph and replayed, so the host costs one graph launch per step instead of six kernel launches
         through ctypes; the library calls are the same either way."""
@@ -154,20 +154,14 @@ def run_ours(args):
         params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags,
                                  ctas_per_sm=args.ctas_per_sm)
 
-        def launch(evs=None):
-            if evs:
-                evs[0].record()
+        def launch():
             eb.eta_append_summary(st.desc, Kd, lens_d, st.musig, st.mnorm)
-            if evs:
-                evs[1].record()
             eb.eta_predict_threshold(static_q, Wd, bias_d, st.tau)
-            if evs:
-                evs[2].record()
             eb.eta_decode(st.desc, params, static_q, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau, None, st.out,
                           st.sel_mask, st.workspace, stats=st.stats, status=st.status)
 
         graph = None
-        if args.graph:
+        if args.graph or profiled:
             side = torch.cuda.Stream()
             side.wait_stream(torch.cuda.current_stream())
             with torch.cuda.stream(side):
@@ -177,15 +171,17 @@ def run_ours(args):
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
             graph = torch.cuda.CUDAGraph()
+            eb.eta_profile_enable(profiled)     # timing events are captured as nodes of the graph
             with torch.cuda.graph(graph):
                 launch()
+            eb.eta_profile_enable(False)
 
-        def step(qd, evs=None):
+        def step(qd):
             static_q.copy_(qd, non_blocking=True)
-            if graph is not None and evs is None:
+            if graph is not None:
                 graph.replay()
             else:
-                launch(evs)
+                launch()
         return step
 
     def timed(step):
@@ -221,18 +217,15 @@ def run_ours(args):
             tot += int(st.stats.sum().item())
         return tot / args.steps
 
-    def kernel_times(step):
-        eb.eta_profile_enable(True)
+    def kernel_times(bias_np, flags=0):
+        """Device time from each launch to the next, averaged over the steps, from events captured in the graph."""
+        stp = make_step(bias_np, flags, profiled=True)
         acc = {}
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         for k in range(args.steps):
             flush.fill_(k & 0xff)
-            step(q_dev[args.warmup + k], evs=evs)
+            stp(q_dev[args.warmup + k])
             for name, v in eb.eta_profile_read().items():
                 acc[name] = acc.get(name, 0.0) + v
-            acc["append_summary_kernel"] = acc.get("append_summary_kernel", 0.0) + evs[0].elapsed_time(evs[1])
-            acc["predict_threshold_kernel"] = acc.get("predict_threshold_kernel", 0.0) + evs[1].elapsed_time(evs[2])
-        eb.eta_profile_enable(False)
         return {k: v / args.steps for k, v in acc.items()}
 
     targets = list(sp.target_sparsity)
@@ -248,7 +241,7 @@ def run_ours(args):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         ms_step = float(tt.item())
     union_main = union_blocks_of(step_main)
-    kt = kernel_times(step_main)
+    kt = kernel_times(load_bias(sp.name, main_target))
     nb_total = sum(int(t) // sp.block_size for t in lens) * sp.n_kv_heads
     ab = algorithmic_bytes(sp, lens, union_main)
     peak, peak_kind = hbm_peak()
@@ -287,7 +280,7 @@ def run_ours(args):
             ub = union_blocks_of(stp)
             abt = algorithmic_bytes(sp, lens, ub)
             m = sum(ms) / len(ms)
-            ktt = kernel_times(stp)
+            ktt = kernel_times(load_bias(sp.name, tgt))
             sweep[f"{tgt:.2f}"] = {"ms_per_step": m, "union_sparsity": 1 - ub / nb_total,
                                    "gbs_on_algorithmic_bytes": abt["total"] / (m * 1e-3) / 1e9, "kernel_ms": ktt,
                                    "decode_kernel_gbs": abt["decode"] / (ktt["decode_kernel"] * 1e-3) / 1e9}
@@ -295,7 +288,7 @@ def run_ours(args):
         ms, _ = timed(stp)
         m = sum(ms) / len(ms)
         abt = algorithmic_bytes(sp, lens, nb_total)
-        ktt = kernel_times(stp)
+        ktt = kernel_times(np.zeros(sp.n_q_heads, np.float32), flags=eb.ETA_FLAG_DENSE)
         sweep["dense_baseline"] = {"ms_per_step": m, "gbs_on_algorithmic_bytes": (abt["decode"]) / (m * 1e-3) / 1e9,
                                    "speedup_of_main": m / ms_step, "kernel_ms": ktt,
                                    "decode_kernel_gbs": abt["decode"] / (ktt["decode_kernel"] * 1e-3) / 1e9}

@@ -193,11 +193,14 @@ size_t eta_static_scratch_bytes(void);
 int eta_decode_kernel_count(void);
 
 /*
- * Per-kernel timing of eta_decode (measurement aid; the paper has no counterpart).  While enabled, every
- * eta_decode call records host-side CUDA events between its kernel launches on the call's stream;
- * eta_profile_read waits for the most recent call to finish and writes the device time of each kernel in
- * milliseconds to ms[0 .. count-1] (n >= eta_decode_kernel_count()), returning the count, or a negative status
- * when no profiled call has been made.  Not thread-safe; leave disabled in production.
+ * Per-kernel timing of a decode step (measurement aid; the paper has no counterpart).  While enabled,
+ * eta_append_summary, eta_predict_threshold and eta_decode record host-side CUDA events before each of their
+ * kernel launches on the call's stream (inside a stream capture they become nodes of the graph).
+ * eta_profile_read waits for the most recent eta_decode to finish and writes the time from each launch to the
+ * next, in milliseconds, to ms[0 .. count-1] (n >= 6), in the order append, predict, screen, plan, decode,
+ * merge, returning the count, or a negative status when no profiled eta_decode has run.  The first two are 0
+ * unless those calls were made, in that order, right before the eta_decode.  Not thread-safe; leave disabled
+ * in production.
  */
 int eta_profile_enable(int on);
 int eta_profile_read(float* ms, int n);

@@ -30,6 +30,29 @@ int validate_desc(const eta_cache_desc* d) {
     return ETA_OK;
 }
 
+// Optional per-kernel timing: host-side CUDA events recorded between the launches of one decode step
+// (append, predict, then the four kernels of eta_decode).  Event k is recorded just before launch k; event 6
+// after the last launch.
+constexpr int N_MARKS = 7;
+static bool g_profile = false;
+static cudaEvent_t g_ev[N_MARKS];
+static bool g_ev_made = false;
+static unsigned g_ev_seen = 0;
+
+void profile_mark(int k, cudaStream_t s) {
+    if (!g_profile) return;
+    if (!g_ev_made) {
+        for (int i = 0; i < N_MARKS; ++i) cudaEventCreate(&g_ev[i]);
+        g_ev_made = true;
+    }
+    // inside a stream capture the record must be an "external" node to stay a real, timeable event at replay
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(s, &cap);
+    if (cap == cudaStreamCaptureStatusActive) cudaEventRecordWithFlags(g_ev[k], s, cudaEventRecordExternal);
+    else cudaEventRecord(g_ev[k], s);
+    g_ev_seen |= 1u << k;
+}
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 WsLayout ws_layout(const eta_cache_desc* d) {
@@ -77,5 +100,32 @@ const char* eta_strerror(int code) {
 }
 
 const char* eta_last_cuda_error(void) { return eta::g_cuda_error; }
+
+int eta_profile_enable(int on) {
+    if (on && !eta::g_profile) eta::g_ev_seen = 0;     // a new profiled run starts; a finished one stays readable
+    eta::g_profile = on != 0;
+    return ETA_OK;
+}
+
+int eta_profile_read(float* ms, int n) {
+    using namespace eta;
+    if (!ms || n < N_MARKS - 1) return ETA_ERR_INVALID_ARG;
+    if ((g_ev_seen & 0x7c) != 0x7c) return ETA_ERR_INVALID_ARG;      // no profiled eta_decode yet
+    cudaError_t e = cudaEventSynchronize(g_ev[6]);
+    for (int k = 0; k < N_MARKS - 1 && e == cudaSuccess; ++k) {
+        ms[k] = 0.f;
+        // append / predict are separate calls: timed only when they were made in the same profiled step
+        if (k < 2 && !((g_ev_seen >> k) & 1)) continue;
+        e = cudaEventElapsedTime(&ms[k], g_ev[k], g_ev[k + 1]);
+    }
+    if (e != cudaSuccess) { set_cuda_error(e, "eta_profile_read"); return ETA_ERR_CUDA; }
+    return N_MARKS - 1;
+}
+
+const char* eta_profile_kernel_name(int k) {
+    static const char* names[6] = {"append_summary_kernel", "predict_threshold_kernel", "screen_kernel",
+                                   "plan_kernel", "decode_kernel", "merge_kernel"};
+    return (k >= 0 && k < 6) ? names[k] : "";
+}
 
 }  // extern "C"

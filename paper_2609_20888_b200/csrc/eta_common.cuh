@@ -20,6 +20,8 @@ inline int check_launch(const char* where) {
     return ETA_OK;
 }
 int validate_desc(const eta_cache_desc* d);
+// Measurement aid: when profiling is enabled, records timing event k on the stream (see eta_profile_enable).
+void profile_mark(int k, cudaStream_t s);
 
 // Screening works on segments of SEG consecutive block records of one
 // (sequence, KV head) row; a segment's survivors are compacted into a list of

@@ -592,45 +592,9 @@ static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const
 
 }  // namespace eta
 
-namespace eta {
-// Optional per-kernel timing of eta_decode: host-side CUDA events recorded between its launches.
-static bool g_profile = false;
-static cudaEvent_t g_ev[5];
-static bool g_ev_made = false, g_ev_valid = false;
-static void profile_mark(int k, cudaStream_t s) {
-    if (!g_profile) return;
-    if (!g_ev_made) {
-        for (int i = 0; i < 5; ++i) cudaEventCreate(&g_ev[i]);
-        g_ev_made = true;
-    }
-    cudaEventRecord(g_ev[k], s);
-    if (k == 4) g_ev_valid = true;
-}
-}  // namespace eta
-
 extern "C" {
 
 int eta_decode_kernel_count(void) { return 4; }
-
-int eta_profile_enable(int on) {
-    eta::g_profile = on != 0;
-    eta::g_ev_valid = false;
-    return ETA_OK;
-}
-
-int eta_profile_read(float* ms, int n) {
-    if (!ms || n < 4) return ETA_ERR_INVALID_ARG;
-    if (!eta::g_ev_valid) return ETA_ERR_INVALID_ARG;
-    cudaError_t e = cudaEventSynchronize(eta::g_ev[4]);
-    for (int k = 0; k < 4 && e == cudaSuccess; ++k) e = cudaEventElapsedTime(&ms[k], eta::g_ev[k], eta::g_ev[k + 1]);
-    if (e != cudaSuccess) { eta::set_cuda_error(e, "eta_profile_read"); return ETA_ERR_CUDA; }
-    return 4;
-}
-
-const char* eta_profile_kernel_name(int k) {
-    static const char* names[4] = {"screen_kernel", "plan_kernel", "decode_kernel", "merge_kernel"};
-    return (k >= 0 && k < 4) ? names[k] : "";
-}
 
 int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q, const void* K, const void* V,
                const int32_t* seq_lens, const void* musig, const float* mnorm, const float* tau,
@@ -682,9 +646,9 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     sa.seg_resc = reinterpret_cast<RescueRec*>(ws + L.seg_resc);
     sa.tau_eff = reinterpret_cast<float*>(ws + L.tau_eff);
     sa.sel_mask = sel_mask;
-    profile_mark(0, s);
+    profile_mark(2, s);
     rc = launch_screen(sa, L.rows, D, G, s);
-    profile_mark(1, s);
+    profile_mark(3, s);
     if (rc != ETA_OK) return rc;
 
     PlanArgs pa;
@@ -702,7 +666,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     pa.n_part = (n_ctas + L.rows) * DECODE_GROUPS * G;
     rc = launch_plan(pa, s);
     if (rc != ETA_OK) return rc;
-    profile_mark(2, s);
+    profile_mark(4, s);
 
     CUtensorMap tmK, tmV;
     rc = make_tmap(&tmK, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t, TS);
@@ -730,7 +694,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
         rc = launch_decode_t<64, 32, 8, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s);
     }
     if (rc != ETA_OK) return rc;
-    profile_mark(3, s);
+    profile_mark(5, s);
 
     MergeArgs ma;
     ma.pref = pa.pref; ma.hdr = pa.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
@@ -738,7 +702,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     const unsigned mgrid = (unsigned)(L.rows * G);
     if (D == 128) merge_kernel<128><<<mgrid, 32 * MERGE_WARPS, 0, s>>>(ma);
     else merge_kernel<64><<<mgrid, 32 * MERGE_WARPS, 0, s>>>(ma);
-    profile_mark(4, s);
+    profile_mark(6, s);
     return check_launch("merge");
 }
 

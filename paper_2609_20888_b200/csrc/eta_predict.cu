@@ -91,6 +91,7 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    eta::profile_mark(1, cfg.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, eta::predict_threshold_kernel, static_cast<const __nv_bfloat16*>(q), W,
                                        bias, tau, (int)n_q_heads, rows);
     if (e != cudaSuccess) { eta::set_cuda_error(e, "eta_predict_threshold"); return ETA_ERR_CUDA; }

@@ -230,6 +230,7 @@ int eta_append_summary(const eta_cache_desc* desc, const void* K, const int32_t*
     const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
     auto Kp = static_cast<const __nv_bfloat16*>(K);
     auto mp = static_cast<__half*>(musig);
+    eta::profile_mark(0, s);
     if (desc->head_dim == 128)
         eta::append_summary_kernel<128><<<rows, eta::SUM_THREADS, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h,
             desc->k_stride_t, desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, seq_lens_after, env, mp,
