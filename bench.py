@@ -116,6 +116,7 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     eb.load()
+    eb.eta_set_pdl(args.pdl)
 
     sp = wl.CONFIGS[args.workload]
     t0 = time.time()
@@ -306,7 +307,7 @@ def run_ours(args):
                        "head_dim": sp.head_dim, "context": sp.context, "block_size": sp.block_size,
                        "target_union_sparsity": main_target, "measured_union_sparsity": 1 - union_main / nb_total,
                        "z": sp.z, "beta": sp.beta, "l2": "flushed between timed steps (384 MiB write)",
-                       "fresh_query_every_step": True, "replicas": world, "cuda_graph": bool(args.graph)},
+                       "fresh_query_every_step": True, "replicas": world, "cuda_graph": bool(args.graph), "pdl": bool(args.pdl)},
             "attention_us_per_token": ms_step * 1e3,
             "achieved_gbs_all_kernels": ab["total"] / (ms_step * 1e-3) / 1e9,
             "frac_of_8tbs_nominal": ab["total"] / (ms_step * 1e-3) / 8e12,
@@ -394,6 +395,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.CONFIGS))
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch the kernels directly every step")
+    ap.add_argument("--no-pdl", dest="pdl", action="store_false", help="fully serialise the kernel launches")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -83,8 +83,12 @@ typedef struct eta_params {
 
 /*
  * Bytes of scratch eta_decode needs for this cache shape (independent of the
- * sequence lengths).  The caller allocates it once, 256-byte aligned, and may
- * reuse it across calls on the same stream.  No device is touched.
+ * sequence lengths).  The caller allocates it once, 256-byte aligned, ZERO-FILLS
+ * it before the first call, and may then reuse it across calls on the same
+ * stream without touching it: a successful call leaves it ready for the next
+ * one (its first batch * n_kv_heads words are per-row tickets that every call
+ * returns to zero).  After a call that reported ETA_DEV_TIMEOUT, zero it again.
+ * No device is touched by this function.
  */
 int eta_workspace_bytes(const eta_cache_desc* desc, size_t* out_bytes);
 
@@ -175,9 +179,10 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
  *   - Set-up: the first call on each device looks up the array's device address (with that device current).
  *     Make that first call ahead of any stream capture.
  *   - Sharing: all calls on a device use the same array, and it keeps the previous call's contents.  Nothing in
- *     it has to be cleared by the caller: each call writes every word before reading it.  For the same reason
- *     two calls whose kernels can overlap on the GPU (different streams, no dependency between them) race on
- *     the array and corrupt each other; calls on one stream, or otherwise ordered, are fine.
+ *     it has to be cleared by the caller: the array starts zeroed when the library is loaded, every call
+ *     returns its per-row tickets to zero, and every other word is written before it is read.  Two calls
+ *     whose kernels can overlap on the GPU (different streams, no dependency between them) race on the array
+ *     and corrupt each other; calls on one stream, or otherwise ordered, are fine.
  */
 #define ETA_STATIC_SCRATCH_BYTES (8u << 20)
 int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, const void* q,
@@ -197,14 +202,31 @@ int eta_decode_kernel_count(void);
  * eta_append_summary, eta_predict_threshold and eta_decode record host-side CUDA events before each of their
  * kernel launches on the call's stream (inside a stream capture they become nodes of the graph).
  * eta_profile_read waits for the most recent eta_decode to finish and writes the time from each launch to the
- * next, in milliseconds, to ms[0 .. count-1] (n >= 6), in the order append, predict, screen, plan, decode,
- * merge, returning the count, or a negative status when no profiled eta_decode has run.  The first two are 0
+ * next, in milliseconds, to ms[0 .. count-1] (n >= 5), in the order append, predict, screen, decode, merge,
+ * returning the count, or a negative status when no profiled eta_decode has run.  The first two are 0
  * unless those calls were made, in that order, right before the eta_decode.  Not thread-safe; leave disabled
  * in production.
  */
 int eta_profile_enable(int on);
 int eta_profile_read(float* ms, int n);
 const char* eta_profile_kernel_name(int k);
+
+/*
+ * Launch policy (the paper has no counterpart).  By default the kernels of a decode step are launched with
+ * programmatic dependent launch: each may start its set-up while its predecessor in the stream drains, and
+ * waits for the predecessor's completion before reading anything it wrote.  eta_set_pdl(0) makes every launch
+ * wait for the full completion of the previous one instead (for A/B timing and for debugging).  Process-wide.
+ */
+int eta_set_pdl(int on);
+
+/*
+ * Development aid (the paper has no counterpart): when dev_buffer is a device array of at least
+ * 8 * 1024 uint64, every CTA c of the screening kernel (c < 512) and of the streaming kernel writes up to eight
+ * %globaltimer stamps (ns) at [k * 8 .. k * 8 + 7], k = c for the streaming kernel and 512 + c for the screening
+ * kernel: kernel entry, set-up done, first copy issued, first tile consumed, last tile consumed, partials stored.
+ * NULL switches it off (the default).
+ */
+int eta_debug_timeline(void* dev_buffer);
 
 /* Text for an eta_status. */
 const char* eta_strerror(int code);

@@ -21,7 +21,7 @@ ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
 EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
            "eta_score_dual", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
-           "eta_profile_kernel_name", "eta_strerror", "eta_last_cuda_error")
+           "eta_profile_kernel_name", "eta_set_pdl", "eta_debug_timeline", "eta_strerror", "eta_last_cuda_error")
 
 
 class CacheDesc(ctypes.Structure):
@@ -69,6 +69,8 @@ def load() -> ctypes.CDLL:
         lib.eta_strerror.argtypes = [ctypes.c_int]
         lib.eta_last_cuda_error.restype = ctypes.c_char_p
         lib.eta_profile_enable.argtypes = [ctypes.c_int]
+        lib.eta_set_pdl.argtypes = [ctypes.c_int]
+        lib.eta_debug_timeline.argtypes = [ctypes.c_void_p]
         lib.eta_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int]
         lib.eta_profile_kernel_name.restype = ctypes.c_char_p
         lib.eta_profile_kernel_name.argtypes = [ctypes.c_int]
@@ -205,6 +207,10 @@ def eta_decode_kernel_count() -> int:
     return load().eta_decode_kernel_count()
 
 
+def eta_set_pdl(on: bool) -> None:
+    _check(load().eta_set_pdl(1 if on else 0), "eta_set_pdl")
+
+
 def eta_profile_enable(on: bool) -> None:
     _check(load().eta_profile_enable(1 if on else 0), "eta_profile_enable")
 
@@ -227,7 +233,7 @@ class DecodeState:
         self.desc = cache_desc(K, V, n_q_heads, block_size)
         self.K, self.V = K, V
         self.musig, self.mnorm = alloc_summaries(self.desc, dev)
-        self.workspace = torch.empty(eta_workspace_bytes(self.desc) + 256, dtype=torch.uint8, device=dev)
+        self.workspace = torch.zeros(eta_workspace_bytes(self.desc) + 256, dtype=torch.uint8, device=dev)
         off = (-self.workspace.data_ptr()) % 256
         self.workspace = self.workspace[off:off + eta_workspace_bytes(self.desc)]
         B, Hkv, d = self.desc.batch, self.desc.n_kv_heads, self.desc.head_dim

@@ -9,6 +9,8 @@ namespace eta {
 
 static thread_local char g_cuda_error[256] = "";
 
+void set_pdl(bool on);
+
 void set_cuda_error(cudaError_t e, const char* where) {
     snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", where, cudaGetErrorString(e));
 }
@@ -24,6 +26,7 @@ int validate_desc(const eta_cache_desc* d) {
     if (d->block_size != 32 && d->block_size != 64 && d->block_size != 128) return ETA_ERR_UNSUPPORTED;
     if ((int64_t)d->nb_cap * d->block_size < d->t_cap - d->block_size + 1) return ETA_ERR_INVALID_ARG;
     if (d->nb_cap >= (1 << 24)) return ETA_ERR_UNSUPPORTED;   // block index shares a word with the head bits
+    if ((int64_t)d->batch * d->n_kv_heads > MAX_ROWS) return ETA_ERR_UNSUPPORTED;
     if (d->k_stride_t % 8 || d->k_stride_h % 8 || d->k_stride_b % 8) return ETA_ERR_UNSUPPORTED;
     if (d->v_stride_t % 8 || d->v_stride_h % 8 || d->v_stride_b % 8) return ETA_ERR_UNSUPPORTED;
     if (d->k_stride_t < d->head_dim || d->v_stride_t < d->head_dim) return ETA_ERR_INVALID_ARG;
@@ -31,9 +34,9 @@ int validate_desc(const eta_cache_desc* d) {
 }
 
 // Optional per-kernel timing: host-side CUDA events recorded between the launches of one decode step
-// (append, predict, then the four kernels of eta_decode).  Event k is recorded just before launch k; event 6
+// (append, predict, then the three kernels of eta_decode).  Event k is recorded just before launch k; event 5
 // after the last launch.
-constexpr int N_MARKS = 7;
+constexpr int N_MARKS = 6;
 static bool g_profile = false;
 static cudaEvent_t g_ev[N_MARKS];
 static bool g_ev_made = false;
@@ -53,6 +56,12 @@ void profile_mark(int k, cudaStream_t s) {
     g_ev_seen |= 1u << k;
 }
 
+static unsigned long long* g_timeline = nullptr;
+unsigned long long* debug_timeline() { return g_timeline; }
+static bool g_pdl = true;
+bool pdl_enabled() { return g_pdl; }
+void set_pdl(bool on) { g_pdl = on; }
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 WsLayout ws_layout(const eta_cache_desc* d) {
@@ -62,12 +71,14 @@ WsLayout ws_layout(const eta_cache_desc* d) {
     L.nseg = (d->nb_cap + SEG - 1) / SEG;
     L.entries = L.rows * (L.nseg + 1);
     size_t off = 0;
+    L.row_ticket = off; off = align_up(off + sizeof(int32_t) * (size_t)L.rows, 256);
     L.hdr = off;        off = align_up(off + 8 * sizeof(int32_t), 256);
     L.seg_count = off;  off = align_up(off + sizeof(int32_t) * (size_t)L.rows * L.nseg, 256);
     L.seg_list = off;   off = align_up(off + sizeof(int32_t) * (size_t)L.rows * L.nseg * LSTRIDE, 256);
     L.seg_resc = off;   off = align_up(off + sizeof(RescueRec) * (size_t)L.rows * L.nseg * G, 256);
-    L.pref = off;       off = align_up(off + sizeof(int32_t) * ((size_t)L.entries + 1), 256);
-    L.cta_start = off;  off = align_up(off + sizeof(int4) * (size_t)MAX_CTAS, 256);
+    L.row_pref = off;   off = align_up(off + sizeof(int32_t) * (size_t)L.entries, 256);
+    L.row_total = off;  off = align_up(off + sizeof(int32_t) * (size_t)L.rows, 256);
+    L.row_start = off;  off = align_up(off + sizeof(int32_t) * ((size_t)L.rows + 1), 256);
     L.tau_eff = off;    off = align_up(off + sizeof(float) * (size_t)d->batch * d->n_q_heads, 256);
     size_t slots = ((size_t)MAX_CTAS + L.rows) * DECODE_GROUPS;
     L.part_ml = off;    off = align_up(off + sizeof(float2) * slots * G, 256);
@@ -101,6 +112,16 @@ const char* eta_strerror(int code) {
 
 const char* eta_last_cuda_error(void) { return eta::g_cuda_error; }
 
+int eta_debug_timeline(void* dev_buffer) {
+    eta::g_timeline = static_cast<unsigned long long*>(dev_buffer);
+    return ETA_OK;
+}
+
+int eta_set_pdl(int on) {
+    eta::set_pdl(on != 0);
+    return ETA_OK;
+}
+
 int eta_profile_enable(int on) {
     if (on && !eta::g_profile) eta::g_ev_seen = 0;     // a new profiled run starts; a finished one stays readable
     eta::g_profile = on != 0;
@@ -110,8 +131,8 @@ int eta_profile_enable(int on) {
 int eta_profile_read(float* ms, int n) {
     using namespace eta;
     if (!ms || n < N_MARKS - 1) return ETA_ERR_INVALID_ARG;
-    if ((g_ev_seen & 0x7c) != 0x7c) return ETA_ERR_INVALID_ARG;      // no profiled eta_decode yet
-    cudaError_t e = cudaEventSynchronize(g_ev[6]);
+    if ((g_ev_seen & 0x3c) != 0x3c) return ETA_ERR_INVALID_ARG;      // no profiled eta_decode yet
+    cudaError_t e = cudaEventSynchronize(g_ev[5]);
     for (int k = 0; k < N_MARKS - 1 && e == cudaSuccess; ++k) {
         ms[k] = 0.f;
         // append / predict are separate calls: timed only when they were made in the same profiled step
@@ -123,9 +144,9 @@ int eta_profile_read(float* ms, int n) {
 }
 
 const char* eta_profile_kernel_name(int k) {
-    static const char* names[6] = {"append_summary_kernel", "predict_threshold_kernel", "screen_kernel",
-                                   "plan_kernel", "decode_kernel", "merge_kernel"};
-    return (k >= 0 && k < 6) ? names[k] : "";
+    static const char* names[5] = {"append_summary_kernel", "predict_threshold_kernel", "screen_kernel",
+                                   "decode_kernel", "merge_kernel"};
+    return (k >= 0 && k < 5) ? names[k] : "";
 }
 
 }  // extern "C"

@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "../../include/eta.h"
 
 namespace eta {
@@ -29,7 +31,7 @@ void profile_mark(int k, cudaStream_t s);
 constexpr int SEG = 64;
 constexpr int LSTRIDE = SEG + 8;
 constexpr int MAX_CTAS = 256;        // upper bound on streaming CTAs (sizes the scratch; a B200 has 148 SMs)
-constexpr int MAX_ENTRIES = 49152;   // plan kernel keeps the unit prefix in shared memory
+constexpr int MAX_ROWS = 1024;        // rows (batch * n_kv_heads) whose unit prefix a streaming CTA keeps in shared memory
 constexpr int DECODE_GROUPS = 3;     // consumer groups per streaming CTA, each with its own partial per piece
 
 // Scratch layout (byte offsets from a 256-byte aligned base).
@@ -37,12 +39,14 @@ struct WsLayout {
     int rows;        // batch * n_kv_heads
     int nseg;        // segments per row
     int entries;     // rows * (nseg + 1): one pseudo-segment per row holds the tail unit
-    size_t hdr;      // int32[8]: [0] total units U, [1] streaming CTAs P
+    size_t row_ticket;  // int32 [rows]: ZERO between calls (the only part of the scratch that carries state)
+    size_t hdr;         // int32[8]: [0] total units U, [1] streaming CTAs P (written by the streaming kernel)
     size_t seg_count;   // int32 [rows * nseg]
     size_t seg_list;    // int32 [rows * nseg * LSTRIDE]: block index | head bits << 24
     size_t seg_resc;    // {int cnt; float maxb; int arg; int pad} [rows * nseg * G]
-    size_t pref;        // int32 [entries + 1] exclusive prefix of units per entry
-    size_t cta_start;   // int4 [MAX_CTAS]: {u0, u1, first entry, 0}
+    size_t row_pref;    // int32 [entries]: exclusive prefix of survivor counts inside each row
+    size_t row_total;   // int32 [rows]: units per row
+    size_t row_start;   // int32 [rows + 1]: global unit prefix over rows (written by the streaming kernel)
     size_t tau_eff;     // float [batch * n_q_heads]
     size_t part_ml;     // float2 [(MAX_CTAS + rows) * DECODE_GROUPS * G]
     size_t part_o;      // float [(MAX_CTAS + rows) * DECODE_GROUPS * G * d]
@@ -69,27 +73,42 @@ struct ScreenArgs {
     RescueRec* seg_resc;
     float* tau_eff;
     uint8_t* sel_mask;
-};
-struct PlanArgs {
-    const int32_t* seq_lens;
-    int Hkv, G, b, t_cap, nb_cap, nseg, rows, entries, rescue_window, n_ctas;
-    int32_t* seg_count;
-    int32_t* seg_list;
-    const RescueRec* seg_resc;
-    uint8_t* sel_mask;
-    int32_t* pref;
-    int4* cta_start;
-    int32_t* hdr;
+    int32_t* row_ticket;   // [rows] zero between calls
+    int32_t* row_pref;     // [rows * (nseg + 1)] exclusive prefix of survivor counts inside each row
+    int32_t* row_total;    // [rows] units of the row (surviving blocks + tail)
     int32_t* stats;
     uint32_t* status;
-    float2* part_ml;   // partial (m, l) slots, reset to "absent" before the streaming kernel runs
-    int n_part;
+    unsigned long long* timeline;
 };
 int launch_screen(const ScreenArgs& a, int rows, int D, int G, cudaStream_t s);
-int launch_plan(const PlanArgs& a, cudaStream_t s);
+
+// Launch with programmatic dependent launch allowed: the grid may start while its predecessor in the stream is
+// still draining, and must call pdl_wait() before touching anything the predecessor wrote.
+unsigned long long* debug_timeline();   // device buffer for per-CTA time stamps, or nullptr (see eta_debug_timeline)
+bool pdl_enabled();          // false after eta_set_pdl(0): every launch is then fully serialised
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // -------------------------------------------------------------- device side
 #ifdef __CUDACC__
+
+// Programmatic dependent launch: let the next kernel of the stream start its prologue now / wait until the
+// previous kernel of the stream has completed and its writes are visible.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls before a bounded wait gives up
 
@@ -156,6 +175,12 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
+}
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }

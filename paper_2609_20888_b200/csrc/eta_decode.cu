@@ -30,17 +30,21 @@ struct DecodeArgs {
     const int32_t* seq_lens;
     const float* tau_eff;
     const int32_t* seg_list;
-    const int32_t* pref;
-    const int4* cta_start;
+    const int32_t* row_pref;
+    const int32_t* row_total;
+    int32_t* row_start;
+    int32_t* hdr;
     float2* part_ml;
     float* part_o;
     uint32_t* status;
     float beta, scale;
-    int Hq, Hkv, G, b, t_cap, nseg, entries;
+    int Hq, Hkv, G, b, t_cap, nseg, entries, rows;
+    unsigned long long* timeline;
 };
 
 constexpr uint32_t UF_END = 1u;
 constexpr int WARPS_PER_GROUP = 4;     // the four warps of a group each take a quarter of a tile's tokens
+constexpr int PW = 512;                // entries of the unit prefix the producer keeps in shared memory
 
 __device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
     return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
@@ -61,7 +65,9 @@ struct DecodeSmem {
     static constexpr int STAGE_BYTES = 2 * HALVES * TILE_BYTES; // K halves then V halves
     static constexpr int BAR_OFF = NSTAGE * STAGE_BYTES;        // full[NSTAGE], empty[NSTAGE], flush[NGROUPS]
     static constexpr int DESC_OFF = BAR_OFF + 8 * (2 * NSTAGE + NGROUPS + (NGROUPS & 1));
-    static constexpr int ML_OFF = DESC_OFF + 16 * NSTAGE;       // float m[NGROUPS][4][8], l[NGROUPS][4][8]
+    static constexpr int WIN_OFF = DESC_OFF + 16 * NSTAGE;      // int32 pwin[PW + 1] (+3 pad): window of the unit prefix
+    static constexpr int ROW_OFF = WIN_OFF + 4 * (PW + 4);      // int32 rowbase[MAX_ROWS + 1]: unit prefix over rows
+    static constexpr int ML_OFF = ROW_OFF + 4 * (MAX_ROWS + 4); // float m[NGROUPS][4][8], l[NGROUPS][4][8]
     static constexpr int MO_OFF = ML_OFF + 4 * 2 * NGROUPS * WARPS_PER_GROUP * 8;
     static size_t bytes(int G) { return 1024 + MO_OFF + sizeof(float) * NGROUPS * WARPS_PER_GROUP * G * D; }
 };
@@ -86,12 +92,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     uint64_t* empty = full + NSTAGE;
     uint64_t* flushbar = empty + NSTAGE;
     int4* desc = reinterpret_cast<int4*>(smem + L::DESC_OFF);
+    int32_t* pwin = reinterpret_cast<int32_t*>(smem + L::WIN_OFF);
+    int32_t* rowbase = reinterpret_cast<int32_t*>(smem + L::ROW_OFF);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int4 cs = a.cta_start[blockIdx.x];
-    const int u0 = cs.x, u1 = cs.y;
-    if (u0 >= u1) return;
-
+    unsigned long long* tl = a.timeline ? a.timeline + (size_t)blockIdx.x * 8 : nullptr;
+    if (tl && tid == 0) tl[0] = globaltimer_ns();
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], WARPS_PER_GROUP); }
         for (int k = 0; k < NGROUPS; ++k) mbar_init(&flushbar[k], 32 * WARPS_PER_GROUP);
@@ -100,74 +106,188 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         prefetch_tmap(&tmV);
     }
     __syncthreads();
+    pdl_wait();          // the screening kernel's lists, row prefixes and row totals are complete from here on
+
+    // ---- every CTA derives its own share of the flattened unit sequence: scan of the per-row unit totals
+    {
+        __shared__ int s_wsum[32];
+        const int nthreads = 32 * (WARPS_PER_GROUP * NGROUPS + 1);
+        int carry = 0;
+        for (int r0 = 0; r0 < a.rows; r0 += nthreads) {
+            const int rr = r0 + tid;
+            const int c = (rr < a.rows) ? __ldg(a.row_total + rr) : 0;
+            int incl = c;
+#pragma unroll
+            for (int s = 1; s < 32; s <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, s);
+                if (lane >= s) incl += o;
+            }
+            if (lane == 31) s_wsum[warp] = incl;
+            __syncthreads();
+            int wbase = 0, tot = 0;
+            for (int w = 0; w < nthreads / 32; ++w) {
+                const int v = s_wsum[w];
+                if (w < warp) wbase += v;
+                tot += v;
+            }
+            if (rr < a.rows) rowbase[rr] = carry + wbase + incl - c;
+            carry += tot;
+            __syncthreads();
+        }
+        if (tid == 0) rowbase[a.rows] = carry;
+        __syncthreads();
+    }
+    const int U = rowbase[a.rows];
+    const int P = gridDim.x;
+    const int u0 = (int)(((int64_t)blockIdx.x * U) / P), u1 = (int)(((int64_t)(blockIdx.x + 1) * U) / P);
+    if (blockIdx.x == 0) {
+        // the merge kernel reads the row ranges and the split from memory
+        for (int rr = tid; rr <= a.rows; rr += 32 * (WARPS_PER_GROUP * NGROUPS + 1)) a.row_start[rr] = rowbase[rr];
+        if (tid == 0) { a.hdr[0] = U; a.hdr[1] = P; }
+    }
+    if (tl && tid == 0) tl[1] = globaltimer_ns();
+    if (u0 >= u1) return;
+    // row holding unit u0: last r with rowbase[r] <= u0
+    int row0;
+    {
+        int lo = 0, hi = a.rows - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (rowbase[mid] <= u0) lo = mid; else hi = mid - 1;
+        }
+        row0 = lo;
+    }
 
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
+        // The CTA's units [u0, u1) are located through a shared-memory window of the unit prefix (PW entries from
+        // entry e_base on): each lane finds the entry of one unit by binary search in the window and fetches that
+        // unit's list word, so a batch of up to 32 units costs one round trip to L2, and the next batch is fetched
+        // while the current one is being issued.
         const int EPR = a.nseg + 1;
         const int E = a.entries;
-        int e = cs.z;
-        int u = u0;
+        int e_base = row0 * EPR;
         uint32_t fill = 0;
-        int piece = -1;
+        int piece = -1, prev_row = -1;
+        uint32_t piece_f0 = 0;
         bool ok = true;
-        while (u < u1 && ok) {
-            // entry holding unit u: pref[e] <= u < pref[e+1]; skip empty entries 32 at a time
-            while (true) {
-                const int pv = __ldg(a.pref + min(e + 1 + lane, E));
-                const unsigned gt = __ballot_sync(0xffffffffu, pv > u);
-                if (gt) { e += __ffs(gt) - 1; break; }
-                e += 32;
-                if (e >= E) { ok = false; break; }     // inconsistent plan: stop instead of walking off
+
+        // groups that receive no tile of a piece never write its partial: mark those slots "absent" for the merge
+        auto close_piece = [&]() {
+            if (prev_row < 0) return;
+            const uint32_t n = fill - piece_f0;
+            for (uint32_t k = n; k < (uint32_t)NGROUPS; ++k) {
+                const int grp = (int)((piece_f0 + k) % NGROUPS);
+                const int64_t slot = ((int64_t)blockIdx.x + prev_row) * NGROUPS + grp;
+                if (lane < a.G) a.part_ml[slot * a.G + lane] = make_float2(-INFINITY, 0.f);
             }
-            if (!ok) break;
-            const int r = e / EPR, sg = e % EPR;
-            const int i = r / a.Hkv, hk = r % a.Hkv;
-            const int pe = __ldg(a.pref + e), pn = __ldg(a.pref + e + 1);
-            const int row_begin = __ldg(a.pref + r * EPR);
-            int T = __ldg(a.seq_lens + i);
-            T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
-            const int NB = T / a.b, tail = T - NB * a.b;
-            const int n_here = min(pn, u1) - u;
-            const int off = u - pe;
-            const bool is_tail = (sg == a.nseg);
-            const int32_t* list = a.seg_list + ((int64_t)r * a.nseg + sg) * LSTRIDE + off;
-            for (int base = 0; base < n_here && ok; base += 32) {
-                int my = 0;
-                if (base + lane < n_here) my = is_tail ? (NB | (0xff << 24)) : __ldg(list + base + lane);
-                const int nb = min(32, n_here - base);
-                for (int k = 0; k < nb && ok; ++k) {
-                    const int ent = __shfl_sync(0xffffffffu, my, k);
-                    const int uu = u + base + k;
-                    const int j = ent & 0xffffff;
-                    const int hmask = (ent >> 24) & 0xff;
-                    const int nrows = is_tail ? tail : a.b;
-                    if (uu == u0 || uu == row_begin) ++piece;      // a new (CTA, row) piece starts here
-                    for (int sub = 0; sub * TS < nrows && ok; ++sub) {
-                        const int nvalid = min(TS, nrows - sub * TS);
-                        const int stage = fill % NSTAGE;
-                        const uint32_t round = fill / NSTAGE;
-                        if (lane == 0) {
-                            if (!mbar_wait(&empty[stage], (round & 1) ^ 1)) {
-                                ok = false;
-                            } else {
-                                desc[stage] = make_int4(r, piece << 1, hmask, nvalid);
-                                unsigned char* st = smem + stage * L::STAGE_BYTES;
-                                mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
-                                const int y = j * a.b + sub * TS;
-#pragma unroll
-                                for (int hf = 0; hf < HALVES; ++hf) {
-                                    tma_load_4d(st + hf * L::TILE_BYTES, &tmK, hf * 64, y, hk, i, &full[stage]);
-                                    tma_load_4d(st + (HALVES + hf) * L::TILE_BYTES, &tmV, hf * 64, y, hk, i, &full[stage]);
-                                }
-                            }
-                        }
-                        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                        ++fill;
-                    }
+        };
+
+        auto load_window = [&]() {
+            __syncwarp();
+            for (int k = lane; k <= PW; k += 32) {
+                const int e = e_base + k;
+                pwin[k] = (e >= E) ? U : rowbase[e / EPR] + __ldg(a.row_pref + e);
+            }
+            __syncwarp();
+        };
+        auto search = [&](int uu) {          // largest k in [0, PW) with pwin[k] <= uu
+            int lo = 0, hi = PW - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (pwin[mid] <= uu) lo = mid; else hi = mid - 1;
+            }
+            return lo;
+        };
+        // make the window hold the entry of unit ub; -> number of units of the batch starting at ub
+        auto batch_size = [&](int ub) {
+            while (true) {
+                const bool reaches_end = (e_base + PW >= E);
+                const int wend = pwin[PW];
+                const int want = min(32, u1 - ub);
+                if (reaches_end || wend >= ub + want) return want;
+                if (wend <= ub) { e_base += PW; load_window(); continue; }
+                const int k0 = search(ub);
+                if (k0 == 0) return min(want, wend - ub);
+                e_base += k0;
+                load_window();
+            }
+        };
+        // per-lane description of unit ub + lane (row < 0: no such unit in this batch)
+        auto fetch = [&](int ub, int nb, int& row, int& ent, int& nrows) {
+            row = -1; ent = 0; nrows = 0;
+            if (lane < nb) {
+                const int uu = ub + lane;
+                const int k = search(uu);
+                const int e = e_base + k;
+                const int r = e / EPR, sg = e % EPR;
+                row = r;
+                if (sg == a.nseg) {
+                    int T = __ldg(a.seq_lens + r / a.Hkv);
+                    T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
+                    const int NB = T / a.b;
+                    ent = NB | (0xff << 24);
+                    nrows = T - NB * a.b;
+                } else {
+                    ent = __ldg(a.seg_list + ((int64_t)r * a.nseg + sg) * LSTRIDE + (uu - pwin[k]));
+                    nrows = a.b;
                 }
             }
-            u += n_here;
+        };
+
+        load_window();
+        int u = u0;
+        int nb = batch_size(u);
+        int c_row, c_ent, c_nrows;
+        fetch(u, nb, c_row, c_ent, c_nrows);
+        while (u < u1 && ok) {
+            // the next batch's loads are in flight while this batch is issued
+            const int un = u + nb;
+            int nbn = 0, n_row = -1, n_ent = 0, n_nrows = 0;
+            if (un < u1) {
+                nbn = batch_size(un);
+                fetch(un, nbn, n_row, n_ent, n_nrows);
+            }
+            for (int k = 0; k < nb && ok; ++k) {
+                const int r = __shfl_sync(0xffffffffu, c_row, k);
+                const int ent = __shfl_sync(0xffffffffu, c_ent, k);
+                const int nrows = __shfl_sync(0xffffffffu, c_nrows, k);
+                const int j = ent & 0xffffff;
+                const int hmask = (ent >> 24) & 0xff;
+                const int i = r / a.Hkv, hk = r % a.Hkv;
+                if (r != prev_row) {                               // a new (CTA, row) piece starts here
+                    close_piece();
+                    ++piece; prev_row = r; piece_f0 = fill;
+                }
+                for (int sub = 0; sub * TS < nrows && ok; ++sub) {
+                    const int nvalid = min(TS, nrows - sub * TS);
+                    const int stage = fill % NSTAGE;
+                    const uint32_t round = fill / NSTAGE;
+                    if (lane == 0) {
+                        if (tl && fill == 0) tl[2] = globaltimer_ns();
+                        if (!mbar_wait(&empty[stage], (round & 1) ^ 1)) {
+                            ok = false;
+                        } else {
+                            desc[stage] = make_int4(r, piece << 1, hmask, nvalid);
+                            unsigned char* st = smem + stage * L::STAGE_BYTES;
+                            mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
+                            const int y = j * a.b + sub * TS;
+#pragma unroll
+                            for (int hf = 0; hf < HALVES; ++hf) {
+                                tma_load_4d(st + hf * L::TILE_BYTES, &tmK, hf * 64, y, hk, i, &full[stage]);
+                                tma_load_4d(st + (HALVES + hf) * L::TILE_BYTES, &tmV, hf * 64, y, hk, i, &full[stage]);
+                            }
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                    ++fill;
+                }
+            }
+            u = un;
+            nb = nbn; c_row = n_row; c_ent = n_ent; c_nrows = n_nrows;
         }
+        close_piece();
+        pdl_trigger();       // everything is issued: the merge kernel may start to set up
         // one end marker per group (no data): the next NGROUPS fills reach every group exactly once
         for (int k = 0; k < NGROUPS && ok; ++k) {
             const int stage = fill % NSTAGE;
@@ -223,9 +343,26 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     uint32_t qa[HALVES][2][4];
     float o[HALVES][4][4];
     float m_run = -INFINITY, l_run = 0.f, te = 0.f;
-    int row = -1, piece = -1;
+    int row = -1, piece = -1, q_row = -1;
     uint32_t flush_phase = 0;
     bool ok = true;
+
+    // query fragments and threshold of a row: head g's slice in the permuted head_dim order of the MMA
+    auto load_q = [&](int r) {
+        const int i = r / a.Hkv, hk = r % a.Hkv;
+        const __nv_bfloat16* qp = a.q + ((int64_t)i * a.Hq + hk * a.G + (head ? g : 0)) * D;
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf)
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (head) v = __ldg(reinterpret_cast<const uint4*>(qp + 64 * hf + 32 * m + 8 * t));
+                qa[hf][m][0] = v.x; qa[hf][m][1] = v.y; qa[hf][m][2] = v.z; qa[hf][m][3] = v.w;
+            }
+        te = head ? __ldg(a.tau_eff + (int64_t)i * a.Hq + hk * a.G + g) : 0.f;
+        q_row = r;
+    };
+    load_q(row0);       // the row of the CTA's first unit: fetched while the producer sets up
 
     for (uint32_t fill = group;; fill += NGROUPS) {
         const int stage = fill % NSTAGE;
@@ -233,6 +370,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const int4 ds = desc[stage];
         const bool end = (ds.y & (int)UF_END) != 0;
         const int new_piece = ds.y >> 1;
+        if (end) pdl_trigger();
+        if (tl && warp == 0 && lane == 0) {
+            if (fill == 0) tl[3] = globaltimer_ns();
+            if (end) tl[4] = globaltimer_ns();
+        }
 
         if ((end || new_piece != piece) && piece >= 0) {
             // ---- this group's part of a piece is complete: combine its four warps and store (m, l, O) per head
@@ -274,7 +416,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             if (!mbar_wait(&flushbar[group], flush_phase)) { ok = false; break; }
             flush_phase ^= 1;
         }
-        if (end) break;
+        if (end) {
+            if (tl && warp == 0 && lane == 0) tl[5] = globaltimer_ns();
+            break;
+        }
 
         const int hmask = ds.z, nvalid = ds.w;
         const uint32_t kbase = smem_u32(smem + stage * L::STAGE_BYTES);
@@ -283,17 +428,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         if (new_piece != piece) {
             piece = new_piece;
             row = ds.x;
-            const int i = row / a.Hkv, hk = row % a.Hkv;
-            const __nv_bfloat16* qp = a.q + ((int64_t)i * a.Hq + hk * a.G + (head ? g : 0)) * D;
-#pragma unroll
-            for (int hf = 0; hf < HALVES; ++hf)
-#pragma unroll
-                for (int m = 0; m < 2; ++m) {
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (head) v = __ldg(reinterpret_cast<const uint4*>(qp + 64 * hf + 32 * m + 8 * t));
-                    qa[hf][m][0] = v.x; qa[hf][m][1] = v.y; qa[hf][m][2] = v.z; qa[hf][m][3] = v.w;
-                }
-            te = head ? __ldg(a.tau_eff + (int64_t)i * a.Hq + hk * a.G + g) : 0.f;
+            if (row != q_row) load_q(row);
             m_run = -INFINITY;
             l_run = 0.f;
 #pragma unroll
@@ -434,7 +569,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
 // Associative merge of the pieces of one (sequence, query head): Algorithm 3, global reduction.
 struct MergeArgs {
-    const int32_t* pref;
+    const int32_t* row_start;
     const int32_t* hdr;
     const float2* part_ml;
     const float* part_o;
@@ -456,8 +591,9 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
-    const int EPR = a.nseg + 1;
-    const int ra = a.pref[r * EPR], rbd = a.pref[(r + 1) * EPR];
+    pdl_trigger();
+    pdl_wait();          // every partial of the streaming kernel is in memory from here on
+    const int ra = a.row_start[r], rbd = a.row_start[r + 1];
     const int64_t U = a.hdr[0], P = a.hdr[1];
     float acc[VPL];
 #pragma unroll
@@ -586,7 +722,9 @@ static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const
         if (e != cudaSuccess) { set_cuda_error(e, "decode smem attribute"); return ETA_ERR_CUDA; }
         configured = smem;
     }
-    decode_kernel<D, TS, NSTAGE, NGROUPS><<<n_ctas, 32 * (WARPS_PER_GROUP * NGROUPS + 1), smem, s>>>(tmK, tmV, a);
+    cudaError_t e = launch_pdl(decode_kernel<D, TS, NSTAGE, NGROUPS>, dim3(n_ctas),
+                               dim3(32 * (WARPS_PER_GROUP * NGROUPS + 1)), smem, s, tmK, tmV, a);
+    if (e != cudaSuccess) { set_cuda_error(e, "decode launch"); return ETA_ERR_CUDA; }
     return check_launch("decode");
 }
 
@@ -594,7 +732,7 @@ static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const
 
 extern "C" {
 
-int eta_decode_kernel_count(void) { return 4; }
+int eta_decode_kernel_count(void) { return 3; }
 
 int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q, const void* K, const void* V,
                const int32_t* seq_lens, const void* musig, const float* mnorm, const float* tau,
@@ -614,7 +752,6 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     const WsLayout L = ws_layout(desc);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
         return ETA_ERR_WORKSPACE;
-    if (L.entries > MAX_ENTRIES) return ETA_ERR_UNSUPPORTED;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -646,27 +783,16 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     sa.seg_resc = reinterpret_cast<RescueRec*>(ws + L.seg_resc);
     sa.tau_eff = reinterpret_cast<float*>(ws + L.tau_eff);
     sa.sel_mask = sel_mask;
+    sa.timeline = debug_timeline();
+    sa.row_ticket = reinterpret_cast<int32_t*>(ws + L.row_ticket);
+    sa.row_pref = reinterpret_cast<int32_t*>(ws + L.row_pref);
+    sa.row_total = reinterpret_cast<int32_t*>(ws + L.row_total);
+    sa.stats = stats;
+    sa.status = status_dev;
     profile_mark(2, s);
     rc = launch_screen(sa, L.rows, D, G, s);
     profile_mark(3, s);
     if (rc != ETA_OK) return rc;
-
-    PlanArgs pa;
-    pa.seq_lens = seq_lens;
-    pa.Hkv = desc->n_kv_heads; pa.G = G; pa.b = b; pa.t_cap = desc->t_cap; pa.nb_cap = desc->nb_cap;
-    pa.nseg = L.nseg; pa.rows = L.rows; pa.entries = L.entries; pa.rescue_window = params->rescue_window;
-    pa.n_ctas = n_ctas;
-    pa.seg_count = sa.seg_count; pa.seg_list = sa.seg_list; pa.seg_resc = sa.seg_resc; pa.sel_mask = sel_mask;
-    pa.pref = reinterpret_cast<int32_t*>(ws + L.pref);
-    pa.cta_start = reinterpret_cast<int4*>(ws + L.cta_start);
-    pa.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
-    pa.stats = stats;
-    pa.status = status_dev;
-    pa.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
-    pa.n_part = (n_ctas + L.rows) * DECODE_GROUPS * G;
-    rc = launch_plan(pa, s);
-    if (rc != ETA_OK) return rc;
-    profile_mark(4, s);
 
     CUtensorMap tmK, tmV;
     rc = make_tmap(&tmK, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t, TS);
@@ -675,14 +801,17 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     if (rc != ETA_OK) return rc;
 
     DecodeArgs da;
-    da.q = sa.q; da.seq_lens = seq_lens; da.tau_eff = sa.tau_eff; da.seg_list = sa.seg_list; da.pref = pa.pref;
-    da.cta_start = pa.cta_start;
+    da.q = sa.q; da.seq_lens = seq_lens; da.tau_eff = sa.tau_eff; da.seg_list = sa.seg_list;
+    da.row_pref = sa.row_pref; da.row_total = sa.row_total;
+    da.row_start = reinterpret_cast<int32_t*>(ws + L.row_start);
+    da.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
     da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
     da.part_o = reinterpret_cast<float*>(ws + L.part_o);
     da.status = status_dev;
     da.beta = params->beta; da.scale = scale;
     da.Hq = desc->n_q_heads; da.Hkv = desc->n_kv_heads; da.G = G; da.b = b; da.t_cap = desc->t_cap;
-    da.nseg = L.nseg; da.entries = L.entries;
+    da.nseg = L.nseg; da.entries = L.entries; da.rows = L.rows;
+    da.timeline = debug_timeline();
     if (D == 128 && TS == 64) {
         rc = (G == 8) ? launch_decode_t<128, 64, 5, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s)
                       : launch_decode_t<128, 64, 6, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s);
@@ -694,15 +823,16 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
         rc = launch_decode_t<64, 32, 8, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s);
     }
     if (rc != ETA_OK) return rc;
-    profile_mark(5, s);
+    profile_mark(4, s);
 
     MergeArgs ma;
-    ma.pref = pa.pref; ma.hdr = pa.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
+    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
     ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS;
     const unsigned mgrid = (unsigned)(L.rows * G);
-    if (D == 128) merge_kernel<128><<<mgrid, 32 * MERGE_WARPS, 0, s>>>(ma);
-    else merge_kernel<64><<<mgrid, 32 * MERGE_WARPS, 0, s>>>(ma);
-    profile_mark(6, s);
+    cudaError_t me = (D == 128) ? launch_pdl(merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
+                                : launch_pdl(merge_kernel<64>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma);
+    if (me != cudaSuccess) { set_cuda_error(me, "merge launch"); return ETA_ERR_CUDA; }
+    profile_mark(5, s);
     return check_launch("merge");
 }
 

@@ -26,6 +26,7 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     const int NRG = PRED_THREADS / Hq;           // row groups inside a CTA
     float* part = sm;                            // [NRG][Hq] partial sums of this CTA
     float* cpart = sm + NRG * Hq;                // [PRED_CLUSTER][Hq], used in the cluster's first CTA
+    pdl_trigger();
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank();
     const int i = blockIdx.y;
@@ -65,6 +66,7 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
         for (int c = 0; c < PRED_CLUSTER; ++c) s += cpart[c * Hq + threadIdx.x];
         tau[(int64_t)i * Hq + threadIdx.x] = s + bias[threadIdx.x];
     }
+    if (threadIdx.x == 0) pdl_wait();
 }
 
 }  // namespace eta
@@ -84,13 +86,18 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
     cfg.blockDim = dim3(eta::PRED_THREADS, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = eta::PRED_CLUSTER;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // the predictor reads nothing an earlier kernel of the stream writes, so it may run beside its predecessor
+    // (typically the summary append); it only waits for it before it exits, which keeps "this kernel is complete"
+    // meaning "everything before it is complete" for whoever comes next
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = eta::pdl_enabled() ? 1 : 0;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     eta::profile_mark(1, cfg.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, eta::predict_threshold_kernel, static_cast<const __nv_bfloat16*>(q), W,
                                        bias, tau, (int)n_q_heads, rows);

@@ -1,6 +1,5 @@
 // Screening stage of eta_decode (Eq. dual_bound_eq; Algorithm 3, screening and
-// rescue lines) and the planning step that turns its output into balanced work
-// for the streaming kernel.
+// rescue lines).
 //
 // screen_kernel: one CTA per (row = sequence x KV head, segment of SEG block
 // records).  The segment's records (centroid and sigma, fp16) are one
@@ -14,9 +13,10 @@
 // are compacted per segment with ballot + popc prefix sums.  Nothing returns
 // to the host.
 //
-// plan_kernel: a single CTA.  Resolves top-1 rescue per query head, scans the
-// per-segment survivor counts into a global unit prefix and gives each
-// streaming CTA an equal, contiguous share of the units.
+// The CTA that finishes a row last (a ticket per row) closes the row: it
+// resolves top-1 rescue per query head from the per-segment window statistics
+// and scans the row's survivor counts into a per-row unit prefix, which is all
+// the streaming kernel needs to split the work evenly.
 #include "eta_common.cuh"
 
 namespace eta {
@@ -52,11 +52,17 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
     const int n_rec = max(0, min(SEG, NB - j0));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool dense = (a.flags & ETA_FLAG_DENSE) != 0;
+    const int cta_lin = blockIdx.y * gridDim.x + blockIdx.x;
+    unsigned long long* tl = (a.timeline && cta_lin < 512) ? a.timeline + (size_t)(512 + cta_lin) * 8 : nullptr;
+    if (tl && tid == 0) tl[0] = globaltimer_ns();
 
-    // thresholds of the G heads of this group (tau_eff = tau - a)
     const int cc = lane % LPR, rg = lane / LPR;
     const int my_g = cc % G;
     const int my_h = hk * G + my_g;
+    // everything above reads only the caller's inputs; the summaries and thresholds may still be in the making
+    pdl_wait();
+    if (tl && tid == 0) tl[1] = globaltimer_ns();
+    // thresholds of the G heads of this group (tau_eff = tau - a)
     float my_te = (a.tau ? a.tau[(int64_t)i * a.Hq + my_h] : a.head_const[my_h]) - a.a;
     if (dense) my_te = -INFINITY;
     if (seg == 0 && tid < G) {
@@ -66,11 +72,14 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
     }
     // mask entries of this segment that are not full blocks read as "not attended"
     if (tid < SEG && tid >= n_rec && j0 + tid < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = 0;
-    if (n_rec == 0) {
-        if (tid == 0) a.seg_count[r * a.nseg + seg] = 0;
-        return;
+    if (n_rec == 0 && tid == 0) a.seg_count[r * a.nseg + seg] = 0;
+    if (seg == 0 && tid == 0 && a.status) {
+        const int Traw = a.seq_lens[i];
+        if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
+        if (Traw <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
     }
 
+    if (n_rec > 0) {
     if (!dense) {
         if (tid == 0) {
 #pragma unroll
@@ -117,6 +126,7 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
 #pragma unroll
         for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
         __syncthreads();   // smn visible
+        if (tl && tid == 0) tl[2] = globaltimer_ns();
 
         for (int base = warp * RB; base < n_rec; base += 8 * RB) {
             // wait (bounded) for the chunks this batch reads
@@ -190,6 +200,8 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
         if (tid < n_rec) smask[tid] = (uint8_t)((1u << G) - 1u);
     }
     __syncthreads();
+    if (tl && tid == 0) tl[3] = globaltimer_ns();
+    pdl_trigger();       // the bulk of this CTA's work is done: the plan kernel may start to set up
 
     // user-visible admission bits
     if (tid < n_rec) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = smask[tid];
@@ -207,6 +219,7 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
             carry += __popc(nz);
         }
         if (lane == 0) a.seg_count[r * a.nseg + seg] = carry;
+        if (tl && lane == 0) tl[4] = globaltimer_ns();
     }
 
     // rescue statistics of the part of the rescue window inside this segment, per query head
@@ -238,38 +251,33 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
             a.seg_resc[((int64_t)r * a.nseg + seg) * G + g] = rr;
         }
     }
-}
+    }   // n_rec > 0
 
-__global__ void __launch_bounds__(1024) plan_kernel(const PlanArgs a) {
-    extern __shared__ int32_t pref_s[];          // [entries + 1]
-    __shared__ int32_t warp_sum[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // ---- row ticket: the CTA that finishes this row last closes it
+    __shared__ int s_last;
+    __shared__ int s_warp_sum[8];
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(a.row_ticket + r, 1) == a.nseg - 1) ? 1 : 0;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
 
-    // partial slots a streaming group never writes must read as "absent" in the merge
-    for (int k = tid; k < a.n_part; k += 1024) a.part_ml[k] = make_float2(-INFINITY, 0.f);
-
-    // ---- top-1 rescue, one warp per row (Algorithm 3: rescue phase of the first chunk).  Lane (g, s) reads the
-    // window statistics of head g in window segment s, all at once; four segments (256 blocks) per pass.
-    for (int r = warp; r < a.rows; r += 32) {
-        const int i = r / a.Hkv;
-        int T = a.seq_lens[i];
-        if (lane == 0 && a.status) {
-            if (T > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
-            if (T <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
-        }
-        T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
-        const int NB = min(T / a.b, a.nb_cap);
-        const int Wr = min(a.rescue_window, NB);
-        const int nsw = (Wr + SEG - 1) / SEG;
-        if (Wr <= 0) continue;
+    // top-1 rescue (Algorithm 3, rescue phase of the first chunk): warp 0, lane (g, s) reads the window statistics
+    // of head g in window segment s; four segments (256 blocks) per pass
+    const int Wr_row = min(a.rescue_window, NB);
+    if (warp == 0 && Wr_row > 0) {
+        const int nsw = (Wr_row + SEG - 1) / SEG;
         const int g = lane >> 2, s4 = lane & 3;
         int cnt = 0, arg = 0x7fffffff;
         float best = -INFINITY;
-        if (g < a.G) {
+        if (g < G) {
             for (int s = s4; s < nsw; s += 4) {
-                const RescueRec rr = a.seg_resc[((int64_t)r * a.nseg + s) * a.G + g];
-                cnt += rr.cnt;
-                if (rr.arg >= 0 && rr.maxb > best) { best = rr.maxb; arg = rr.arg; }
+                const RescueRec* rp = a.seg_resc + ((int64_t)r * a.nseg + s) * G + g;
+                const int4 raw = __ldcg(reinterpret_cast<const int4*>(rp));
+                cnt += raw.x;
+                const float mb = __int_as_float(raw.y);
+                if (raw.z >= 0 && mb > best) { best = mb; arg = raw.z; }
             }
         }
 #pragma unroll
@@ -279,7 +287,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(const PlanArgs a) {
             const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
             if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
         }
-        unsigned need = __ballot_sync(0xffffffffu, g < a.G && s4 == 0 && cnt == 0);
+        unsigned need = __ballot_sync(0xffffffffu, g < G && s4 == 0 && cnt == 0);
         while (need) {
             const int src = __ffs(need) - 1;
             need &= need - 1;
@@ -288,87 +296,58 @@ __global__ void __launch_bounds__(1024) plan_kernel(const PlanArgs a) {
             const int j = (ja == 0x7fffffff) ? 0 : ja;
             const int s = j / SEG;
             int32_t* list = a.seg_list + ((int64_t)r * a.nseg + s) * LSTRIDE;
-            const int n = a.seg_count[r * a.nseg + s];
+            const int n = __ldcg(a.seg_count + r * a.nseg + s);
             int found = -1;
             for (int k = lane; k < n; k += 32)
-                if ((list[k] & 0xffffff) == j) found = k;
+                if ((__ldcg(list + k) & 0xffffff) == j) found = k;
             const unsigned fb = __ballot_sync(0xffffffffu, found >= 0);
             if (fb) {
-                if (found >= 0) list[found] |= 1 << (24 + gg);
+                if (found >= 0) list[found] = __ldcg(list + found) | (1 << (24 + gg));
             } else if (lane == 0) {
                 list[n] = j | (1 << (24 + gg));
                 a.seg_count[r * a.nseg + s] = n + 1;
             }
-            if (lane == 0) a.sel_mask[(int64_t)r * a.nb_cap + j] |= (uint8_t)(1u << gg);
-            __threadfence_block();
+            if (lane == 0) {
+                uint8_t* mp = a.sel_mask + (int64_t)r * a.nb_cap + j;
+                const unsigned w = *reinterpret_cast<volatile uint8_t*>(mp);
+                *mp = (uint8_t)(w | (1u << gg));
+            }
+            __threadfence();
             __syncwarp();
         }
     }
     __syncthreads();
 
-    // ---- exclusive prefix of units over (row, segment) entries; the last entry of a row is its tail unit
-    const int E = a.entries;
-    const int per = (E + 1023) / 1024;
-    const int e0 = min(E, tid * per), e1 = min(E, e0 + per);
-    int local = 0;
-    for (int e = e0; e < e1; ++e) {
-        const int r = e / (a.nseg + 1), s = e % (a.nseg + 1);
-        int c;
-        if (s < a.nseg) {
-            c = a.seg_count[r * a.nseg + s];
-        } else {
-            int T = a.seq_lens[r / a.Hkv];
-            T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
-            c = (T % a.b) ? 1 : 0;
-        }
-        pref_s[e] = c;      // own slots only; turned into the prefix below
-        local += c;
-    }
-    int incl = local;
-    for (int s = 1; s < 32; s <<= 1) {
-        const int o = __shfl_up_sync(0xffffffffu, incl, s);
-        if (lane >= s) incl += o;
-    }
-    if (lane == 31) warp_sum[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        int w = warp_sum[lane];
-        int wi = w;
+    // exclusive prefix of the row's survivor counts; the entry after the last segment holds the block total
+    int32_t* rp = a.row_pref + (int64_t)r * (a.nseg + 1);
+    int carry = 0;
+    for (int s0 = 0; s0 < a.nseg; s0 += 256) {
+        const int sgi = s0 + tid;
+        const int c = (sgi < a.nseg) ? __ldcg(a.seg_count + r * a.nseg + sgi) : 0;
+        int incl = c;
+#pragma unroll
         for (int s = 1; s < 32; s <<= 1) {
-            const int o = __shfl_up_sync(0xffffffffu, wi, s);
-            if (lane >= s) wi += o;
+            const int o = __shfl_up_sync(0xffffffffu, incl, s);
+            if (lane >= s) incl += o;
         }
-        warp_sum[lane] = wi - w;   // exclusive
-    }
-    __syncthreads();
-    int run = warp_sum[warp] + incl - local;
-    for (int e = e0; e < e1; ++e) {
-        const int c = pref_s[e];
-        pref_s[e] = run;
-        a.pref[e] = run;
-        run += c;
-    }
-    if (tid == 1023) { pref_s[E] = run; a.pref[E] = run; }
-    __syncthreads();
-
-    const int U = pref_s[E];
-    if (tid == 0) { a.hdr[0] = U; a.hdr[1] = a.n_ctas; }
-    if (a.stats) {
-        for (int r = tid; r < a.rows; r += 1024) {
-            int T = a.seq_lens[r / a.Hkv];
-            T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
-            a.stats[r] = pref_s[(r + 1) * (a.nseg + 1)] - pref_s[r * (a.nseg + 1)] - ((T % a.b) ? 1 : 0);
+        if (lane == 31) s_warp_sum[warp] = incl;
+        __syncthreads();
+        int wbase = 0, tot = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            const int v = s_warp_sum[w];
+            if (w < warp) wbase += v;
+            tot += v;
         }
+        if (sgi < a.nseg) rp[sgi] = carry + wbase + incl - c;
+        carry += tot;
+        __syncthreads();
     }
-    // ---- equal contiguous shares of the unit sequence for the streaming CTAs
-    for (int c = tid; c < a.n_ctas; c += 1024) {
-        const int u0 = (int)(((int64_t)c * U) / a.n_ctas), u1 = (int)(((int64_t)(c + 1) * U) / a.n_ctas);
-        int lo = 0, hi = E;              // last e with pref[e] <= u0
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (pref_s[mid] <= u0) lo = mid; else hi = mid - 1;
-        }
-        a.cta_start[c] = make_int4(u0, u1, min(lo, E - 1), 0);
+    if (tid == 0) {
+        rp[a.nseg] = carry;
+        a.row_total[r] = carry + ((T % a.b) ? 1 : 0);      // the tail, when there is one, is one more unit
+        if (a.stats) a.stats[r] = carry;
+        a.row_ticket[r] = 0;                                // ready for the next call
     }
 }
 
@@ -411,7 +390,8 @@ __global__ void __launch_bounds__(128) score_dual_kernel(
 template <int D, int G>
 static void launch_screen_t(const ScreenArgs& a, int rows, cudaStream_t s) {
     dim3 grid(a.nseg, rows);
-    screen_kernel<D, G><<<grid, 256, 0, s>>>(a);
+    cudaError_t e = launch_pdl(screen_kernel<D, G>, grid, dim3(256), 0, s, a);
+    if (e != cudaSuccess) set_cuda_error(e, "screen launch");
 }
 
 int launch_screen(const ScreenArgs& a, int rows, int D, int G, cudaStream_t s) {
@@ -420,17 +400,6 @@ int launch_screen(const ScreenArgs& a, int rows, int D, int G, cudaStream_t s) {
     ETA_CASE(64, 1) ETA_CASE(64, 2) ETA_CASE(64, 4) ETA_CASE(64, 8)
 #undef ETA_CASE
     return ETA_ERR_UNSUPPORTED;
-}
-
-int launch_plan(const PlanArgs& a, cudaStream_t s) {
-    const size_t smem = sizeof(int32_t) * ((size_t)a.entries + 1);
-    if (a.entries > MAX_ENTRIES) return ETA_ERR_UNSUPPORTED;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { set_cuda_error(e, "plan smem attribute"); return ETA_ERR_CUDA; }
-    }
-    plan_kernel<<<1, 1024, smem, s>>>(a);
-    return check_launch("plan");
 }
 
 }  // namespace eta

@@ -180,6 +180,7 @@ __global__ void __launch_bounds__(SUM_THREADS) append_summary_kernel(
     const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig, float* __restrict__ mnorm) {
     const int r = blockIdx.x;
     const int i = r / Hkv, hk = r % Hkv;
+    pdl_trigger();       // nothing later in a decode step needs this kernel's output before it has waited for it
     const int T = seq_lens[i];
     if (T <= 0 || T > t_cap || T % b != 0) return;
     const int j = T / b - 1;

@@ -58,9 +58,9 @@ def test_static_scratch_variant_matches_eta_decode_twice_in_a_row():
 def test_static_scratch_variant_refuses_shapes_beyond_its_limit():
     from paper_2609_20888_b200 import binding as eb
     lib = eb.load()
-    # 256 sequences x 8 KV heads x 64K tokens: needs far more than 8 MiB of scratch; refused before any launch
-    d = eb.CacheDesc(256, 32, 8, 128, 64, 65536, 1024, 8 * 65536 * 128, 65536 * 128, 128, 8 * 65536 * 128,
-                     65536 * 128, 128)
+    # 64 sequences x 8 KV heads x 512K tokens: needs far more than 8 MiB of scratch; refused before any launch
+    T = 512 * 1024
+    d = eb.CacheDesc(64, 32, 8, 128, 64, T, T // 64, 8 * T * 128, T * 128, 128, 8 * T * 128, T * 128, 128)
     assert eb.eta_workspace_bytes(d) > eb.eta_static_scratch_bytes()
     p = eb.DecodeParams().c()
     one, null = ctypes.c_void_p(256), ctypes.c_void_p(None)
