@@ -83,11 +83,9 @@ typedef struct eta_params {
 
 /*
  * Bytes of scratch eta_decode needs for this cache shape (independent of the
- * sequence lengths).  The caller allocates it once, 256-byte aligned, ZERO-FILLS
- * it before the first call, and may then reuse it across calls on the same
- * stream without touching it: a successful call leaves it ready for the next
- * one (its first batch * n_kv_heads words are per-row tickets that every call
- * returns to zero).  After a call that reported ETA_DEV_TIMEOUT, zero it again.
+ * sequence lengths).  The caller allocates it once, 256-byte aligned, and may
+ * reuse it across calls on the same stream; it carries no state between calls
+ * (every word is written before it is read) and needs no initialisation.
  * No device is touched by this function.
  */
 int eta_workspace_bytes(const eta_cache_desc* desc, size_t* out_bytes);
@@ -179,10 +177,9 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
  *   - Set-up: the first call on each device looks up the array's device address (with that device current).
  *     Make that first call ahead of any stream capture.
  *   - Sharing: all calls on a device use the same array, and it keeps the previous call's contents.  Nothing in
- *     it has to be cleared by the caller: the array starts zeroed when the library is loaded, every call
- *     returns its per-row tickets to zero, and every other word is written before it is read.  Two calls
- *     whose kernels can overlap on the GPU (different streams, no dependency between them) race on the array
- *     and corrupt each other; calls on one stream, or otherwise ordered, are fine.
+ *     it has to be cleared by the caller: each call writes every word before reading it.  For the same reason
+ *     two calls whose kernels can overlap on the GPU (different streams, no dependency between them) race on
+ *     the array and corrupt each other; calls on one stream, or otherwise ordered, are fine.
  */
 #define ETA_STATIC_SCRATCH_BYTES (8u << 20)
 int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, const void* q,

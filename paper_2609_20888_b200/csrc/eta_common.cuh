@@ -38,14 +38,11 @@ constexpr int DECODE_GROUPS = 3;     // consumer groups per streaming CTA, each 
 struct WsLayout {
     int rows;        // batch * n_kv_heads
     int nseg;        // segments per row
-    int entries;     // rows * (nseg + 1): one pseudo-segment per row holds the tail unit
-    size_t row_ticket;  // int32 [rows]: ZERO between calls (the only part of the scratch that carries state)
+    int entries;     // rows * (nseg + 2): per row its segments, a rescue pseudo-entry and a tail pseudo-entry
     size_t hdr;         // int32[8]: [0] total units U, [1] streaming CTAs P (written by the streaming kernel)
     size_t seg_count;   // int32 [rows * nseg]
     size_t seg_list;    // int32 [rows * nseg * LSTRIDE]: block index | head bits << 24
     size_t seg_resc;    // {int cnt; float maxb; int arg; int pad} [rows * nseg * G]
-    size_t row_pref;    // int32 [entries]: exclusive prefix of survivor counts inside each row
-    size_t row_total;   // int32 [rows]: units per row
     size_t row_start;   // int32 [rows + 1]: global unit prefix over rows (written by the streaming kernel)
     size_t tau_eff;     // float [batch * n_q_heads]
     size_t part_ml;     // float2 [(MAX_CTAS + rows) * DECODE_GROUPS * G]
@@ -67,20 +64,16 @@ struct ScreenArgs {
     float z, a, scale;
     int lwb, rescue_window;
     uint32_t flags;
-    int Hq, Hkv, b, t_cap, nb_cap, nseg;
+    int Hq, Hkv, b, t_cap, nb_cap, nseg, rows;
     int32_t* seg_count;
     int32_t* seg_list;
     RescueRec* seg_resc;
     float* tau_eff;
     uint8_t* sel_mask;
-    int32_t* row_ticket;   // [rows] zero between calls
-    int32_t* row_pref;     // [rows * (nseg + 1)] exclusive prefix of survivor counts inside each row
-    int32_t* row_total;    // [rows] units of the row (surviving blocks + tail)
-    int32_t* stats;
     uint32_t* status;
     unsigned long long* timeline;
 };
-int launch_screen(const ScreenArgs& a, int rows, int D, int G, cudaStream_t s);
+int launch_screen(const ScreenArgs& a, int rows, int D, int G, int n_ctas, cudaStream_t s);
 
 // Launch with programmatic dependent launch allowed: the grid may start while its predecessor in the stream is
 // still draining, and must call pdl_wait() before touching anything the predecessor wrote.
@@ -143,8 +136,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: false when the limit ran out (the caller then abandons the work
 // and reports ETA_DEV_TIMEOUT instead of spinning forever).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (it >= 2) __nanosleep(40);      // leave the issue slots to the warps that have work
+    }
     return false;
 }
 

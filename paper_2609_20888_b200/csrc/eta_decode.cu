@@ -30,21 +30,23 @@ struct DecodeArgs {
     const int32_t* seq_lens;
     const float* tau_eff;
     const int32_t* seg_list;
-    const int32_t* row_pref;
-    const int32_t* row_total;
+    const int32_t* seg_count;
+    const RescueRec* seg_resc;
+    uint8_t* sel_mask;
+    int32_t* stats;
     int32_t* row_start;
     int32_t* hdr;
     float2* part_ml;
     float* part_o;
     uint32_t* status;
     float beta, scale;
-    int Hq, Hkv, G, b, t_cap, nseg, entries, rows;
+    int Hq, Hkv, G, b, t_cap, nb_cap, nseg, entries, rows, rescue_window;
     unsigned long long* timeline;
 };
 
 constexpr uint32_t UF_END = 1u;
 constexpr int WARPS_PER_GROUP = 4;     // the four warps of a group each take a quarter of a tile's tokens
-constexpr int PW = 512;                // entries of the unit prefix the producer keeps in shared memory
+constexpr int PW = 256;                // entries of the unit prefix the producer keeps in shared memory
 
 __device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
     return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
@@ -58,6 +60,63 @@ __device__ __forceinline__ float rcp_approx(float x) {
     return y;
 }
 
+
+// Top-1 rescue of query head g of row r (Algorithm 3, rescue phase): if none of the first
+// Wr = min(rescue_window, NB) blocks was admitted for the head, the first block with the largest bound among them
+// is.  Combines the per-segment statistics the screening kernel left.  -> rescued block index, or -1.
+__device__ __forceinline__ int rescue_of(const RescueRec* __restrict__ seg_resc, int r, int g, int G, int nseg,
+                                          int Wr) {
+    if (Wr <= 0) return -1;
+    const int nsw = (Wr + SEG - 1) / SEG;
+    int cnt = 0, arg = -1;
+    float best = -INFINITY;
+    for (int s0 = 0; s0 < nsw; s0 += 4) {
+        int4 raw[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)          // four segments' statistics in flight at once
+            raw[k] = (s0 + k < nsw) ? __ldg(reinterpret_cast<const int4*>(seg_resc + ((int64_t)r * nseg + s0 + k) * G + g))
+                                    : make_int4(0, 0, -1, 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            cnt += raw[k].x;
+            const float mb = __int_as_float(raw[k].y);
+            if (raw[k].z >= 0 && mb > best) { best = mb; arg = raw[k].z; }   // ascending segments: ties keep the lowest index
+        }
+    }
+    if (cnt != 0) return -1;
+    return arg < 0 ? 0 : arg;
+}
+
+// The rescued blocks of a row as fetch units: heads that rescue the same block share one unit.
+// -> number of units; unit k is block uj[k] with head bits um[k].
+__device__ __forceinline__ int rescue_units(const RescueRec* __restrict__ seg_resc, int r, int G, int nseg, int Wr,
+                                            int (&uj)[8], int (&um)[8]) {
+    int n = 0;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        uj[g] = -1; um[g] = 0;
+    }
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        if (g < G) {
+            const int j = rescue_of(seg_resc, r, g, G, nseg, Wr);
+            if (j >= 0) {
+                bool merged = false;
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (k < n && uj[k] == j) { um[k] |= 1 << g; merged = true; }
+                if (!merged) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (k == n) { uj[k] = j; um[k] = 1 << g; }
+                    ++n;
+                }
+            }
+        }
+    }
+    return n;
+}
+
 template <int D, int TS, int NSTAGE, int NGROUPS>
 struct DecodeSmem {
     static constexpr int HALVES = D / 64;
@@ -67,7 +126,8 @@ struct DecodeSmem {
     static constexpr int DESC_OFF = BAR_OFF + 8 * (2 * NSTAGE + NGROUPS + (NGROUPS & 1));
     static constexpr int WIN_OFF = DESC_OFF + 16 * NSTAGE;      // int32 pwin[PW + 1] (+3 pad): window of the unit prefix
     static constexpr int ROW_OFF = WIN_OFF + 4 * (PW + 4);      // int32 rowbase[MAX_ROWS + 1]: unit prefix over rows
-    static constexpr int ML_OFF = ROW_OFF + 4 * (MAX_ROWS + 4); // float m[NGROUPS][4][8], l[NGROUPS][4][8]
+    static constexpr int INFO_OFF = ROW_OFF + 4 * (MAX_ROWS + 4);   // uint8 per row: rescue units | tail flag << 7
+    static constexpr int ML_OFF = INFO_OFF + MAX_ROWS;          // float m[NGROUPS][4][8], l[NGROUPS][4][8]
     static constexpr int MO_OFF = ML_OFF + 4 * 2 * NGROUPS * WARPS_PER_GROUP * 8;
     static size_t bytes(int G) { return 1024 + MO_OFF + sizeof(float) * NGROUPS * WARPS_PER_GROUP * G * D; }
 };
@@ -94,6 +154,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     int4* desc = reinterpret_cast<int4*>(smem + L::DESC_OFF);
     int32_t* pwin = reinterpret_cast<int32_t*>(smem + L::WIN_OFF);
     int32_t* rowbase = reinterpret_cast<int32_t*>(smem + L::ROW_OFF);
+    uint8_t* rowinfo = smem + L::INFO_OFF;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long* tl = a.timeline ? a.timeline + (size_t)blockIdx.x * 8 : nullptr;
@@ -105,17 +166,80 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         prefetch_tmap(&tmK);
         prefetch_tmap(&tmV);
     }
+    // scratch for the layout, in the (still unused) stage memory
+    constexpr int NWARPS = WARPS_PER_GROUP * NGROUPS + 1;
+    constexpr int NTHREADS = 32 * NWARPS;
+    int* cnt32 = reinterpret_cast<int*>(smem);                 // [rows] surviving blocks of the row
+    int* resc_j = cnt32 + MAX_ROWS;                            // [rows][8] rescued block per head, -1: none
+    int* s_len = resc_j + 8 * MAX_ROWS;                        // [rows] clamped sequence length
+    uint8_t* cnt8 = reinterpret_cast<uint8_t*>(s_len + MAX_ROWS);   // [rows * nseg] survivors per segment
+    const bool counts_in_smem = (size_t)a.rows * a.nseg + 10 * 4 * MAX_ROWS <= (size_t)NSTAGE * L::STAGE_BYTES;
+    // sequence lengths are a caller input: they can be read while the previous kernel is still running
+    for (int rr = tid; rr < a.rows; rr += NTHREADS) {
+        const int T = __ldg(a.seq_lens + rr / a.Hkv);
+        s_len[rr] = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
+        cnt32[rr] = 0;
+    }
     __syncthreads();
-    pdl_wait();          // the screening kernel's lists, row prefixes and row totals are complete from here on
+    pdl_wait();          // the screening kernel's lists, counts and window statistics are complete from here on
 
-    // ---- every CTA derives its own share of the flattened unit sequence: scan of the per-row unit totals
+    // ---- every CTA lays out the flattened unit sequence for itself: per row the surviving blocks of its
+    // segments, then its rescued blocks, then its tail; a scan over the rows gives each row's first unit
     {
         __shared__ int s_wsum[32];
-        const int nthreads = 32 * (WARPS_PER_GROUP * NGROUPS + 1);
+        // all loads of the layout are independent and issued together: segment counts (summed per row with
+        // shared-memory atomics) and, per (row, head), the window statistics of the rescue window's segments
+        for (int e0 = tid; e0 < a.rows * a.nseg; e0 += 8 * NTHREADS) {
+            int cv[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * NTHREADS;
+                cv[k] = (e < a.rows * a.nseg) ? __ldg(a.seg_count + e) : 0;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * NTHREADS;
+                if (e < a.rows * a.nseg) {
+                    if (counts_in_smem) cnt8[e] = (uint8_t)cv[k];
+                    if (cv[k]) atomicAdd(&cnt32[e / a.nseg], cv[k]);
+                }
+            }
+        }
+        for (int p = tid; p < a.rows * a.G; p += NTHREADS) {
+            const int rr = p / a.G, g = p % a.G;
+            const int NB = min(s_len[rr] / a.b, a.nb_cap);
+            resc_j[rr * 8 + g] = rescue_of(a.seg_resc, rr, g, a.G, a.nseg, min(a.rescue_window, NB));
+        }
+        __syncthreads();
+        for (int rr = tid; rr < a.rows; rr += NTHREADS) {
+            const int tailf = (s_len[rr] % a.b) ? 1 : 0;
+            // heads that rescue the same block share one unit
+            int resc = 0, extra = 0;
+            for (int g = 0; g < a.G; ++g) {
+                const int j = resc_j[rr * 8 + g];
+                if (j < 0) continue;
+                bool dup = false;
+                for (int g2 = 0; g2 < g; ++g2) dup = dup || (resc_j[rr * 8 + g2] == j);
+                if (!dup) ++resc;
+                if (blockIdx.x == 0) {
+                    // the first CTA publishes the rescued heads' admission bits
+                    uint8_t* mp = a.sel_mask + (int64_t)rr * a.nb_cap + j;
+                    const unsigned w = *mp;
+                    if (w == 0) ++extra;          // a block no head had admitted: one more block fetched
+                    *mp = (uint8_t)(w | (1u << g));
+                }
+            }
+            rowinfo[rr] = (uint8_t)(resc | (tailf << 7));
+            const int c = cnt32[rr];
+            rowbase[rr] = c + resc + tailf;          // units of the row; turned into the prefix below
+            if (blockIdx.x == 0 && a.stats) a.stats[rr] = c + extra;
+        }
+        __syncthreads();
+        const int nthreads = NTHREADS;
         int carry = 0;
         for (int r0 = 0; r0 < a.rows; r0 += nthreads) {
             const int rr = r0 + tid;
-            const int c = (rr < a.rows) ? __ldg(a.row_total + rr) : 0;
+            const int c = (rr < a.rows) ? rowbase[rr] : 0;
             int incl = c;
 #pragma unroll
             for (int s = 1; s < 32; s <<= 1) {
@@ -125,7 +249,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             if (lane == 31) s_wsum[warp] = incl;
             __syncthreads();
             int wbase = 0, tot = 0;
-            for (int w = 0; w < nthreads / 32; ++w) {
+            for (int w = 0; w < NWARPS; ++w) {
                 const int v = s_wsum[w];
                 if (w < warp) wbase += v;
                 tot += v;
@@ -164,9 +288,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         // entry e_base on): each lane finds the entry of one unit by binary search in the window and fetches that
         // unit's list word, so a batch of up to 32 units costs one round trip to L2, and the next batch is fetched
         // while the current one is being issued.
-        const int EPR = a.nseg + 1;
+        const int EPR = a.nseg + 2;        // per row: its segments, then the rescue entry, then the tail entry
         const int E = a.entries;
         int e_base = row0 * EPR;
+        int base_units = rowbase[row0];    // units before entry e_base
         uint32_t fill = 0;
         int piece = -1, prev_row = -1;
         uint32_t piece_f0 = 0;
@@ -183,12 +308,34 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
         };
 
+        // units of entry e: survivors of a segment, rescue units of the row, or the row's tail
+        bool first_window = counts_in_smem;     // the counts of the layout phase are still in the stage memory
+        auto entry_count = [&](int e) {
+            if (e >= E) return 0;
+            const int r = e / EPR, sg = e % EPR;
+            if (sg < a.nseg) return first_window ? (int)cnt8[r * a.nseg + sg] : (int)__ldg(a.seg_count + r * a.nseg + sg);
+            const int info = rowinfo[r];
+            return sg == a.nseg ? (info & 0x7f) : (info >> 7);
+        };
+        // pwin[k] = units before entry e_base + k, k = 0 .. PW (PW a multiple of 32): a warp scan, 32 entries a round
         auto load_window = [&]() {
             __syncwarp();
-            for (int k = lane; k <= PW; k += 32) {
-                const int e = e_base + k;
-                pwin[k] = (e >= E) ? U : rowbase[e / EPR] + __ldg(a.row_pref + e);
+            int cw[PW / 32];
+#pragma unroll
+            for (int m = 0; m < PW / 32; ++m) cw[m] = entry_count(e_base + 32 * m + lane);   // all loads in flight
+            int run = base_units;
+#pragma unroll
+            for (int m = 0; m < PW / 32; ++m) {
+                int incl = cw[m];
+#pragma unroll
+                for (int s = 1; s < 32; s <<= 1) {
+                    const int o = __shfl_up_sync(0xffffffffu, incl, s);
+                    if (lane >= s) incl += o;
+                }
+                pwin[32 * m + lane] = run + incl - cw[m];
+                run += __shfl_sync(0xffffffffu, incl, 31);
             }
+            if (lane == 0) pwin[PW] = run;
             __syncwarp();
         };
         auto search = [&](int uu) {          // largest k in [0, PW) with pwin[k] <= uu
@@ -206,9 +353,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const int wend = pwin[PW];
                 const int want = min(32, u1 - ub);
                 if (reaches_end || wend >= ub + want) return want;
-                if (wend <= ub) { e_base += PW; load_window(); continue; }
+                if (wend <= ub) { e_base += PW; base_units = wend; load_window(); continue; }
                 const int k0 = search(ub);
                 if (k0 == 0) return min(want, wend - ub);
+                base_units = pwin[k0];
                 e_base += k0;
                 load_window();
             }
@@ -222,12 +370,25 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const int e = e_base + k;
                 const int r = e / EPR, sg = e % EPR;
                 row = r;
-                if (sg == a.nseg) {
+                if (sg >= a.nseg) {
                     int T = __ldg(a.seq_lens + r / a.Hkv);
                     T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
-                    const int NB = T / a.b;
-                    ent = NB | (0xff << 24);
-                    nrows = T - NB * a.b;
+                    const int NB = min(T / a.b, a.nb_cap);
+                    if (sg == a.nseg) {
+                        // a rescued block, attended by the rescued head(s) only
+                        int uj[8], um[8];
+                        rescue_units(a.seg_resc, r, a.G, a.nseg, min(a.rescue_window, NB), uj, um);
+                        const int idx = uu - pwin[k];
+                        int j = 0, m = 0;
+#pragma unroll
+                        for (int q8 = 0; q8 < 8; ++q8)
+                            if (q8 == idx) { j = uj[q8]; m = um[q8]; }
+                        ent = j | (m << 24);
+                        nrows = a.b;
+                    } else {
+                        ent = NB | (0xff << 24);           // the tail: every head attends it
+                        nrows = T - NB * a.b;
+                    }
                 } else {
                     ent = __ldg(a.seg_list + ((int64_t)r * a.nseg + sg) * LSTRIDE + (uu - pwin[k]));
                     nrows = a.b;
@@ -236,10 +397,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         };
 
         load_window();
+        first_window = false;       // from the first copy on, the stage memory belongs to the tiles
+        if (tl && lane == 0) tl[6] = globaltimer_ns();
         int u = u0;
         int nb = batch_size(u);
         int c_row, c_ent, c_nrows;
         fetch(u, nb, c_row, c_ent, c_nrows);
+        if (tl && lane == 0) tl[7] = globaltimer_ns() + (c_ent & 0);
         while (u < u1 && ok) {
             // the next batch's loads are in flight while this batch is issued
             const int un = u + nb;
@@ -777,20 +941,16 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     sa.z = params->z; sa.a = params->a; sa.scale = scale;
     sa.lwb = params->lwb; sa.rescue_window = params->rescue_window; sa.flags = params->flags;
     sa.Hq = desc->n_q_heads; sa.Hkv = desc->n_kv_heads; sa.b = b; sa.t_cap = desc->t_cap; sa.nb_cap = desc->nb_cap;
-    sa.nseg = L.nseg;
+    sa.nseg = L.nseg; sa.rows = L.rows;
     sa.seg_count = reinterpret_cast<int32_t*>(ws + L.seg_count);
     sa.seg_list = reinterpret_cast<int32_t*>(ws + L.seg_list);
     sa.seg_resc = reinterpret_cast<RescueRec*>(ws + L.seg_resc);
     sa.tau_eff = reinterpret_cast<float*>(ws + L.tau_eff);
     sa.sel_mask = sel_mask;
     sa.timeline = debug_timeline();
-    sa.row_ticket = reinterpret_cast<int32_t*>(ws + L.row_ticket);
-    sa.row_pref = reinterpret_cast<int32_t*>(ws + L.row_pref);
-    sa.row_total = reinterpret_cast<int32_t*>(ws + L.row_total);
-    sa.stats = stats;
     sa.status = status_dev;
     profile_mark(2, s);
-    rc = launch_screen(sa, L.rows, D, G, s);
+    rc = launch_screen(sa, L.rows, D, G, 2 * n_sm, s);
     profile_mark(3, s);
     if (rc != ETA_OK) return rc;
 
@@ -802,7 +962,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
 
     DecodeArgs da;
     da.q = sa.q; da.seq_lens = seq_lens; da.tau_eff = sa.tau_eff; da.seg_list = sa.seg_list;
-    da.row_pref = sa.row_pref; da.row_total = sa.row_total;
+    da.seg_count = sa.seg_count; da.seg_resc = sa.seg_resc; da.sel_mask = sel_mask; da.stats = stats;
     da.row_start = reinterpret_cast<int32_t*>(ws + L.row_start);
     da.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
     da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
@@ -810,7 +970,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.status = status_dev;
     da.beta = params->beta; da.scale = scale;
     da.Hq = desc->n_q_heads; da.Hkv = desc->n_kv_heads; da.G = G; da.b = b; da.t_cap = desc->t_cap;
-    da.nseg = L.nseg; da.entries = L.entries; da.rows = L.rows;
+    da.nseg = L.nseg; da.entries = L.entries; da.rows = L.rows; da.nb_cap = desc->nb_cap;
+    da.rescue_window = params->rescue_window;
     da.timeline = debug_timeline();
     if (D == 128 && TS == 64) {
         rc = (G == 8) ? launch_decode_t<128, 64, 5, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s)

@@ -60,9 +60,9 @@ int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, cons
     void* scratch = nullptr;
     rc = eta::static_scratch_ptr(&scratch);
     if (rc != ETA_OK) return rc;
-    // the array is zero when the module is loaded and every call returns its per-row tickets to zero; every other
-    // word a kernel reads is written earlier in the same call, so nothing carried over from the previous call
-    // is ever consumed
+    // every word of the scratch that a kernel reads is written earlier in the same call (counts, lists and window
+    // statistics by the screening kernel, partial slots by the streaming kernel), so nothing carried over from
+    // the previous call is ever consumed
     return eta_decode(desc, params, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask, stats,
                       status_dev, scratch, eta::STATIC_SCRATCH_BYTES, stream);
 }

@@ -13,10 +13,10 @@
 // are compacted per segment with ballot + popc prefix sums.  Nothing returns
 // to the host.
 //
-// The CTA that finishes a row last (a ticket per row) closes the row: it
-// resolves top-1 rescue per query head from the per-segment window statistics
-// and scans the row's survivor counts into a per-row unit prefix, which is all
-// the streaming kernel needs to split the work evenly.
+// Top-1 rescue needs the whole rescue window of a head, which may span several
+// segments: this kernel only leaves per-segment window statistics (admitted
+// count, largest bound and its index per head); the streaming kernel combines
+// them when it lays out its work.
 #include "eta_common.cuh"
 
 namespace eta {
@@ -27,328 +27,284 @@ __device__ __forceinline__ float min_keep_nan(float g, float s) {
 }
 
 template <int D, int G>
+struct ScreenSmem {
+    static constexpr int REC_BYTES = 4 * D;                    // fp16 mu[d] + fp16 sigma[d]
+    static constexpr int BUF_BYTES = SEG * REC_BYTES + G * D * 2;   // a segment's records, then the group's queries
+    static constexpr int BAR_OFF = 2 * BUF_BYTES;
+    static constexpr int BOUND_OFF = BAR_OFF + 16;
+    static constexpr int MN_OFF = BOUND_OFF + 4 * SEG * G;
+    static constexpr int MASK_OFF = MN_OFF + 4 * SEG;
+    static constexpr int MISC_OFF = MASK_OFF + SEG;            // int s_last, int warp sums[8]
+    static constexpr int LEN_OFF = MISC_OFF + 64;              // int32 clamped sequence lengths [MAX_ROWS]
+    static constexpr int BYTES = LEN_OFF + 4 * MAX_ROWS + 128; // + slack for the 128-byte alignment of the base
+};
+
+// Persistent screening kernel: every CTA owns a contiguous range of (row, segment) items and double-buffers
+// them, so the records (and the group's queries) of the next item are in flight while the current one is
+// evaluated.
+template <int D, int G>
 __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
+    using L = ScreenSmem<D, G>;
     constexpr int LPR = D / 8;            // lanes sharing one record
     constexpr int RPW = 32 / LPR;         // records per warp instruction
     constexpr int NI = LPR / G;           // iterations whose partial sums are reduced together
     constexpr int NV = 2 * LPR;           // partial sums per lane before the butterfly
     constexpr int RB = RPW * NI;          // records per warp per batch
-    constexpr int REC_BYTES = 4 * D;      // fp16 mu[d] + fp16 sigma[d]
+    constexpr int REC_BYTES = L::REC_BYTES;
     constexpr bool USE_Q2 = (G <= 4);
     static_assert(NI >= 1, "group size too large for this head_dim");
 
-    __shared__ __align__(128) unsigned char srec[SEG * REC_BYTES];
-    __shared__ __align__(8) uint64_t bars[4];
-    __shared__ float sbound[SEG][G];
-    __shared__ float smn[SEG];
-    __shared__ uint8_t smask[SEG];
+    extern __shared__ unsigned char scr_raw[];
+    unsigned char* sm = scr_raw + ((128u - (smem_u32(scr_raw) & 127u)) & 127u);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::BAR_OFF);
+    float (*sbound)[G] = reinterpret_cast<float (*)[G]>(sm + L::BOUND_OFF);
+    float* smn = reinterpret_cast<float*>(sm + L::MN_OFF);
+    uint8_t* smask = sm + L::MASK_OFF;
+    int* s_len = reinterpret_cast<int*>(sm + L::LEN_OFF);
 
-    const int seg = blockIdx.x, r = blockIdx.y;
-    const int i = r / a.Hkv, hk = r % a.Hkv;
-    int T = a.seq_lens[i];
-    T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
-    const int NB = min(T / a.b, a.nb_cap);
-    const int j0 = seg * SEG;
-    const int n_rec = max(0, min(SEG, NB - j0));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool dense = (a.flags & ETA_FLAG_DENSE) != 0;
-    const int cta_lin = blockIdx.y * gridDim.x + blockIdx.x;
-    unsigned long long* tl = (a.timeline && cta_lin < 512) ? a.timeline + (size_t)(512 + cta_lin) * 8 : nullptr;
+    unsigned long long* tl = (a.timeline && blockIdx.x < 512) ? a.timeline + (size_t)(512 + blockIdx.x) * 8 : nullptr;
     if (tl && tid == 0) tl[0] = globaltimer_ns();
 
+    const int n_items = a.rows * a.nseg;
+    const int it0 = (int)(((int64_t)blockIdx.x * n_items) / gridDim.x);
+    const int it1 = (int)(((int64_t)(blockIdx.x + 1) * n_items) / gridDim.x);
     const int cc = lane % LPR, rg = lane / LPR;
     const int my_g = cc % G;
-    const int my_h = hk * G + my_g;
-    // everything above reads only the caller's inputs; the summaries and thresholds may still be in the making
+
+    if (tid == 0) {
+        mbar_init(&bars[0], 1);
+        mbar_init(&bars[1], 1);
+        fence_barrier_init();
+    }
+    // sequence lengths (a caller input) of every row, clamped, once: the per-item geometry then needs no global load
+    for (int rr = tid; rr < a.rows; rr += 256) {
+        const int T = a.seq_lens[rr / a.Hkv];
+        s_len[rr] = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
+    }
+    __syncthreads();
+    // everything above touches only this CTA; the summaries and thresholds may still be in the making
     pdl_wait();
     if (tl && tid == 0) tl[1] = globaltimer_ns();
-    // thresholds of the G heads of this group (tau_eff = tau - a)
-    float my_te = (a.tau ? a.tau[(int64_t)i * a.Hq + my_h] : a.head_const[my_h]) - a.a;
-    if (dense) my_te = -INFINITY;
-    if (seg == 0 && tid < G) {
-        int h = hk * G + tid;
-        float te = (a.tau ? a.tau[(int64_t)i * a.Hq + h] : a.head_const[h]) - a.a;
-        a.tau_eff[(int64_t)i * a.Hq + h] = dense ? -INFINITY : te;
-    }
-    // mask entries of this segment that are not full blocks read as "not attended"
-    if (tid < SEG && tid >= n_rec && j0 + tid < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = 0;
-    if (n_rec == 0 && tid == 0) a.seg_count[r * a.nseg + seg] = 0;
-    if (seg == 0 && tid == 0 && a.status) {
-        const int Traw = a.seq_lens[i];
-        if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
-        if (Traw <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
-    }
+    if (it0 >= it1) return;
 
-    if (n_rec > 0) {
-    if (!dense) {
-        if (tid == 0) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) mbar_init(&bars[c], 1);
-            fence_barrier_init();
-        }
-        __syncthreads();
-        if (tid == 0) {
+    // geometry of an item
+    auto item_geom = [&](int item, int& r, int& seg, int& i, int& hk, int& T, int& NB, int& j0, int& n_rec) {
+        r = item / a.nseg; seg = item % a.nseg;
+        i = r / a.Hkv; hk = r % a.Hkv;
+        T = s_len[r];
+        NB = min(T / a.b, a.nb_cap);
+        j0 = seg * SEG;
+        n_rec = max(0, min(SEG, NB - j0));
+    };
+    // one thread starts the copies of an item into buffer `buf`
+    auto issue = [&](int item, int buf) {
+        int r, seg, i, hk, T, NB, j0, n_rec;
+        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
+        if (n_rec > 0 && !dense) {
+            unsigned char* dst = sm + buf * L::BUF_BYTES;
             const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
                                        ((int64_t)r * a.nb_cap + j0) * REC_BYTES;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                int n = min(16, n_rec - 16 * c);
-                if (n > 0) {
-                    mbar_arrive_expect_tx(&bars[c], n * REC_BYTES);
-                    tma_load_1d(srec + c * 16 * REC_BYTES, src + (size_t)c * 16 * REC_BYTES, n * REC_BYTES, &bars[c]);
-                }
-            }
+            mbar_arrive_expect_tx(&bars[buf], n_rec * REC_BYTES + G * D * 2);
+            tma_load_1d(dst, src, n_rec * REC_BYTES, &bars[buf]);
+            tma_load_1d(dst + SEG * REC_BYTES, a.q + ((int64_t)i * a.Hq + hk * G) * D, G * D * 2, &bars[buf]);
+        } else {
+            mbar_arrive(&bars[buf]);      // nothing to copy: the phase completes at once
         }
-        if (tid < n_rec) smn[tid] = a.mnorm[(int64_t)r * a.nb_cap + j0 + tid];
+    };
+    // per-thread prefetch of the small per-item scalars (largest-norm entry of record tid, threshold of head my_g)
+    auto prefetch_scalars = [&](int item, float& mnv, float& te) {
+        int r, seg, i, hk, T, NB, j0, n_rec;
+        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
+        mnv = (tid < n_rec && !dense) ? __ldg(a.mnorm + (int64_t)r * a.nb_cap + j0 + tid) : 0.f;
+        const int h = hk * G + my_g;
+        te = dense ? -INFINITY : ((a.tau ? __ldg(a.tau + (int64_t)i * a.Hq + h) : __ldg(a.head_const + h)) - a.a);
+    };
 
-        // this lane's slice of the G query vectors, in fp32
-        float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)i * a.Hq + hk * G + g) * D + cc * 8));
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-            float n2 = 0.f;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                qf[g][2 * k] = bf16_lo(w[k]);
-                qf[g][2 * k + 1] = bf16_hi(w[k]);
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                n2 = fmaf(qf[g][k], qf[g][k], n2);
-                if (USE_Q2) q2[g][k] = qf[g][k] * qf[g][k];
-            }
-#pragma unroll
-            for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
-            qn[g] = sqrtf(n2);
+    if (tid == 0) issue(it0, 0);
+    float mn_cur, te_cur;
+    prefetch_scalars(it0, mn_cur, te_cur);
+
+    for (int item = it0; item < it1; ++item) {
+        const int k = item - it0, buf = k & 1;
+        int r, seg, i, hk, T, NB, j0, n_rec;
+        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
+        float mn_next = 0.f, te_next = 0.f;
+        if (item + 1 < it1) {
+            if (tid == 0) issue(item + 1, buf ^ 1);
+            prefetch_scalars(item + 1, mn_next, te_next);
         }
-        float my_qn = qn[0];
-#pragma unroll
-        for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
-        __syncthreads();   // smn visible
-        if (tl && tid == 0) tl[2] = globaltimer_ns();
+        const float my_te = te_cur;
+        if (tid < SEG) smn[tid] = mn_cur;
+        if (seg == 0 && tid < G) a.tau_eff[(int64_t)i * a.Hq + hk * G + tid] = my_te;     // lane g < G holds head g
+        if (seg == 0 && tid == 0 && a.status) {
+            const int Traw = __ldg(a.seq_lens + i);
+            if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
+            if (Traw <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
+        }
+        // mask entries of this segment that are not full blocks read as "not attended"
+        if (tid < SEG && tid >= n_rec && j0 + tid < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = 0;
+        if (n_rec == 0 && tid == 0) a.seg_count[r * a.nseg + seg] = 0;
 
-        for (int base = warp * RB; base < n_rec; base += 8 * RB) {
-            // wait (bounded) for the chunks this batch reads
-            const int c_lo = base / 16, c_hi = min(3, (min(base + RB, n_rec) - 1) / 16);
-            bool ok = true;
-            for (int c = c_lo; c <= c_hi; ++c) ok = mbar_wait(&bars[c], 0) && ok;
-            ok = __all_sync(0xffffffffu, ok);
-            // a wait that ran out: admit everything in this batch (errs toward loading) - never seen in practice
-            float v[NV];
-#pragma unroll
-            for (int it = 0; it < NI; ++it) {
-                const int rec = base + it * RPW + rg;
-                float mu[8], s2[8];
-                if (rec < n_rec && ok) {
-                    const uint32_t addr = smem_u32(srec) + rec * REC_BYTES + cc * 16;
-                    const uint4 m4 = lds128(addr), s4 = lds128(addr + 2 * D);
-                    const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw[k]));
-                        float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[k]));
-                        mu[2 * k] = mf.x; mu[2 * k + 1] = mf.y;
-                        s2[2 * k] = USE_Q2 ? sf.x * sf.x : sf.x;
-                        s2[2 * k + 1] = USE_Q2 ? sf.y * sf.y : sf.y;
-                    }
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) { mu[k] = 0.f; s2[k] = 0.f; }
-                }
+        bool ok = mbar_wait(&bars[buf], (k >> 1) & 1);
+        ok = __all_sync(0xffffffffu, ok);
+        __syncthreads();       // smn visible
+        if (tl && tid == 0 && item == it0) tl[2] = globaltimer_ns();
+
+        if (n_rec > 0) {
+            const uint32_t rec_base = smem_u32(sm + buf * L::BUF_BYTES);
+            if (!dense) {
+                // this lane's slice of the G query vectors, in fp32
+                float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G];
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    float dot = 0.f, var = 0.f;
+                    const uint4 v = lds128(rec_base + SEG * REC_BYTES + (g * D + cc * 8) * 2);
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                    float n2 = 0.f;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        dot = fmaf(qf[g][k], mu[k], dot);
-                        if (USE_Q2) {
-                            var = fmaf(q2[g][k], s2[k], var);
+                    for (int kk = 0; kk < 4; ++kk) {
+                        qf[g][2 * kk] = bf16_lo(w[kk]);
+                        qf[g][2 * kk + 1] = bf16_hi(w[kk]);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        n2 = fmaf(qf[g][kk], qf[g][kk], n2);
+                        if (USE_Q2) q2[g][kk] = qf[g][kk] * qf[g][kk];
+                    }
+#pragma unroll
+                    for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+                    qn[g] = sqrtf(n2);
+                }
+                float my_qn = qn[0];
+#pragma unroll
+                for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
+
+                for (int base = warp * RB; base < n_rec; base += 8 * RB) {
+                    // a wait that ran out: admit everything (errs toward loading) - never seen in practice
+                    float v[NV];
+#pragma unroll
+                    for (int it = 0; it < NI; ++it) {
+                        const int rec = base + it * RPW + rg;
+                        float mu[8], s2[8];
+                        if (rec < n_rec && ok) {
+                            const uint32_t addr = rec_base + rec * REC_BYTES + cc * 16;
+                            const uint4 m4 = lds128(addr), s4 = lds128(addr + 2 * D);
+                            const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) {
+                                float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw[kk]));
+                                float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
+                                mu[2 * kk] = mf.x; mu[2 * kk + 1] = mf.y;
+                                s2[2 * kk] = USE_Q2 ? sf.x * sf.x : sf.x;
+                                s2[2 * kk + 1] = USE_Q2 ? sf.y * sf.y : sf.y;
+                            }
                         } else {
-                            const float t = qf[g][k] * s2[k];
-                            var = fmaf(t, t, var);
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) { mu[kk] = 0.f; s2[kk] = 0.f; }
+                        }
+#pragma unroll
+                        for (int g = 0; g < G; ++g) {
+                            float dot = 0.f, var = 0.f;
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) {
+                                dot = fmaf(qf[g][kk], mu[kk], dot);
+                                if (USE_Q2) {
+                                    var = fmaf(q2[g][kk], s2[kk], var);
+                                } else {
+                                    const float t = qf[g][kk] * s2[kk];
+                                    var = fmaf(t, t, var);
+                                }
+                            }
+                            v[(it * G + g) * 2] = dot;
+                            v[(it * G + g) * 2 + 1] = var;
                         }
                     }
-                    v[(it * G + g) * 2] = dot;
-                    v[(it * G + g) * 2 + 1] = var;
+                    // transposed butterfly over the LPR lanes of a record: halves the values held at every step
+#pragma unroll
+                    for (int s = LPR / 2, n = NV / 2; s >= 1; s >>= 1, n >>= 1) {
+                        const bool upper = (lane & s) != 0;
+#pragma unroll
+                        for (int kk = 0; kk < n; ++kk) {
+                            const float send = upper ? v[kk] : v[kk + n];
+                            const float keep = upper ? v[kk + n] : v[kk];
+                            v[kk] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+                        }
+                    }
+                    // lane cc now holds (dot, var) of pair cc = it * G + g
+                    const int it = cc / G;
+                    const int rec = base + it * RPW + rg;
+                    const bool valid = rec < n_rec;
+                    const float mnv = valid ? smn[rec] : 0.f;
+                    const float bound = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * mnv);
+                    const bool pinned = (j0 + rec) >= NB - a.lwb;
+                    const bool admit = valid && (!(bound < my_te) || pinned || !ok);
+                    if (valid) sbound[rec][my_g] = bound;
+                    const unsigned bal = __ballot_sync(0xffffffffu, admit);
+                    if (valid && my_g == 0) smask[rec] = (uint8_t)((bal >> lane) & ((1u << G) - 1u));
+                }
+            } else {
+                if (tid < n_rec) smask[tid] = (uint8_t)((1u << G) - 1u);
+            }
+            __syncthreads();
+            if (tl && tid == 0 && item == it0) tl[3] = globaltimer_ns();
+
+            // user-visible admission bits
+            if (tid < n_rec) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = smask[tid];
+
+            // segment-local compaction of the union (ballot + popc prefix), ascending block order
+            if (warp == 7) {
+                int carry = 0;
+                int32_t* list = a.seg_list + ((int64_t)r * a.nseg + seg) * LSTRIDE;
+#pragma unroll
+                for (int half = 0; half < SEG / 32; ++half) {
+                    const int rec = half * 32 + lane;
+                    const unsigned m = (rec < n_rec) ? smask[rec] : 0u;
+                    const unsigned nz = __ballot_sync(0xffffffffu, m != 0);
+                    if (m) list[carry + __popc(nz & ((1u << lane) - 1u))] = (j0 + rec) | (int)(m << 24);
+                    carry += __popc(nz);
+                }
+                if (lane == 0) a.seg_count[r * a.nseg + seg] = carry;
+            }
+
+            // rescue statistics of the part of the rescue window inside this segment, per query head
+            const int Wr = min(a.rescue_window, NB);
+            if (j0 < Wr && warp < G) {
+                const int g = warp;
+                const int nwin = min(n_rec, Wr - j0);
+                int cnt = 0, arg = 0x7fffffff;
+                float best = -INFINITY;
+#pragma unroll
+                for (int half = 0; half < SEG / 32; ++half) {
+                    const int rec = half * 32 + lane;
+                    if (rec < nwin) {
+                        cnt += (smask[rec] >> g) & 1;
+                        const float bd = dense ? 0.f : sbound[rec][g];
+                        if (bd > best) { best = bd; arg = rec; }
+                    }
+                }
+#pragma unroll
+                for (int s = 16; s >= 1; s >>= 1) {
+                    cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
+                    const float ob = __shfl_xor_sync(0xffffffffu, best, s);
+                    const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
+                    if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+                }
+                if (lane == 0) {
+                    RescueRec rr;
+                    rr.cnt = cnt; rr.maxb = best; rr.arg = (arg == 0x7fffffff) ? -1 : (j0 + arg); rr.pad = 0;
+                    a.seg_resc[((int64_t)r * a.nseg + seg) * G + g] = rr;
                 }
             }
-            // transposed butterfly over the LPR lanes of a record: halves the values held at every step
-#pragma unroll
-            for (int s = LPR / 2, n = NV / 2; s >= 1; s >>= 1, n >>= 1) {
-                const bool upper = (lane & s) != 0;
-#pragma unroll
-                for (int k = 0; k < n; ++k) {
-                    const float send = upper ? v[k] : v[k + n];
-                    const float keep = upper ? v[k + n] : v[k];
-                    v[k] = keep + __shfl_xor_sync(0xffffffffu, send, s);
-                }
-            }
-            // lane cc now holds (dot, var) of pair cc = it * G + g
-            const int it = cc / G;
-            const int rec = base + it * RPW + rg;
-            const bool valid = rec < n_rec;
-            const float mnv = valid ? smn[rec] : 0.f;
-            const float bound = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * mnv);
-            const bool pinned = (j0 + rec) >= NB - a.lwb;
-            const bool admit = valid && (!(bound < my_te) || pinned || !ok);
-            if (valid) sbound[rec][my_g] = bound;
-            const unsigned bal = __ballot_sync(0xffffffffu, admit);
-            if (valid && my_g == 0) smask[rec] = (uint8_t)((bal >> lane) & ((1u << G) - 1u));
-        }
-    } else {
-        if (tid < n_rec) smask[tid] = (uint8_t)((1u << G) - 1u);
-    }
-    __syncthreads();
-    if (tl && tid == 0) tl[3] = globaltimer_ns();
-    pdl_trigger();       // the bulk of this CTA's work is done: the plan kernel may start to set up
+        }   // n_rec > 0
 
-    // user-visible admission bits
-    if (tid < n_rec) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = smask[tid];
-
-    // segment-local compaction of the union (ballot + popc prefix), ascending block order
-    if (warp == 7) {
-        int carry = 0;
-        int32_t* list = a.seg_list + ((int64_t)r * a.nseg + seg) * LSTRIDE;
-#pragma unroll
-        for (int half = 0; half < SEG / 32; ++half) {
-            const int rec = half * 32 + lane;
-            const unsigned m = (rec < n_rec) ? smask[rec] : 0u;
-            const unsigned nz = __ballot_sync(0xffffffffu, m != 0);
-            if (m) list[carry + __popc(nz & ((1u << lane) - 1u))] = (j0 + rec) | (int)(m << 24);
-            carry += __popc(nz);
-        }
-        if (lane == 0) a.seg_count[r * a.nseg + seg] = carry;
-        if (tl && lane == 0) tl[4] = globaltimer_ns();
+        __syncthreads();       // the item's shared-memory state may be overwritten from here on
+        if (tl && tid == 0 && item == it0) tl[4] = globaltimer_ns();
+        mn_cur = mn_next;
+        te_cur = te_next;
     }
-
-    // rescue statistics of the part of the rescue window inside this segment, per query head
-    const int Wr = min(a.rescue_window, NB);
-    if (j0 < Wr && warp < G) {
-        const int g = warp;
-        const int nwin = min(n_rec, Wr - j0);
-        int cnt = 0, arg = 0x7fffffff;
-        float best = -INFINITY;
-#pragma unroll
-        for (int half = 0; half < SEG / 32; ++half) {
-            const int rec = half * 32 + lane;
-            if (rec < nwin) {
-                cnt += (smask[rec] >> g) & 1;
-                const float bd = dense ? 0.f : sbound[rec][g];
-                if (bd > best) { best = bd; arg = rec; }
-            }
-        }
-#pragma unroll
-        for (int s = 16; s >= 1; s >>= 1) {
-            cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
-            const float ob = __shfl_xor_sync(0xffffffffu, best, s);
-            const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
-            if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
-        }
-        if (lane == 0) {
-            RescueRec rr;
-            rr.cnt = cnt; rr.maxb = best; rr.arg = (arg == 0x7fffffff) ? -1 : (j0 + arg); rr.pad = 0;
-            a.seg_resc[((int64_t)r * a.nseg + seg) * G + g] = rr;
-        }
-    }
-    }   // n_rec > 0
-
-    // ---- row ticket: the CTA that finishes this row last closes it
-    __shared__ int s_last;
-    __shared__ int s_warp_sum[8];
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(a.row_ticket + r, 1) == a.nseg - 1) ? 1 : 0;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-
-    // top-1 rescue (Algorithm 3, rescue phase of the first chunk): warp 0, lane (g, s) reads the window statistics
-    // of head g in window segment s; four segments (256 blocks) per pass
-    const int Wr_row = min(a.rescue_window, NB);
-    if (warp == 0 && Wr_row > 0) {
-        const int nsw = (Wr_row + SEG - 1) / SEG;
-        const int g = lane >> 2, s4 = lane & 3;
-        int cnt = 0, arg = 0x7fffffff;
-        float best = -INFINITY;
-        if (g < G) {
-            for (int s = s4; s < nsw; s += 4) {
-                const RescueRec* rp = a.seg_resc + ((int64_t)r * a.nseg + s) * G + g;
-                const int4 raw = __ldcg(reinterpret_cast<const int4*>(rp));
-                cnt += raw.x;
-                const float mb = __int_as_float(raw.y);
-                if (raw.z >= 0 && mb > best) { best = mb; arg = raw.z; }
-            }
-        }
-#pragma unroll
-        for (int s = 1; s <= 2; s <<= 1) {
-            cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
-            const float ob = __shfl_xor_sync(0xffffffffu, best, s);
-            const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
-            if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
-        }
-        unsigned need = __ballot_sync(0xffffffffu, g < G && s4 == 0 && cnt == 0);
-        while (need) {
-            const int src = __ffs(need) - 1;
-            need &= need - 1;
-            const int gg = src >> 2;
-            const int ja = __shfl_sync(0xffffffffu, arg, src);
-            const int j = (ja == 0x7fffffff) ? 0 : ja;
-            const int s = j / SEG;
-            int32_t* list = a.seg_list + ((int64_t)r * a.nseg + s) * LSTRIDE;
-            const int n = __ldcg(a.seg_count + r * a.nseg + s);
-            int found = -1;
-            for (int k = lane; k < n; k += 32)
-                if ((__ldcg(list + k) & 0xffffff) == j) found = k;
-            const unsigned fb = __ballot_sync(0xffffffffu, found >= 0);
-            if (fb) {
-                if (found >= 0) list[found] = __ldcg(list + found) | (1 << (24 + gg));
-            } else if (lane == 0) {
-                list[n] = j | (1 << (24 + gg));
-                a.seg_count[r * a.nseg + s] = n + 1;
-            }
-            if (lane == 0) {
-                uint8_t* mp = a.sel_mask + (int64_t)r * a.nb_cap + j;
-                const unsigned w = *reinterpret_cast<volatile uint8_t*>(mp);
-                *mp = (uint8_t)(w | (1u << gg));
-            }
-            __threadfence();
-            __syncwarp();
-        }
-    }
-    __syncthreads();
-
-    // exclusive prefix of the row's survivor counts; the entry after the last segment holds the block total
-    int32_t* rp = a.row_pref + (int64_t)r * (a.nseg + 1);
-    int carry = 0;
-    for (int s0 = 0; s0 < a.nseg; s0 += 256) {
-        const int sgi = s0 + tid;
-        const int c = (sgi < a.nseg) ? __ldcg(a.seg_count + r * a.nseg + sgi) : 0;
-        int incl = c;
-#pragma unroll
-        for (int s = 1; s < 32; s <<= 1) {
-            const int o = __shfl_up_sync(0xffffffffu, incl, s);
-            if (lane >= s) incl += o;
-        }
-        if (lane == 31) s_warp_sum[warp] = incl;
-        __syncthreads();
-        int wbase = 0, tot = 0;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-            const int v = s_warp_sum[w];
-            if (w < warp) wbase += v;
-            tot += v;
-        }
-        if (sgi < a.nseg) rp[sgi] = carry + wbase + incl - c;
-        carry += tot;
-        __syncthreads();
-    }
-    if (tid == 0) {
-        rp[a.nseg] = carry;
-        a.row_total[r] = carry + ((T % a.b) ? 1 : 0);      // the tail, when there is one, is one more unit
-        if (a.stats) a.stats[r] = carry;
-        a.row_ticket[r] = 0;                                // ready for the next call
-    }
+    if (tl && tid == 0) tl[5] = globaltimer_ns();
+    pdl_trigger();
 }
 
 // Diagnostic evaluation of Eq. dual_bound_eq: one warp per (sequence, query head, block).
@@ -388,14 +344,23 @@ __global__ void __launch_bounds__(128) score_dual_kernel(
 // ------------------------------------------------------------------ launchers (host)
 
 template <int D, int G>
-static void launch_screen_t(const ScreenArgs& a, int rows, cudaStream_t s) {
-    dim3 grid(a.nseg, rows);
-    cudaError_t e = launch_pdl(screen_kernel<D, G>, grid, dim3(256), 0, s, a);
-    if (e != cudaSuccess) set_cuda_error(e, "screen launch");
+static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream_t s) {
+    const size_t smem = ScreenSmem<D, G>::BYTES;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(screen_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) { set_cuda_error(e, "screen smem attribute"); return ETA_ERR_CUDA; }
+        configured = true;
+    }
+    const int n_items = rows * a.nseg;
+    const int grid = n_items < n_ctas ? n_items : n_ctas;
+    cudaError_t e = launch_pdl(screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, a);
+    if (e != cudaSuccess) { set_cuda_error(e, "screen launch"); return ETA_ERR_CUDA; }
+    return check_launch("screen");
 }
 
-int launch_screen(const ScreenArgs& a, int rows, int D, int G, cudaStream_t s) {
-#define ETA_CASE(DD, GG) if (D == DD && G == GG) { launch_screen_t<DD, GG>(a, rows, s); return check_launch("screen"); }
+int launch_screen(const ScreenArgs& a, int rows, int D, int G, int n_ctas, cudaStream_t s) {
+#define ETA_CASE(DD, GG) if (D == DD && G == GG) return launch_screen_t<DD, GG>(a, rows, n_ctas, s);
     ETA_CASE(128, 1) ETA_CASE(128, 2) ETA_CASE(128, 4) ETA_CASE(128, 8)
     ETA_CASE(64, 1) ETA_CASE(64, 2) ETA_CASE(64, 4) ETA_CASE(64, 8)
 #undef ETA_CASE
