@@ -99,6 +99,42 @@ def algorithmic_bytes(sp, lens, union_blocks: float):
     return {"screen": float(screen), "decode": float(decode), "total": float(screen + decode + other)}
 
 
+def max_over_ranks(x: float, dist, dev) -> float:
+    """Device-timed numbers are reported as the maximum over ranks."""
+    if dist is None:
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, batch: int, ms_step: float) -> float:
+    """Replicas only: every rank decodes its own batch, so the job answers world * batch queries per step."""
+    return world * batch / (ms_step * 1e-3)
+
+
+def run_dry(args):
+    """Host-side logic of the multi-rank run without a GPU (gloo): rendezvous, barrier, max over ranks, one JSON
+    line from rank 0.  Each rank pretends to have measured 1.0 + 0.5 * rank ms per step."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    sp = wl.CONFIGS[args.workload]
+    ms = max_over_ranks(1.0 + 0.5 * rank, dist if world > 1 else None, torch.device("cpu"))
+    if world > 1:
+        dist.barrier()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": whole_job_value(world, sp.batch, ms), "unit": UNIT,
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": "weak", "dry_run": True,
+                          "config": {"workload": sp.name, "replicas": world}}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_ours(args):
     from paper_2609_20888_b200 import binding as eb
     from paper_2609_20888_b200 import build as ebuild
@@ -108,6 +144,7 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    dist = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
@@ -236,11 +273,7 @@ def run_ours(args):
     sampler.start()
     step_main = make_step(load_bias(sp.name, main_target))
     ms_main, wall_main = timed(step_main)
-    ms_step = sum(ms_main) / len(ms_main)
-    if world > 1:
-        tt = torch.tensor([ms_step], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_step = float(tt.item())
+    ms_step = max_over_ranks(sum(ms_main) / len(ms_main), dist if world > 1 else None, dev)
     union_main = union_blocks_of(step_main)
     kt = kernel_times(load_bias(sp.name, main_target))
     nb_total = sum(int(t) // sp.block_size for t in lens) * sp.n_kv_heads
@@ -263,11 +296,7 @@ def run_ours(args):
         b_ev.record()
         torch.cuda.synchronize()
         e2e_ms += a_ev.elapsed_time(b_ev)
-    e2e_s = e2e_ms * 1e-3 / args.steps
-    if world > 1:
-        tt = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_s = float(tt.item())
+    e2e_s = max_over_ranks(e2e_ms * 1e-3 / args.steps, dist if world > 1 else None, dev)
 
     clocks = sampler.stop()
 
@@ -300,7 +329,7 @@ def run_ours(args):
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": world * sp.batch / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": whole_job_value(world, sp.batch, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": sp.name, "batch": sp.batch, "n_q_heads": sp.n_q_heads, "n_kv_heads": sp.n_kv_heads,
@@ -398,10 +427,13 @@ def main():
     ap.add_argument("--no-pdl", dest="pdl", action="store_false", help="fully serialise the kernel launches")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--dry-run", action="store_true", help="exercise the multi-rank host logic on CPU (gloo)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.dry_run:
+        run_dry(args)
     else:
         run_ours(args)
 
