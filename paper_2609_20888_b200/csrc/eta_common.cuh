@@ -53,6 +53,26 @@ WsLayout ws_layout(const eta_cache_desc* d);
 
 struct RescueRec { int cnt; float maxb; int arg; int pad; };
 
+// Division by a run-time constant as multiply-high + shift (exact for 0 <= n < 2^31): integer division costs
+// dozens of instructions, and the single-warp set-up code of the kernels divides by the same few numbers.
+struct FastDiv {
+    uint32_t d, mul, shr;
+    FastDiv() : d(1), mul(0), shr(0) {}
+    explicit FastDiv(int divisor) : d((uint32_t)divisor), mul(0), shr(0) {
+        if (d > 1) {
+            uint32_t lg = 0;
+            while ((1ull << lg) < d) ++lg;
+            const uint32_t p = 31 + lg;
+            mul = (uint32_t)(((1ull << p) + d - 1) / d);
+            shr = p - 32;
+        }
+    }
+#ifdef __CUDACC__
+    __device__ __forceinline__ int div(int n) const { return d == 1 ? n : (int)(__umulhi((uint32_t)n, mul) >> shr); }
+    __device__ __forceinline__ void divmod(int n, int& q, int& r) const { q = div(n); r = n - q * (int)d; }
+#endif
+};
+
 // Arguments of the screening and planning kernels (defined in eta_screen.cu, launched from eta_decode).
 struct ScreenArgs {
     const __nv_bfloat16* q;

@@ -41,11 +41,13 @@ struct DecodeArgs {
     uint32_t* status;
     float beta, scale;
     int Hq, Hkv, G, b, t_cap, nb_cap, nseg, entries, rows, rescue_window;
+    FastDiv div_nseg, div_epr, div_hkv, div_g;
     unsigned long long* timeline;
 };
 
 constexpr uint32_t UF_END = 1u;
 constexpr int WARPS_PER_GROUP = 4;     // the four warps of a group each take a quarter of a tile's tokens
+constexpr int RESC_ROWS = 8;           // rows (from the CTA's first) whose rescue decisions stay in shared memory
 constexpr int PW = 256;                // entries of the unit prefix the producer keeps in shared memory
 
 __device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
@@ -127,7 +129,8 @@ struct DecodeSmem {
     static constexpr int WIN_OFF = DESC_OFF + 16 * NSTAGE;      // int32 pwin[PW + 1] (+3 pad): window of the unit prefix
     static constexpr int ROW_OFF = WIN_OFF + 4 * (PW + 4);      // int32 rowbase[MAX_ROWS + 1]: unit prefix over rows
     static constexpr int INFO_OFF = ROW_OFF + 4 * (MAX_ROWS + 4);   // uint8 per row: rescue units | tail flag << 7
-    static constexpr int ML_OFF = INFO_OFF + MAX_ROWS;          // float m[NGROUPS][4][8], l[NGROUPS][4][8]
+    static constexpr int RESC_OFF = INFO_OFF + MAX_ROWS;        // int32 [RESC_ROWS][8]: rescued block per head, first rows
+    static constexpr int ML_OFF = RESC_OFF + 4 * 8 * RESC_ROWS; // float m[NGROUPS][4][8], l[NGROUPS][4][8]
     static constexpr int MO_OFF = ML_OFF + 4 * 2 * NGROUPS * WARPS_PER_GROUP * 8;
     static size_t bytes(int G) { return 1024 + MO_OFF + sizeof(float) * NGROUPS * WARPS_PER_GROUP * G * D; }
 };
@@ -155,6 +158,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     int32_t* pwin = reinterpret_cast<int32_t*>(smem + L::WIN_OFF);
     int32_t* rowbase = reinterpret_cast<int32_t*>(smem + L::ROW_OFF);
     uint8_t* rowinfo = smem + L::INFO_OFF;
+    int32_t* resc_tab = reinterpret_cast<int32_t*>(smem + L::RESC_OFF);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long* tl = a.timeline ? a.timeline + (size_t)blockIdx.x * 8 : nullptr;
@@ -176,7 +180,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const bool counts_in_smem = (size_t)a.rows * a.nseg + 10 * 4 * MAX_ROWS <= (size_t)NSTAGE * L::STAGE_BYTES;
     // sequence lengths are a caller input: they can be read while the previous kernel is still running
     for (int rr = tid; rr < a.rows; rr += NTHREADS) {
-        const int T = __ldg(a.seq_lens + rr / a.Hkv);
+        const int T = __ldg(a.seq_lens + a.div_hkv.div(rr));
         s_len[rr] = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
         cnt32[rr] = 0;
     }
@@ -201,12 +205,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const int e = e0 + k * NTHREADS;
                 if (e < a.rows * a.nseg) {
                     if (counts_in_smem) cnt8[e] = (uint8_t)cv[k];
-                    if (cv[k]) atomicAdd(&cnt32[e / a.nseg], cv[k]);
+                    if (cv[k]) atomicAdd(&cnt32[a.div_nseg.div(e)], cv[k]);
                 }
             }
         }
         for (int p = tid; p < a.rows * a.G; p += NTHREADS) {
-            const int rr = p / a.G, g = p % a.G;
+            int rr, g;
+            a.div_g.divmod(p, rr, g);
             const int NB = min(s_len[rr] / a.b, a.nb_cap);
             resc_j[rr * 8 + g] = rescue_of(a.seg_resc, rr, g, a.G, a.nseg, min(a.rescue_window, NB));
         }
@@ -281,6 +286,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         row0 = lo;
     }
+    // the rescue decisions of the first rows of this CTA's range outlive the layout scratch
+    if (tid < 8 * RESC_ROWS) {
+        const int rr = row0 + tid / 8;
+        resc_tab[tid] = (rr < a.rows && (tid & 7) < a.G) ? resc_j[rr * 8 + (tid & 7)] : -1;
+    }
+    __syncthreads();
 
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
@@ -312,7 +323,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         bool first_window = counts_in_smem;     // the counts of the layout phase are still in the stage memory
         auto entry_count = [&](int e) {
             if (e >= E) return 0;
-            const int r = e / EPR, sg = e % EPR;
+            int r, sg;
+            a.div_epr.divmod(e, r, sg);
             if (sg < a.nseg) return first_window ? (int)cnt8[r * a.nseg + sg] : (int)__ldg(a.seg_count + r * a.nseg + sg);
             const int info = rowinfo[r];
             return sg == a.nseg ? (info & 0x7f) : (info >> 7);
@@ -368,16 +380,40 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const int uu = ub + lane;
                 const int k = search(uu);
                 const int e = e_base + k;
-                const int r = e / EPR, sg = e % EPR;
+                int r, sg;
+                a.div_epr.divmod(e, r, sg);
                 row = r;
                 if (sg >= a.nseg) {
-                    int T = __ldg(a.seq_lens + r / a.Hkv);
+                    int T = __ldg(a.seq_lens + a.div_hkv.div(r));
                     T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
                     const int NB = min(T / a.b, a.nb_cap);
                     if (sg == a.nseg) {
                         // a rescued block, attended by the rescued head(s) only
                         int uj[8], um[8];
-                        rescue_units(a.seg_resc, r, a.G, a.nseg, min(a.rescue_window, NB), uj, um);
+                        if (r - row0 < RESC_ROWS) {
+                            // same merge of equal blocks as rescue_units, from the table kept in shared memory
+                            int n = 0;
+#pragma unroll
+                            for (int g8 = 0; g8 < 8; ++g8) { uj[g8] = -1; um[g8] = 0; }
+#pragma unroll
+                            for (int g8 = 0; g8 < 8; ++g8) {
+                                const int j8 = resc_tab[(r - row0) * 8 + g8];
+                                if (j8 >= 0) {
+                                    bool merged = false;
+#pragma unroll
+                                    for (int q8 = 0; q8 < 8; ++q8)
+                                        if (q8 < n && uj[q8] == j8) { um[q8] |= 1 << g8; merged = true; }
+                                    if (!merged) {
+#pragma unroll
+                                        for (int q8 = 0; q8 < 8; ++q8)
+                                            if (q8 == n) { uj[q8] = j8; um[q8] = 1 << g8; }
+                                        ++n;
+                                    }
+                                }
+                            }
+                        } else {
+                            rescue_units(a.seg_resc, r, a.G, a.nseg, min(a.rescue_window, NB), uj, um);
+                        }
                         const int idx = uu - pwin[k];
                         int j = 0, m = 0;
 #pragma unroll
@@ -405,20 +441,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         fetch(u, nb, c_row, c_ent, c_nrows);
         if (tl && lane == 0) tl[7] = globaltimer_ns() + (c_ent & 0);
         while (u < u1 && ok) {
-            // the next batch's loads are in flight while this batch is issued
+            // the next batch is fetched once the first tiles of this batch are on their way, so that its loads
+            // are in flight while the rest of this batch is issued
             const int un = u + nb;
             int nbn = 0, n_row = -1, n_ent = 0, n_nrows = 0;
-            if (un < u1) {
-                nbn = batch_size(un);
-                fetch(un, nbn, n_row, n_ent, n_nrows);
-            }
+            const int k_prefetch = min(nb, NSTAGE) - 1;
             for (int k = 0; k < nb && ok; ++k) {
                 const int r = __shfl_sync(0xffffffffu, c_row, k);
                 const int ent = __shfl_sync(0xffffffffu, c_ent, k);
                 const int nrows = __shfl_sync(0xffffffffu, c_nrows, k);
                 const int j = ent & 0xffffff;
                 const int hmask = (ent >> 24) & 0xff;
-                const int i = r / a.Hkv, hk = r % a.Hkv;
+                int i, hk;
+                a.div_hkv.divmod(r, i, hk);
                 if (r != prev_row) {                               // a new (CTA, row) piece starts here
                     close_piece();
                     ++piece; prev_row = r; piece_f0 = fill;
@@ -445,6 +480,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     }
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                     ++fill;
+                }
+                if (k == k_prefetch && un < u1) {
+                    nbn = batch_size(un);
+                    fetch(un, nbn, n_row, n_ent, n_nrows);
                 }
             }
             u = un;
@@ -513,7 +552,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     // query fragments and threshold of a row: head g's slice in the permuted head_dim order of the MMA
     auto load_q = [&](int r) {
-        const int i = r / a.Hkv, hk = r % a.Hkv;
+        int i, hk;
+        a.div_hkv.divmod(r, i, hk);
         const __nv_bfloat16* qp = a.q + ((int64_t)i * a.Hq + hk * a.G + (head ? g : 0)) * D;
 #pragma unroll
         for (int hf = 0; hf < HALVES; ++hf)
@@ -972,6 +1012,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.Hq = desc->n_q_heads; da.Hkv = desc->n_kv_heads; da.G = G; da.b = b; da.t_cap = desc->t_cap;
     da.nseg = L.nseg; da.entries = L.entries; da.rows = L.rows; da.nb_cap = desc->nb_cap;
     da.rescue_window = params->rescue_window;
+    da.div_nseg = FastDiv(L.nseg); da.div_epr = FastDiv(L.nseg + 2); da.div_hkv = FastDiv(desc->n_kv_heads);
+    da.div_g = FastDiv(G);
     da.timeline = debug_timeline();
     if (D == 128 && TS == 64) {
         rc = (G == 8) ? launch_decode_t<128, 64, 5, DECODE_GROUPS>(tmK, tmV, da, n_ctas, s)

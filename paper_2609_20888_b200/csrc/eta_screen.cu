@@ -43,7 +43,7 @@ struct ScreenSmem {
 // them, so the records (and the group's queries) of the next item are in flight while the current one is
 // evaluated.
 template <int D, int G>
-__global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
+__global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     using L = ScreenSmem<D, G>;
     constexpr int LPR = D / 8;            // lanes sharing one record
     constexpr int RPW = 32 / LPR;         // records per warp instruction
@@ -84,9 +84,6 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
         s_len[rr] = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
     }
     __syncthreads();
-    // everything above touches only this CTA; the summaries and thresholds may still be in the making
-    pdl_wait();
-    if (tl && tid == 0) tl[1] = globaltimer_ns();
     if (it0 >= it1) return;
 
     // geometry of an item
@@ -113,31 +110,49 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
             mbar_arrive(&bars[buf]);      // nothing to copy: the phase completes at once
         }
     };
-    // per-thread prefetch of the small per-item scalars (largest-norm entry of record tid, threshold of head my_g)
-    auto prefetch_scalars = [&](int item, float& mnv, float& te) {
+    // The summaries and thresholds may still be in the making when this kernel starts (programmatic dependent
+    // launch): the append kernel writes the record and the norm of a block that has just filled up, the predictor
+    // writes tau.  Everything else this kernel reads is final, so only an item that holds a row's newest block of
+    // a just-completed length must wait before its copies; the thresholds are fetched after the wait, which
+    // the first item reaches only when its bounds are already computed.
+    auto safe_item = [&](int item) {
         int r, seg, i, hk, T, NB, j0, n_rec;
         item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
-        mnv = (tid < n_rec && !dense) ? __ldg(a.mnorm + (int64_t)r * a.nb_cap + j0 + tid) : 0.f;
+        return !(n_rec > 0 && (T % a.b) == 0 && j0 + n_rec == NB);
+    };
+    auto load_mn = [&](int item) {        // largest-norm entry of record `tid` of the item
+        int r, seg, i, hk, T, NB, j0, n_rec;
+        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
+        return (tid < n_rec && !dense) ? __ldg(a.mnorm + (int64_t)r * a.nb_cap + j0 + tid) : 0.f;
+    };
+    auto load_te = [&](int item) {        // effective threshold of head my_g of the item's group
+        int r, seg, i, hk, T, NB, j0, n_rec;
+        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
         const int h = hk * G + my_g;
-        te = dense ? -INFINITY : ((a.tau ? __ldg(a.tau + (int64_t)i * a.Hq + h) : __ldg(a.head_const + h)) - a.a);
+        return dense ? -INFINITY : ((a.tau ? __ldg(a.tau + (int64_t)i * a.Hq + h) : __ldg(a.head_const + h)) - a.a);
     };
 
+    bool waited = false;
+    if (!safe_item(it0)) { pdl_wait(); waited = true; }
     if (tid == 0) issue(it0, 0);
-    float mn_cur, te_cur;
-    prefetch_scalars(it0, mn_cur, te_cur);
+    float mn_cur = load_mn(it0);
+    float te_cur = waited ? load_te(it0) : 0.f;
+    if (tl && tid == 0) tl[1] = globaltimer_ns();
 
     for (int item = it0; item < it1; ++item) {
         const int k = item - it0, buf = k & 1;
         int r, seg, i, hk, T, NB, j0, n_rec;
         item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
         float mn_next = 0.f, te_next = 0.f;
-        if (item + 1 < it1) {
+        bool next_issued = false, next_te = false;
+        if (item + 1 < it1 && (waited || safe_item(item + 1))) {
             if (tid == 0) issue(item + 1, buf ^ 1);
-            prefetch_scalars(item + 1, mn_next, te_next);
+            mn_next = load_mn(item + 1);
+            next_issued = true;
         }
-        const float my_te = te_cur;
+        if (item + 1 < it1 && waited) { te_next = load_te(item + 1); next_te = true; }
+        float my_te = te_cur;
         if (tid < SEG) smn[tid] = mn_cur;
-        if (seg == 0 && tid < G) a.tau_eff[(int64_t)i * a.Hq + hk * G + tid] = my_te;     // lane g < G holds head g
         if (seg == 0 && tid == 0 && a.status) {
             const int Traw = __ldg(a.seq_lens + i);
             if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
@@ -238,6 +253,7 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
                     const float mnv = valid ? smn[rec] : 0.f;
                     const float bound = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * mnv);
                     const bool pinned = (j0 + rec) >= NB - a.lwb;
+                    if (!waited) { pdl_wait(); waited = true; my_te = load_te(item); }     // first item only
                     const bool admit = valid && (!(bound < my_te) || pinned || !ok);
                     if (valid) sbound[rec][my_g] = bound;
                     const unsigned bal = __ballot_sync(0xffffffffu, admit);
@@ -246,6 +262,7 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
             } else {
                 if (tid < n_rec) smask[tid] = (uint8_t)((1u << G) - 1u);
             }
+            if (!waited) { pdl_wait(); waited = true; my_te = load_te(item); }     // warps without a batch
             __syncthreads();
             if (tl && tid == 0 && item == it0) tl[3] = globaltimer_ns();
 
@@ -297,6 +314,13 @@ __global__ void __launch_bounds__(256) screen_kernel(const ScreenArgs a) {
                 }
             }
         }   // n_rec > 0
+        if (!waited) { pdl_wait(); waited = true; my_te = load_te(item); }
+        if (seg == 0 && tid < G) a.tau_eff[(int64_t)i * a.Hq + hk * G + tid] = my_te;     // lane g < G holds head g
+        if (item + 1 < it1 && !next_issued) {
+            if (tid == 0) issue(item + 1, buf ^ 1);
+            mn_next = load_mn(item + 1);
+        }
+        if (item + 1 < it1 && !next_te) te_next = load_te(item + 1);
 
         __syncthreads();       // the item's shared-memory state may be overwritten from here on
         if (tl && tid == 0 && item == it0) tl[4] = globaltimer_ns();
