@@ -35,6 +35,7 @@ struct DecodeArgs {
     uint8_t* sel_mask;
     int32_t* stats;
     int32_t* row_start;
+    int2* cta_range;
     int32_t* hdr;
     float2* part_ml;
     float* part_o;
@@ -274,6 +275,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         for (int rr = tid; rr <= a.rows; rr += 32 * (WARPS_PER_GROUP * NGROUPS + 1)) a.row_start[rr] = rowbase[rr];
         if (tid == 0) { a.hdr[0] = U; a.hdr[1] = P; }
     }
+    if (tid == 0) a.cta_range[blockIdx.x] = make_int2(u0, u1);      // read by the merge kernel
     if (tl && tid == 0) tl[1] = globaltimer_ns();
     if (u0 >= u1) return;
     // row holding unit u0: last r with rowbase[r] <= u0
@@ -774,6 +776,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 // Associative merge of the pieces of one (sequence, query head): Algorithm 3, global reduction.
 struct MergeArgs {
     const int32_t* row_start;
+    const int2* cta_range;
     const int32_t* hdr;
     const float2* part_ml;
     const float* part_o;
@@ -783,16 +786,20 @@ struct MergeArgs {
 
 constexpr int MERGE_WARPS = 8;
 
-// One CTA per (row, query head).  Every warp reads the (m, l) of all candidate parts (lanes in parallel) and
-// takes the largest m; warp w then weighs and adds the O of parts w, w + 8, ... (all of its loads in flight at
-// once), and the eight warp sums are added in a fixed order:
+// One CTA per (row, query head).  The candidate parts are the (streaming CTA, consumer group) pairs whose CTA's
+// unit range meets the row's range; the CTA ranges are read from memory (written by the streaming kernel).
+// Pass 1: all threads read the (m, l) of the candidates and the CTA takes the largest m.  Pass 2: warp w weighs
+// and adds the O of its contiguous share of the candidates, eight loads in flight, and the eight warp sums are
+// added in a fixed order:
 //   o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
 template <int D>
 __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs a) {
     constexpr int VPL = D / 32;
+    constexpr int NT = 32 * MERGE_WARPS;
     __shared__ float s_acc[MERGE_WARPS][D];
     __shared__ float s_l[MERGE_WARPS];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __shared__ float s_m[MERGE_WARPS];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
     pdl_trigger();
@@ -803,75 +810,91 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
 #pragma unroll
     for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
     float lw_sum = 0.f;
+    int c_lo = 0, n_cand = 0;
     if (rbd > ra && U > 0) {
-        // streaming CTAs whose unit range meets this row's range [ra, rbd): a superset, then tested exactly
-        int c_lo = (int)(((int64_t)ra * P) / U) - 1;
+        // streaming CTAs whose unit range can meet [ra, rbd): a superset, tested exactly against their ranges
+        c_lo = (int)(((int64_t)ra * P) / U) - 1;
         int c_hi = (int)(((int64_t)rbd * P + U - 1) / U) + 1;
         c_lo = c_lo < 0 ? 0 : c_lo;
         c_hi = c_hi > (int)P - 1 ? (int)P - 1 : c_hi;
-        const int n_cand = (c_hi - c_lo + 1) * a.ngroups;
-        float mg = -INFINITY;
-        for (int k0 = 0; k0 < n_cand; k0 += 32) {
+        n_cand = (c_hi - c_lo + 1) * a.ngroups;
+    }
+    // a candidate's slot if its CTA's range meets the row, else -1
+    auto slot_of = [&](int k) -> int64_t {
+        const int c = c_lo + k / a.ngroups;
+        const int2 rg = __ldg(a.cta_range + c);
+        if (max(rg.x, ra) >= min(rg.y, rbd)) return -1;
+        return ((int64_t)c + r) * a.ngroups + k % a.ngroups;
+    };
+    float mg = -INFINITY;
+    for (int k = tid; k < n_cand; k += NT) {
+        const int64_t slot = slot_of(k);
+        if (slot >= 0) mg = fmaxf(mg, a.part_ml[slot * a.G + gq].x);
+    }
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, s));
+    if (lane == 0) s_m[warp] = mg;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < MERGE_WARPS; ++w) mg = fmaxf(mg, s_m[w]);
+    if (mg != -INFINITY) {
+        // warp w takes candidates [w * per, (w + 1) * per): lane j of a round reads the statistics of one
+        // candidate, then the warp adds the candidates' O rows, eight at a time
+        const int per = (n_cand + MERGE_WARPS - 1) / MERGE_WARPS;
+        const int k_begin = warp * per, k_end = min(n_cand, k_begin + per);
+        for (int k0 = k_begin; k0 < k_end; k0 += 32) {
             const int k = k0 + lane;
-            if (k < n_cand) {
-                const int c = c_lo + k / a.ngroups;
-                const int cu0 = (int)(((int64_t)c * U) / P), cu1 = (int)(((int64_t)(c + 1) * U) / P);
-                if (max(cu0, ra) < min(cu1, rbd)) {
-                    const int64_t slot = ((int64_t)c + r) * a.ngroups + k % a.ngroups;
-                    mg = fmaxf(mg, a.part_ml[slot * a.G + gq].x);
+            float w = 0.f;
+            int64_t slot = -1;
+            if (k < k_end) {
+                slot = slot_of(k);
+                if (slot >= 0) {
+                    const float2 ml = a.part_ml[slot * a.G + gq];
+                    if (ml.x != -INFINITY) { w = __expf(ml.x - mg); lw_sum = fmaf(ml.y, w, lw_sum); }
                 }
             }
-        }
+            const int nk = min(32, k_end - k0);
+            for (int j0 = 0; j0 < nk; j0 += 8) {
+                float wv[8];
+                float xv[8][VPL];
 #pragma unroll
-        for (int s = 16; s >= 1; s >>= 1) mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, s));
-        if (mg != -INFINITY) {
-            // this warp's parts, four at a time
-            for (int k0 = warp; k0 < n_cand; k0 += 4 * MERGE_WARPS) {
-                float wv[4];
-                float xv[4][VPL];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int k = k0 + u * MERGE_WARPS;
-                    wv[u] = 0.f;
+                for (int u = 0; u < 8; ++u) {
+                    const int src = min(j0 + u, 31);
+                    const float wk = __shfl_sync(0xffffffffu, w, src);
+                    const int64_t sk = __shfl_sync(0xffffffffu, slot, src);
+                    wv[u] = (j0 + u < nk) ? wk : 0.f;
 #pragma unroll
                     for (int v = 0; v < VPL; ++v) xv[u][v] = 0.f;
-                    if (k < n_cand) {
-                        const int c = c_lo + k / a.ngroups;
-                        const int cu0 = (int)(((int64_t)c * U) / P), cu1 = (int)(((int64_t)(c + 1) * U) / P);
-                        if (max(cu0, ra) < min(cu1, rbd)) {
-                            const int64_t slot = ((int64_t)c + r) * a.ngroups + k % a.ngroups;
-                            const float2 ml = a.part_ml[slot * a.G + gq];
-                            if (ml.x != -INFINITY) {     // cleared by the plan step and never written: no such part
-                                wv[u] = __expf(ml.x - mg);
-                                lw_sum = fmaf(ml.y, wv[u], lw_sum);
-                                const float* po = a.part_o + (slot * a.G + gq) * D + lane * VPL;
-                                if (VPL == 4) {
-                                    const float4 x = __ldg(reinterpret_cast<const float4*>(po));
-                                    xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
-                                } else {
-                                    const float2 x = __ldg(reinterpret_cast<const float2*>(po));
-                                    xv[u][0] = x.x; xv[u][1] = x.y;
-                                }
-                            }
+                    if (wv[u] != 0.f) {
+                        const float* po = a.part_o + (sk * a.G + gq) * D + lane * VPL;
+                        if (VPL == 4) {
+                            const float4 x = __ldg(reinterpret_cast<const float4*>(po));
+                            xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
+                        } else {
+                            const float2 x = __ldg(reinterpret_cast<const float2*>(po));
+                            xv[u][0] = x.x; xv[u][1] = x.y;
                         }
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
+                for (int u = 0; u < 8; ++u)
 #pragma unroll
                     for (int v = 0; v < VPL; ++v) acc[v] = fmaf(xv[u][v], wv[u], acc[v]);
             }
         }
     }
+    // lanes hold different candidates' l * w: sum inside the warp, then across warps in a fixed order
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) lw_sum += __shfl_xor_sync(0xffffffffu, lw_sum, s);
 #pragma unroll
     for (int v = 0; v < VPL; ++v) s_acc[warp][lane * VPL + v] = acc[v];
-    if (lane == 0) s_l[warp] = lw_sum;      // every lane of a warp holds the same sum
+    if (lane == 0) s_l[warp] = lw_sum;
     __syncthreads();
-    if (threadIdx.x < D) {
+    if (tid < D) {
         float o = 0.f, l = 0.f;
 #pragma unroll
-        for (int w = 0; w < MERGE_WARPS; ++w) { o += s_acc[w][threadIdx.x]; l += s_l[w]; }
-        a.out[((int64_t)i * a.Hq + hk * a.G + gq) * D + threadIdx.x] = l > 0.f ? o / l : 0.f;
+        for (int w = 0; w < MERGE_WARPS; ++w) { o += s_acc[w][tid]; l += s_l[w]; }
+        a.out[((int64_t)i * a.Hq + hk * a.G + gq) * D + tid] = l > 0.f ? o / l : 0.f;
     }
 }
 
@@ -1005,6 +1028,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.seg_count = sa.seg_count; da.seg_resc = sa.seg_resc; da.sel_mask = sel_mask; da.stats = stats;
     da.row_start = reinterpret_cast<int32_t*>(ws + L.row_start);
     da.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
+    da.cta_range = reinterpret_cast<int2*>(ws + L.cta_range);
     da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
     da.part_o = reinterpret_cast<float*>(ws + L.part_o);
     da.status = status_dev;
@@ -1029,7 +1053,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     profile_mark(4, s);
 
     MergeArgs ma;
-    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
+    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.cta_range = da.cta_range; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
     ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS;
     const unsigned mgrid = (unsigned)(L.rows * G);
     cudaError_t me = (D == 128) ? launch_pdl(merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
