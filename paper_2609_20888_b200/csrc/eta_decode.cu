@@ -48,6 +48,7 @@ struct DecodeArgs {
 
 constexpr uint32_t UF_END = 1u;
 constexpr int WARPS_PER_GROUP = 4;     // the four warps of a group each take a quarter of a tile's tokens
+constexpr int PIECE_COST = 3;          // tiles a row boundary inside a CTA's range is worth (flush + query reload)
 constexpr int RESC_ROWS = 8;           // rows (from the CTA's first) whose rescue decisions stay in shared memory
 constexpr int PW = 256;                // entries of the unit prefix the producer keeps in shared memory
 
@@ -190,6 +191,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     // ---- every CTA lays out the flattened unit sequence for itself: per row the surviving blocks of its
     // segments, then its rescued blocks, then its tail; a scan over the rows gives each row's first unit
+    int nz_rows = 0;      // rows that have at least one unit
     {
         __shared__ int s_wsum[32];
         // all loads of the layout are independent and issued together: segment counts (summed per row with
@@ -241,35 +243,61 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             if (blockIdx.x == 0 && a.stats) a.stats[rr] = c + extra;
         }
         __syncthreads();
-        const int nthreads = NTHREADS;
-        int carry = 0;
-        for (int r0 = 0; r0 < a.rows; r0 += nthreads) {
-            const int rr = r0 + tid;
-            const int c = (rr < a.rows) ? rowbase[rr] : 0;
-            int incl = c;
+        // exclusive block scan over the rows: value of row rr from get(rr), prefix handed to put(rr, prefix)
+        auto scan_rows = [&](auto get, auto put) {
+            int carry = 0;
+            for (int r0 = 0; r0 < a.rows; r0 += NTHREADS) {
+                const int rr = r0 + tid;
+                const int c = (rr < a.rows) ? get(rr) : 0;
+                int incl = c;
 #pragma unroll
-            for (int s = 1; s < 32; s <<= 1) {
-                const int o = __shfl_up_sync(0xffffffffu, incl, s);
-                if (lane >= s) incl += o;
+                for (int s = 1; s < 32; s <<= 1) {
+                    const int o = __shfl_up_sync(0xffffffffu, incl, s);
+                    if (lane >= s) incl += o;
+                }
+                if (lane == 31) s_wsum[warp] = incl;
+                __syncthreads();
+                int wbase = 0, tot = 0;
+                for (int w = 0; w < NWARPS; ++w) {
+                    const int v = s_wsum[w];
+                    if (w < warp) wbase += v;
+                    tot += v;
+                }
+                if (rr < a.rows) put(rr, carry + wbase + incl - c);
+                carry += tot;
+                __syncthreads();
             }
-            if (lane == 31) s_wsum[warp] = incl;
-            __syncthreads();
-            int wbase = 0, tot = 0;
-            for (int w = 0; w < NWARPS; ++w) {
-                const int v = s_wsum[w];
-                if (w < warp) wbase += v;
-                tot += v;
-            }
-            if (rr < a.rows) rowbase[rr] = carry + wbase + incl - c;
-            carry += tot;
-            __syncthreads();
-        }
-        if (tid == 0) rowbase[a.rows] = carry;
+            return carry;
+        };
+        // cnt32 (scratch) <- rows with at least one unit before row rr; rowbase <- units before row rr
+        const int nz_total = scan_rows([&](int rr) { return rowbase[rr] > 0 ? 1 : 0; },
+                                       [&](int rr, int p) { cnt32[rr] = p; });
+        const int u_total = scan_rows([&](int rr) { return rowbase[rr]; }, [&](int rr, int p) { rowbase[rr] = p; });
+        if (tid == 0) { rowbase[a.rows] = u_total; s_wsum[0] = nz_total; }
         __syncthreads();
+        nz_rows = s_wsum[0];
     }
     const int U = rowbase[a.rows];
     const int P = gridDim.x;
-    const int u0 = (int)(((int64_t)blockIdx.x * U) / P), u1 = (int)(((int64_t)(blockIdx.x + 1) * U) / P);
+    // Equal shares of COST, not of units: a row that starts inside a CTA's range costs that CTA a flush of its
+    // partials and a query reload, worth about PIECE_COST tiles.  Row rr spans the cost interval
+    // [rowbase[rr] + PIECE_COST * cnt32[rr], +PIECE_COST (if it has units) + its units).
+    auto cost_to_unit = [&](int64_t x) {
+        int lo = 0, hi = a.rows;         // last rr in [0, rows] with cost_start(rr) <= x
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            const int nzb = (mid < a.rows) ? cnt32[mid] : nz_rows;
+            if ((int64_t)rowbase[mid] + (int64_t)PIECE_COST * nzb <= x) lo = mid; else hi = mid - 1;
+        }
+        if (lo >= a.rows) return U;
+        const int units = rowbase[lo + 1] - rowbase[lo];
+        int64_t off = x - ((int64_t)rowbase[lo] + (int64_t)PIECE_COST * cnt32[lo]) - (units > 0 ? PIECE_COST : 0);
+        off = off < 0 ? 0 : (off > units ? units : off);
+        return rowbase[lo] + (int)off;
+    };
+    const int64_t C = (int64_t)U + (int64_t)PIECE_COST * nz_rows;
+    const int u0 = cost_to_unit((blockIdx.x * C) / P);
+    const int u1 = (blockIdx.x + 1 == P) ? U : cost_to_unit(((blockIdx.x + 1) * C) / P);
     if (blockIdx.x == 0) {
         // the merge kernel reads the row ranges and the split from memory
         for (int rr = tid; rr <= a.rows; rr += 32 * (WARPS_PER_GROUP * NGROUPS + 1)) a.row_start[rr] = rowbase[rr];
@@ -805,20 +833,24 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     pdl_trigger();
     pdl_wait();          // every partial of the streaming kernel is in memory from here on
     const int ra = a.row_start[r], rbd = a.row_start[r + 1];
-    const int64_t U = a.hdr[0], P = a.hdr[1];
+    const int64_t P = a.hdr[1];
     float acc[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
     float lw_sum = 0.f;
-    int c_lo = 0, n_cand = 0;
-    if (rbd > ra && U > 0) {
-        // streaming CTAs whose unit range can meet [ra, rbd): a superset, tested exactly against their ranges
-        c_lo = (int)(((int64_t)ra * P) / U) - 1;
-        int c_hi = (int)(((int64_t)rbd * P + U - 1) / U) + 1;
-        c_lo = c_lo < 0 ? 0 : c_lo;
-        c_hi = c_hi > (int)P - 1 ? (int)P - 1 : c_hi;
-        n_cand = (c_hi - c_lo + 1) * a.ngroups;
+    // streaming CTAs whose unit range meets the row's range [ra, rbd): a contiguous run of CTA indices
+    __shared__ int s_clo, s_chi;
+    if (tid == 0) { s_clo = 0x7fffffff; s_chi = -1; }
+    __syncthreads();
+    if (rbd > ra) {
+        for (int c = tid; c < (int)P; c += NT) {
+            const int2 rg = __ldg(a.cta_range + c);
+            if (max(rg.x, ra) < min(rg.y, rbd)) { atomicMin(&s_clo, c); atomicMax(&s_chi, c); }
+        }
     }
+    __syncthreads();
+    const int c_lo = s_clo;
+    const int n_cand = (s_chi >= c_lo) ? (s_chi - c_lo + 1) * a.ngroups : 0;
     // a candidate's slot if its CTA's range meets the row, else -1
     auto slot_of = [&](int k) -> int64_t {
         const int c = c_lo + k / a.ngroups;
