@@ -74,6 +74,8 @@ struct FastDiv {
 #endif
 };
 
+
+
 // Arguments of the screening and planning kernels (defined in eta_screen.cu, launched from eta_decode).
 struct ScreenArgs {
     const __nv_bfloat16* q;
@@ -85,7 +87,8 @@ struct ScreenArgs {
     float z, a, scale;
     int lwb, rescue_window;
     uint32_t flags;
-    int Hq, Hkv, b, t_cap, nb_cap, nseg, rows;
+    int Hq, Hkv, b, b_shift, t_cap, nb_cap, nseg, rows;
+    FastDiv div_nseg, div_hkv;
     int32_t* seg_count;
     int32_t* seg_list;
     RescueRec* seg_resc;

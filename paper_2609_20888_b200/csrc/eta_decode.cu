@@ -1037,6 +1037,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     sa.lwb = params->lwb; sa.rescue_window = params->rescue_window; sa.flags = params->flags;
     sa.Hq = desc->n_q_heads; sa.Hkv = desc->n_kv_heads; sa.b = b; sa.t_cap = desc->t_cap; sa.nb_cap = desc->nb_cap;
     sa.nseg = L.nseg; sa.rows = L.rows;
+    sa.b_shift = (b == 32) ? 5 : (b == 64 ? 6 : 7);
+    sa.div_nseg = FastDiv(L.nseg); sa.div_hkv = FastDiv(desc->n_kv_heads);
     sa.seg_count = reinterpret_cast<int32_t*>(ws + L.seg_count);
     sa.seg_list = reinterpret_cast<int32_t*>(ws + L.seg_list);
     sa.seg_resc = reinterpret_cast<RescueRec*>(ws + L.seg_resc);

@@ -86,26 +86,27 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     __syncthreads();
     if (it0 >= it1) return;
 
-    // geometry of an item
-    auto item_geom = [&](int item, int& r, int& seg, int& i, int& hk, int& T, int& NB, int& j0, int& n_rec) {
-        r = item / a.nseg; seg = item % a.nseg;
-        i = r / a.Hkv; hk = r % a.Hkv;
-        T = s_len[r];
-        NB = min(T / a.b, a.nb_cap);
-        j0 = seg * SEG;
-        n_rec = max(0, min(SEG, NB - j0));
+    // geometry of an item, computed once per item (multiply-high divisions; b is a power of two)
+    struct Geom { int r, seg, i, hk, T, NB, j0, n_rec; };
+    auto item_geom = [&](int item) {
+        Geom g;
+        a.div_nseg.divmod(item, g.r, g.seg);
+        a.div_hkv.divmod(g.r, g.i, g.hk);
+        g.T = s_len[g.r];
+        g.NB = min(g.T >> a.b_shift, a.nb_cap);
+        g.j0 = g.seg * SEG;
+        g.n_rec = max(0, min(SEG, g.NB - g.j0));
+        return g;
     };
     // one thread starts the copies of an item into buffer `buf`
-    auto issue = [&](int item, int buf) {
-        int r, seg, i, hk, T, NB, j0, n_rec;
-        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
-        if (n_rec > 0 && !dense) {
+    auto issue = [&](const Geom& g, int buf) {
+        if (g.n_rec > 0 && !dense) {
             unsigned char* dst = sm + buf * L::BUF_BYTES;
             const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
-                                       ((int64_t)r * a.nb_cap + j0) * REC_BYTES;
-            mbar_arrive_expect_tx(&bars[buf], n_rec * REC_BYTES + G * D * 2);
-            tma_load_1d(dst, src, n_rec * REC_BYTES, &bars[buf]);
-            tma_load_1d(dst + SEG * REC_BYTES, a.q + ((int64_t)i * a.Hq + hk * G) * D, G * D * 2, &bars[buf]);
+                                       ((int64_t)g.r * a.nb_cap + g.j0) * REC_BYTES;
+            mbar_arrive_expect_tx(&bars[buf], g.n_rec * REC_BYTES + G * D * 2);
+            tma_load_1d(dst, src, g.n_rec * REC_BYTES, &bars[buf]);
+            tma_load_1d(dst + SEG * REC_BYTES, a.q + ((int64_t)g.i * a.Hq + g.hk * G) * D, G * D * 2, &bars[buf]);
         } else {
             mbar_arrive(&bars[buf]);      // nothing to copy: the phase completes at once
         }
@@ -115,42 +116,42 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     // writes tau.  Everything else this kernel reads is final, so only an item that holds a row's newest block of
     // a just-completed length must wait before its copies; the thresholds are fetched after the wait, which
     // the first item reaches only when its bounds are already computed.
-    auto safe_item = [&](int item) {
-        int r, seg, i, hk, T, NB, j0, n_rec;
-        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
-        return !(n_rec > 0 && (T % a.b) == 0 && j0 + n_rec == NB);
+    auto safe_item = [&](const Geom& g) {
+        return !(g.n_rec > 0 && (g.T & (a.b - 1)) == 0 && g.j0 + g.n_rec == g.NB);
     };
-    auto load_mn = [&](int item) {        // largest-norm entry of record `tid` of the item
-        int r, seg, i, hk, T, NB, j0, n_rec;
-        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
-        return (tid < n_rec && !dense) ? __ldg(a.mnorm + (int64_t)r * a.nb_cap + j0 + tid) : 0.f;
+    auto load_mn = [&](const Geom& g) {        // largest-norm entry of record `tid` of the item
+        return (tid < g.n_rec && !dense) ? __ldg(a.mnorm + (int64_t)g.r * a.nb_cap + g.j0 + tid) : 0.f;
     };
-    auto load_te = [&](int item) {        // effective threshold of head my_g of the item's group
-        int r, seg, i, hk, T, NB, j0, n_rec;
-        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
-        const int h = hk * G + my_g;
-        return dense ? -INFINITY : ((a.tau ? __ldg(a.tau + (int64_t)i * a.Hq + h) : __ldg(a.head_const + h)) - a.a);
+    auto load_te = [&](const Geom& g) {        // effective threshold of head my_g of the item's group
+        const int h = g.hk * G + my_g;
+        return dense ? -INFINITY : ((a.tau ? __ldg(a.tau + (int64_t)g.i * a.Hq + h) : __ldg(a.head_const + h)) - a.a);
     };
 
+    float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G], my_qn = 0.f;
+    int q_row = -1;
     bool waited = false;
-    if (!safe_item(it0)) { pdl_wait(); waited = true; }
-    if (tid == 0) issue(it0, 0);
-    float mn_cur = load_mn(it0);
-    float te_cur = waited ? load_te(it0) : 0.f;
-    if (tl && tid == 0) tl[1] = globaltimer_ns();
+    Geom gc = item_geom(it0);
+    if (!safe_item(gc)) { pdl_wait(); waited = true; }
+    if (tid == 0) issue(gc, 0);
+    float mn_cur = load_mn(gc);
+    float te_cur = waited ? load_te(gc) : 0.f;
 
     for (int item = it0; item < it1; ++item) {
         const int k = item - it0, buf = k & 1;
-        int r, seg, i, hk, T, NB, j0, n_rec;
-        item_geom(item, r, seg, i, hk, T, NB, j0, n_rec);
+        const int r = gc.r, seg = gc.seg, i = gc.i, hk = gc.hk, T = gc.T, NB = gc.NB, j0 = gc.j0, n_rec = gc.n_rec;
+        (void)T;
+        Geom gn = gc;
         float mn_next = 0.f, te_next = 0.f;
         bool next_issued = false, next_te = false;
-        if (item + 1 < it1 && (waited || safe_item(item + 1))) {
-            if (tid == 0) issue(item + 1, buf ^ 1);
-            mn_next = load_mn(item + 1);
-            next_issued = true;
+        if (item + 1 < it1) {
+            gn = item_geom(item + 1);
+            if (waited || safe_item(gn)) {
+                if (tid == 0) issue(gn, buf ^ 1);
+                mn_next = load_mn(gn);
+                next_issued = true;
+            }
+            if (waited) { te_next = load_te(gn); next_te = true; }
         }
-        if (item + 1 < it1 && waited) { te_next = load_te(item + 1); next_te = true; }
         float my_te = te_cur;
         if (tid < SEG) smn[tid] = mn_cur;
         if (seg == 0 && tid == 0 && a.status) {
@@ -162,16 +163,19 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         if (tid < SEG && tid >= n_rec && j0 + tid < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = 0;
         if (n_rec == 0 && tid == 0) a.seg_count[r * a.nseg + seg] = 0;
 
+        if (tl && tid == 0 && item == it0 + 1) tl[6] = globaltimer_ns();
         bool ok = mbar_wait(&bars[buf], (k >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         __syncthreads();       // smn visible
         if (tl && tid == 0 && item == it0) tl[2] = globaltimer_ns();
+        if (tl && tid == 0 && item == it0 + 1) tl[7] = globaltimer_ns();
 
         if (n_rec > 0) {
             const uint32_t rec_base = smem_u32(sm + buf * L::BUF_BYTES);
             if (!dense) {
-                // this lane's slice of the G query vectors, in fp32
-                float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G];
+                // this lane's slice of the G query vectors, in fp32: kept across the items of one row
+                if (r != q_row) {
+                q_row = r;
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     const uint4 v = lds128(rec_base + SEG * REC_BYTES + (g * D + cc * 8) * 2);
@@ -191,9 +195,10 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                     for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
                     qn[g] = sqrtf(n2);
                 }
-                float my_qn = qn[0];
+                my_qn = qn[0];
 #pragma unroll
                 for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
+                }
 
                 for (int base = warp * RB; base < n_rec; base += 8 * RB) {
                     // a wait that ran out: admit everything (errs toward loading) - never seen in practice
@@ -253,7 +258,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                     const float mnv = valid ? smn[rec] : 0.f;
                     const float bound = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * mnv);
                     const bool pinned = (j0 + rec) >= NB - a.lwb;
-                    if (!waited) { pdl_wait(); waited = true; my_te = load_te(item); }     // first item only
+                    if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }     // first item only
                     const bool admit = valid && (!(bound < my_te) || pinned || !ok);
                     if (valid) sbound[rec][my_g] = bound;
                     const unsigned bal = __ballot_sync(0xffffffffu, admit);
@@ -262,9 +267,10 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
             } else {
                 if (tid < n_rec) smask[tid] = (uint8_t)((1u << G) - 1u);
             }
-            if (!waited) { pdl_wait(); waited = true; my_te = load_te(item); }     // warps without a batch
+            if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }     // warps without a batch
             __syncthreads();
             if (tl && tid == 0 && item == it0) tl[3] = globaltimer_ns();
+            if (tl && tid == 0 && item == it0 + 1) tl[1] = globaltimer_ns();
 
             // user-visible admission bits
             if (tid < n_rec) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = smask[tid];
@@ -314,18 +320,19 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                 }
             }
         }   // n_rec > 0
-        if (!waited) { pdl_wait(); waited = true; my_te = load_te(item); }
+        if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }
         if (seg == 0 && tid < G) a.tau_eff[(int64_t)i * a.Hq + hk * G + tid] = my_te;     // lane g < G holds head g
         if (item + 1 < it1 && !next_issued) {
-            if (tid == 0) issue(item + 1, buf ^ 1);
-            mn_next = load_mn(item + 1);
+            if (tid == 0) issue(gn, buf ^ 1);
+            mn_next = load_mn(gn);
         }
-        if (item + 1 < it1 && !next_te) te_next = load_te(item + 1);
+        if (item + 1 < it1 && !next_te) te_next = load_te(gn);
 
         __syncthreads();       // the item's shared-memory state may be overwritten from here on
         if (tl && tid == 0 && item == it0) tl[4] = globaltimer_ns();
         mn_cur = mn_next;
         te_cur = te_next;
+        gc = gn;
     }
     if (tl && tid == 0) tl[5] = globaltimer_ns();
     pdl_trigger();
