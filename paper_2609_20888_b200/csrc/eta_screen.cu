@@ -167,7 +167,6 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         bool ok = mbar_wait(&bars[buf], (k >> 1) & 1);
         ok = __all_sync(0xffffffffu, ok);
         __syncthreads();       // smn visible
-        if (tl && tid == 0 && item == it0) tl[2] = globaltimer_ns();
         if (tl && tid == 0 && item == it0 + 1) tl[7] = globaltimer_ns();
 
         if (n_rec > 0) {
@@ -269,7 +268,6 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
             }
             if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }     // warps without a batch
             __syncthreads();
-            if (tl && tid == 0 && item == it0) tl[3] = globaltimer_ns();
             if (tl && tid == 0 && item == it0 + 1) tl[1] = globaltimer_ns();
 
             // user-visible admission bits
@@ -329,7 +327,6 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         if (item + 1 < it1 && !next_te) te_next = load_te(gn);
 
         __syncthreads();       // the item's shared-memory state may be overwritten from here on
-        if (tl && tid == 0 && item == it0) tl[4] = globaltimer_ns();
         mn_cur = mn_next;
         te_cur = te_next;
         gc = gn;
@@ -383,8 +380,10 @@ static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream
         if (e != cudaSuccess) { set_cuda_error(e, "screen smem attribute"); return ETA_ERR_CUDA; }
         configured = true;
     }
+    // every CTA gets the same number of items (the last ones one fewer): the slowest CTA sets the kernel's end
     const int n_items = rows * a.nseg;
-    const int grid = n_items < n_ctas ? n_items : n_ctas;
+    const int per_cta = (n_items + n_ctas - 1) / n_ctas;
+    const int grid = (n_items + per_cta - 1) / per_cta;
     cudaError_t e = launch_pdl(screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, a);
     if (e != cudaSuccess) { set_cuda_error(e, "screen launch"); return ETA_ERR_CUDA; }
     return check_launch("screen");
