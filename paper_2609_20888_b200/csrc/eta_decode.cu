@@ -501,11 +501,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                             unsigned char* st = smem + stage * L::STAGE_BYTES;
                             mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
                             const int y = j * a.b + sub * TS;
-#pragma unroll
-                            for (int hf = 0; hf < HALVES; ++hf) {
-                                tma_load_4d(st + hf * L::TILE_BYTES, &tmK, hf * 64, y, hk, i, &full[stage]);
-                                tma_load_4d(st + (HALVES + hf) * L::TILE_BYTES, &tmV, hf * 64, y, hk, i, &full[stage]);
-                            }
+                            // one copy per tile: 64 columns x TS tokens x HALVES half tiles, each half swizzled
+                            tma_load_5d(st, &tmK, 0, y, 0, hk, i, &full[stage]);
+                            tma_load_5d(st + HALVES * L::TILE_BYTES, &tmV, 0, y, 0, hk, i, &full[stage]);
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -951,16 +949,18 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// K or V as a 4-D tensor (c, t, hk, i) of bf16; a box is 64 columns x TS tokens, 128-byte swizzled.
+// K or V as a 5-D tensor (c within a 64-column half, t, half, hk, i) of bf16; a box is 64 columns x TS tokens x
+// all halves: in shared memory, one 128-byte-swizzled [TS][64] tile per half, back to back.
 static int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d, int64_t sb, int64_t sh, int64_t st,
                      int TS) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return ETA_ERR_CUDA;
-    cuuint64_t dims[4] = {(cuuint64_t)d->head_dim, (cuuint64_t)d->t_cap, (cuuint64_t)d->n_kv_heads, (cuuint64_t)d->batch};
-    cuuint64_t strides[3] = {(cuuint64_t)st * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)TS, 1, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+    const cuuint32_t halves = (cuuint32_t)(d->head_dim / 64);
+    cuuint64_t dims[5] = {64, (cuuint64_t)d->t_cap, halves, (cuuint64_t)d->n_kv_heads, (cuuint64_t)d->batch};
+    cuuint64_t strides[4] = {(cuuint64_t)st * 2, 128, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+    cuuint32_t box[5] = {64, (cuuint32_t)TS, halves, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (rc != CUDA_SUCCESS) {
