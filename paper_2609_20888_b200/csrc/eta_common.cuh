@@ -45,6 +45,7 @@ struct WsLayout {
     size_t seg_resc;    // {int cnt; float maxb; int arg; int pad} [rows * nseg * G]
     size_t row_start;   // int32 [rows + 1]: global unit prefix over rows (written by the streaming kernel)
     size_t cta_range;   // int2 [MAX_CTAS]: unit range of every streaming CTA (written by the streaming kernel)
+    size_t row_cand;    // int2 [rows]: first and last streaming CTA whose range meets the row
     size_t tau_eff;     // float [batch * n_q_heads]
     size_t part_ml;     // float2 [(MAX_CTAS + rows) * DECODE_GROUPS * G]
     size_t part_o;      // float [(MAX_CTAS + rows) * DECODE_GROUPS * G * d]

@@ -36,6 +36,7 @@ struct DecodeArgs {
     int32_t* stats;
     int32_t* row_start;
     int2* cta_range;
+    int2* row_cand;
     int32_t* hdr;
     float2* part_ml;
     float* part_o;
@@ -303,7 +304,27 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         for (int rr = tid; rr <= a.rows; rr += 32 * (WARPS_PER_GROUP * NGROUPS + 1)) a.row_start[rr] = rowbase[rr];
         if (tid == 0) { a.hdr[0] = U; a.hdr[1] = P; }
     }
-    if (tid == 0) a.cta_range[blockIdx.x] = make_int2(u0, u1);      // read by the merge kernel
+    if (tid == 0) {
+        a.cta_range[blockIdx.x] = make_int2(u0, u1);      // read by the merge kernel
+        // the streaming CTAs whose ranges meet row rr, for the rows this CTA looks after: first CTA that ends
+        // after the row's first unit, last CTA that starts before the row's end
+        for (int rr = blockIdx.x; rr < a.rows; rr += P) {
+            const int ra = rowbase[rr], rb = rowbase[rr + 1];
+            int lo = 0, hi = P - 1;
+            while (lo < hi) {             // first c with u1(c) > ra
+                const int mid = (lo + hi) >> 1;
+                const int e1 = (mid + 1 == P) ? U : cost_to_unit(((mid + 1) * C) / P);
+                if (e1 > ra) hi = mid; else lo = mid + 1;
+            }
+            const int c_lo = lo;
+            lo = 0; hi = P - 1;
+            while (lo < hi) {             // last c with u0(c) < rb
+                const int mid = (lo + hi + 1) >> 1;
+                if (cost_to_unit((mid * C) / P) < rb) lo = mid; else hi = mid - 1;
+            }
+            a.row_cand[rr] = make_int2(c_lo, rb > ra ? lo : c_lo - 1);
+        }
+    }
     if (tl && tid == 0) tl[1] = globaltimer_ns();
     if (u0 >= u1) return;
     // row holding unit u0: last r with rowbase[r] <= u0
@@ -803,6 +824,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 struct MergeArgs {
     const int32_t* row_start;
     const int2* cta_range;
+    const int2* row_cand;
     const int32_t* hdr;
     const float2* part_ml;
     const float* part_o;
@@ -812,16 +834,15 @@ struct MergeArgs {
 
 constexpr int MERGE_WARPS = 8;
 
-// One CTA per (row, query head).  The candidate parts are the (streaming CTA, consumer group) pairs whose CTA's
-// unit range meets the row's range; the CTA ranges are read from memory (written by the streaming kernel).
-// Pass 1: all threads read the (m, l) of the candidates and the CTA takes the largest m.  Pass 2: warp w weighs
-// and adds the O of its contiguous share of the candidates, eight loads in flight, and the eight warp sums are
-// added in a fixed order:
+// One CTA per (row, query head).  The candidate parts are the (streaming CTA, consumer group) pairs of the
+// CTAs the streaming kernel listed for the row; a CTA whose range turns out not to meet the row, and a part
+// marked absent, weigh nothing.  Warp w takes a contiguous share of the candidates: a lane reads the statistics
+// of one candidate, the warp takes the largest m of its share, then weighs and adds the candidates' O rows, eight
+// loads in flight; the eight warps' (m, l, O) are combined in a fixed order:
 //   o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
 template <int D>
 __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs a) {
     constexpr int VPL = D / 32;
-    constexpr int NT = 32 * MERGE_WARPS;
     __shared__ float s_acc[MERGE_WARPS][D];
     __shared__ float s_l[MERGE_WARPS];
     __shared__ float s_m[MERGE_WARPS];
@@ -831,99 +852,86 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     pdl_trigger();
     pdl_wait();          // every partial of the streaming kernel is in memory from here on
     const int ra = a.row_start[r], rbd = a.row_start[r + 1];
-    const int64_t P = a.hdr[1];
+    const int2 cand = a.row_cand[r];
+    const int c_lo = cand.x;
+    const int n_cand = (rbd > ra && cand.y >= cand.x) ? (cand.y - cand.x + 1) * a.ngroups : 0;
     float acc[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
-    float lw_sum = 0.f;
-    // streaming CTAs whose unit range meets the row's range [ra, rbd): a contiguous run of CTA indices
-    __shared__ int s_clo, s_chi;
-    if (tid == 0) { s_clo = 0x7fffffff; s_chi = -1; }
-    __syncthreads();
-    if (rbd > ra) {
-        for (int c = tid; c < (int)P; c += NT) {
-            const int2 rg = __ldg(a.cta_range + c);
-            if (max(rg.x, ra) < min(rg.y, rbd)) { atomicMin(&s_clo, c); atomicMax(&s_chi, c); }
+    float m_w = -INFINITY, l_w = 0.f;        // this warp's running maximum and weighted l
+    const int per = (n_cand + MERGE_WARPS - 1) / MERGE_WARPS;
+    const int k_begin = warp * per, k_end = min(n_cand, k_begin + per);
+    for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+        const int k = k0 + lane;
+        float m_k = -INFINITY, l_k = 0.f;
+        int64_t slot = 0;
+        if (k < k_end) {
+            const int c = c_lo + k / a.ngroups;
+            slot = ((int64_t)c + r) * a.ngroups + k % a.ngroups;
+            const int2 rg = __ldg(a.cta_range + c);                // both loads are issued before either is used
+            const float2 ml = a.part_ml[slot * a.G + gq];
+            if (max(rg.x, ra) < min(rg.y, rbd)) { m_k = ml.x; l_k = ml.y; }
         }
-    }
-    __syncthreads();
-    const int c_lo = s_clo;
-    const int n_cand = (s_chi >= c_lo) ? (s_chi - c_lo + 1) * a.ngroups : 0;
-    // a candidate's slot if its CTA's range meets the row, else -1
-    auto slot_of = [&](int k) -> int64_t {
-        const int c = c_lo + k / a.ngroups;
-        const int2 rg = __ldg(a.cta_range + c);
-        if (max(rg.x, ra) >= min(rg.y, rbd)) return -1;
-        return ((int64_t)c + r) * a.ngroups + k % a.ngroups;
-    };
-    float mg = -INFINITY;
-    for (int k = tid; k < n_cand; k += NT) {
-        const int64_t slot = slot_of(k);
-        if (slot >= 0) mg = fmaxf(mg, a.part_ml[slot * a.G + gq].x);
-    }
+        float m_round = m_k;
 #pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, s));
-    if (lane == 0) s_m[warp] = mg;
-    __syncthreads();
+        for (int s = 16; s >= 1; s >>= 1) m_round = fmaxf(m_round, __shfl_xor_sync(0xffffffffu, m_round, s));
+        const float m_new = fmaxf(m_w, m_round);
+        if (m_new == -INFINITY) continue;        // nothing real in this round (warp-uniform)
+        const float rescale = (m_w == -INFINITY) ? 0.f : __expf(m_w - m_new);
+        const float w = (m_k == -INFINITY) ? 0.f : __expf(m_k - m_new);
 #pragma unroll
-    for (int w = 0; w < MERGE_WARPS; ++w) mg = fmaxf(mg, s_m[w]);
-    if (mg != -INFINITY) {
-        // warp w takes candidates [w * per, (w + 1) * per): lane j of a round reads the statistics of one
-        // candidate, then the warp adds the candidates' O rows, eight at a time
-        const int per = (n_cand + MERGE_WARPS - 1) / MERGE_WARPS;
-        const int k_begin = warp * per, k_end = min(n_cand, k_begin + per);
-        for (int k0 = k_begin; k0 < k_end; k0 += 32) {
-            const int k = k0 + lane;
-            float w = 0.f;
-            int64_t slot = -1;
-            if (k < k_end) {
-                slot = slot_of(k);
-                if (slot >= 0) {
-                    const float2 ml = a.part_ml[slot * a.G + gq];
-                    if (ml.x != -INFINITY) { w = __expf(ml.x - mg); lw_sum = fmaf(ml.y, w, lw_sum); }
-                }
-            }
-            const int nk = min(32, k_end - k0);
-            for (int j0 = 0; j0 < nk; j0 += 8) {
-                float wv[8];
-                float xv[8][VPL];
+        for (int v = 0; v < VPL; ++v) acc[v] *= rescale;
+        float lw = l_k * w;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int src = min(j0 + u, 31);
-                    const float wk = __shfl_sync(0xffffffffu, w, src);
-                    const int64_t sk = __shfl_sync(0xffffffffu, slot, src);
-                    wv[u] = (j0 + u < nk) ? wk : 0.f;
+        for (int s = 16; s >= 1; s >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, s);
+        l_w = l_w * rescale + lw;
+        m_w = m_new;
+        const int nk = min(32, k_end - k0);
+        for (int j0 = 0; j0 < nk; j0 += 8) {
+            float wv[8];
+            float xv[8][VPL];
 #pragma unroll
-                    for (int v = 0; v < VPL; ++v) xv[u][v] = 0.f;
-                    if (wv[u] != 0.f) {
-                        const float* po = a.part_o + (sk * a.G + gq) * D + lane * VPL;
-                        if (VPL == 4) {
-                            const float4 x = __ldg(reinterpret_cast<const float4*>(po));
-                            xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
-                        } else {
-                            const float2 x = __ldg(reinterpret_cast<const float2*>(po));
-                            xv[u][0] = x.x; xv[u][1] = x.y;
-                        }
+            for (int u = 0; u < 8; ++u) {
+                const int src = min(j0 + u, 31);
+                const float wk = __shfl_sync(0xffffffffu, w, src);
+                const int64_t sk = __shfl_sync(0xffffffffu, slot, src);
+                wv[u] = (j0 + u < nk) ? wk : 0.f;
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) xv[u][v] = 0.f;
+                if (wv[u] != 0.f) {
+                    const float* po = a.part_o + (sk * a.G + gq) * D + lane * VPL;
+                    if (VPL == 4) {
+                        const float4 x = __ldg(reinterpret_cast<const float4*>(po));
+                        xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
+                    } else {
+                        const float2 x = __ldg(reinterpret_cast<const float2*>(po));
+                        xv[u][0] = x.x; xv[u][1] = x.y;
                     }
                 }
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-#pragma unroll
-                    for (int v = 0; v < VPL; ++v) acc[v] = fmaf(xv[u][v], wv[u], acc[v]);
             }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) acc[v] = fmaf(xv[u][v], wv[u], acc[v]);
         }
     }
-    // lanes hold different candidates' l * w: sum inside the warp, then across warps in a fixed order
-#pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) lw_sum += __shfl_xor_sync(0xffffffffu, lw_sum, s);
 #pragma unroll
     for (int v = 0; v < VPL; ++v) s_acc[warp][lane * VPL + v] = acc[v];
-    if (lane == 0) s_l[warp] = lw_sum;
+    if (lane == 0) { s_l[warp] = l_w; s_m[warp] = m_w; }
     __syncthreads();
     if (tid < D) {
-        float o = 0.f, l = 0.f;
+        float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < MERGE_WARPS; ++w) { o += s_acc[w][tid]; l += s_l[w]; }
+        for (int w = 0; w < MERGE_WARPS; ++w) M = fmaxf(M, s_m[w]);
+        float o = 0.f, l = 0.f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < MERGE_WARPS; ++w) {
+                const float sc = (s_m[w] == -INFINITY) ? 0.f : __expf(s_m[w] - M);
+                o = fmaf(s_acc[w][tid], sc, o);
+                l = fmaf(s_l[w], sc, l);
+            }
+        }
         a.out[((int64_t)i * a.Hq + hk * a.G + gq) * D + tid] = l > 0.f ? o / l : 0.f;
     }
 }
@@ -1063,6 +1071,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.row_start = reinterpret_cast<int32_t*>(ws + L.row_start);
     da.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
     da.cta_range = reinterpret_cast<int2*>(ws + L.cta_range);
+    da.row_cand = reinterpret_cast<int2*>(ws + L.row_cand);
     da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
     da.part_o = reinterpret_cast<float*>(ws + L.part_o);
     da.status = status_dev;
@@ -1087,7 +1096,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     profile_mark(4, s);
 
     MergeArgs ma;
-    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.cta_range = da.cta_range; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
+    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.cta_range = da.cta_range; ma.row_cand = da.row_cand; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
     ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS;
     const unsigned mgrid = (unsigned)(L.rows * G);
     cudaError_t me = (D == 128) ? launch_pdl(merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
