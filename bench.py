@@ -39,6 +39,9 @@ DEFAULT_TARGET = 0.90
 CALIB = os.path.join(ROOT, "tests", "golden", "workload_calibration.json")
 PEAKS = os.path.join(ROOT, "MEASURED_PEAKS.json")
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) per launch of the streaming kernel from the ncu capture summarised in
+# profiles/decode_kernel_c3_128k_s90.md (mean of the two captured launches), keyed by (workload, target sparsity).
+NCU_TRAFFIC_BYTES = {("c3_128k", 0.90): 217.7e6}
 
 
 def load_bias(name: str, target: float) -> np.ndarray:
@@ -346,7 +349,8 @@ def run_ours(args):
                     "d2h_bytes_per_step": out_host.numel() * 4},
             "gpu_launches": args.steps * (2 + eb.eta_decode_kernel_count()),
             "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak,
-                         "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES.get((sp.name, main_target)), "traffic_unit": "bytes per launch",
                          "algorithmic_bytes_per_launch": ab["decode"]},
             "prefill_build": {"ms": build_ms, "gbs": k_bytes / (build_ms * 1e-3) / 1e9},
             "sweep": sweep,
@@ -360,11 +364,12 @@ def run_ours(args):
 
 def cpu_baseline(sp, w, bias, budget_s: float, steps: int | None = None):
     """The oracle, as it stands, on this machine's host cores: whole decode steps (threshold prediction, bounds,
-    selection, gated attention over the admitted blocks) on the first sequence of the workload."""
+    selection, gated attention over the admitted blocks) on the whole batch of the workload, a bounded number of
+    steps."""
     from oracle import eta_oracle as orc
     from tests.helpers import bits
     orc.build()
-    nseq = 1
+    nseq = sp.batch
     K, V = bits(w.K[:nseq]), bits(w.V[:nseq])
     lens = w.seq_lens.numpy().astype(np.int32)[:nseq].copy()
     c = orc.Cache(K, V, lens, sp.block_size)
@@ -383,12 +388,12 @@ def cpu_baseline(sp, w, bias, budget_s: float, steps: int | None = None):
         if steps is not None:
             if s >= steps:
                 break
-        elif time.perf_counter() - t_all > budget_s or s >= 64:
+        elif time.perf_counter() - t_all > budget_s or s >= 128:
             break
     per = sum(times) / len(times)
     return {"value": nseq / per, "unit": UNIT, "cores": orc.n_threads(), "kind": "oracle",
-            "sample": f"{len(times)} decode steps of sequence 0 of {sp.name} (1 of {sp.batch} sequences, all "
-                      f"{sp.n_q_heads} heads, full context)", "s_per_step": per}
+            "sample": f"{len(times)} decode steps of {sp.name} (all {sp.batch} sequences, all {sp.n_q_heads} heads, "
+                      f"full context), {sum(times):.1f} s of CPU work", "s_per_step": per}
 
 
 def run_reference(args):
