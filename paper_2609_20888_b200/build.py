@@ -30,6 +30,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared", "-o", LIB] + sources()
+    cmd[1:1] = os.environ.get("ETA_NVCC_FLAGS", "").split()     # e.g. -DETA_WAIT_LIMIT=65536 while debugging
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

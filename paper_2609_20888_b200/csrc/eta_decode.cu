@@ -53,18 +53,6 @@ constexpr int PIECE_COST = 3;          // tiles a row boundary inside a CTA's ra
 constexpr int RESC_ROWS = 8;           // rows (from the CTA's first) whose rescue decisions stay in shared memory
 constexpr int PW = 256;                // entries of the unit prefix the producer keeps in shared memory
 
-__device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
-    return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
-}
-// token row inside an 8-row group that MMA column n reads: bits 0 and 2 of n swapped, so that the two
-// rows a quarter-warp touches in one 16-byte load sit in different halves of the swizzle pattern
-__device__ __forceinline__ int rho(int n) { return (n & 2) | ((n & 1) << 2) | ((n >> 2) & 1); }
-__device__ __forceinline__ float rcp_approx(float x) {
-    float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
 
 // Top-1 rescue of query head g of row r (Algorithm 3, rescue phase): if none of the first
 // Wr = min(rescue_window, NB) blocks was admitted for the head, the first block with the largest bound among them
@@ -166,7 +154,15 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long* tl = a.timeline ? a.timeline + (size_t)blockIdx.x * 8 : nullptr;
     if (tl && tid == 0) tl[0] = globaltimer_ns();
+    // When NSTAGE is not a multiple of NGROUPS a stage serves different groups in successive rounds, and a parity
+    // wait only tells the current phase of a barrier from the one before it: a group that runs ahead could ask for
+    // round k of a stage while round k - 1 (another group's) has not completed and be told "done".  In those
+    // configurations the producer publishes the number of fills it has started (each only after the stage's
+    // previous round was consumed) and a consumer looks at its barrier only once its fill is among them.
+    constexpr bool SHARED_STAGES = (NSTAGE % NGROUPS) != 0;
+    __shared__ int s_fill_started;
     if (tid == 0) {
+        s_fill_started = 0;
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], WARPS_PER_GROUP); }
         for (int k = 0; k < NGROUPS; ++k) mbar_init(&flushbar[k], 32 * WARPS_PER_GROUP);
         fence_barrier_init();
@@ -518,6 +514,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                         if (!mbar_wait(&empty[stage], (round & 1) ^ 1)) {
                             ok = false;
                         } else {
+                            if (SHARED_STAGES) st_volatile(&s_fill_started, (int)fill + 1);
                             desc[stage] = make_int4(r, piece << 1, hmask, nvalid);
                             unsigned char* st = smem + stage * L::STAGE_BYTES;
                             mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
@@ -547,6 +544,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 if (!mbar_wait(&empty[stage], ((fill / NSTAGE) & 1) ^ 1)) {
                     ok = false;
                 } else {
+                    if (SHARED_STAGES) st_volatile(&s_fill_started, (int)fill + 1);
                     desc[stage] = make_int4(0, (int)UF_END, 0, 0);
                     mbar_arrive(&full[stage]);
                 }
@@ -619,6 +617,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     for (uint32_t fill = group;; fill += NGROUPS) {
         const int stage = fill % NSTAGE;
+        if (SHARED_STAGES) {
+            bool started = false;
+            for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+                if ((uint32_t)ld_volatile(&s_fill_started) > fill) { started = true; break; }
+                __nanosleep(40);
+            }
+            if (!started) { ok = false; break; }
+        }
         if (!mbar_wait(&full[stage], (fill / NSTAGE) & 1)) { ok = false; break; }
         const int4 ds = desc[stage];
         const bool end = (ds.y & (int)UF_END) != 0;
@@ -959,7 +965,7 @@ static EncodeTiledFn encode_fn() {
 
 // K or V as a 5-D tensor (c within a 64-column half, t, half, hk, i) of bf16; a box is 64 columns x TS tokens x
 // all halves: in shared memory, one 128-byte-swizzled [TS][64] tile per half, back to back.
-static int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d, int64_t sb, int64_t sh, int64_t st,
+int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d, int64_t sb, int64_t sh, int64_t st,
                      int TS) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return ETA_ERR_CUDA;
@@ -999,7 +1005,10 @@ static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const
 
 extern "C" {
 
-int eta_decode_kernel_count(void) { return 3; }
+static thread_local int g_last_kernel_count = 3;
+// Whether eta_decode picks the single-kernel path by itself where it applies (it is always available on request).
+static bool fused_default() { return false; }
+int eta_decode_kernel_count(void) { return g_last_kernel_count; }
 
 int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q, const void* K, const void* V,
                const int32_t* seq_lens, const void* musig, const float* mnorm, const float* tau,
@@ -1019,6 +1028,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     const WsLayout L = ws_layout(desc);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
         return ETA_ERR_WORKSPACE;
+    if ((params->flags & ETA_FLAG_THREE_KERNELS) && (params->flags & ETA_FLAG_SINGLE_KERNEL)) return ETA_ERR_INVALID_ARG;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -1033,6 +1043,19 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     const int TS = b < 64 ? b : 64;
     int n_ctas = n_sm;                  // one persistent CTA per SM; the shared-memory ring fills the SM
     if (n_ctas > MAX_CTAS) n_ctas = MAX_CTAS;
+
+    // Two ways to run the call.  The single kernel overlaps screening with streaming and wins whenever there
+    // are enough claims to keep every CTA busy; the three-kernel sequence lays the survivors out exactly and
+    // serves small problems, the dense baseline, wide rescue windows and workspaces of the minimum size.
+    const bool can_fuse = !dense && !(params->flags & ETA_FLAG_THREE_KERNELS) &&
+                          fused_eligible(desc, params, L, workspace_bytes);
+    if ((params->flags & ETA_FLAG_SINGLE_KERNEL) && !can_fuse) return ETA_ERR_UNSUPPORTED;
+    if (can_fuse && ((params->flags & ETA_FLAG_SINGLE_KERNEL) || (fused_default() && fused_claims(desc, params, L) >= 4 * n_ctas))) {
+        g_last_kernel_count = 2;
+        return launch_fused_decode(desc, params, L, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,
+                                   stats, status_dev, ws, n_ctas, s);
+    }
+    g_last_kernel_count = 3;
 
     ScreenArgs sa;
     sa.q = static_cast<const __nv_bfloat16*>(q);
