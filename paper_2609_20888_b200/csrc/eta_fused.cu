@@ -61,18 +61,17 @@ constexpr int F_SCR_WARP0 = F_PRODUCER_WARP + 1;
 constexpr int F_SCR_WARPS = 3;
 constexpr int F_SCR_THREADS = 32 * F_SCR_WARPS;
 constexpr int F_THREADS = 32 * (F_SCR_WARP0 + F_SCR_WARPS);
-constexpr int F_NSB = 3;                         // record buffers of the screening warps
+constexpr int F_NSB = F_SCR_WARPS;               // record buffers: one per screening warp
 constexpr int F_RING = 8;                        // chunk records between the screening warps and the producer
 constexpr int F_BACKLOG = 8;                     // list entries pushed but not yet issued above which screening pauses
 constexpr int F_LIST = FSEG + 12;
 constexpr uint32_t FD_END = 1u, FD_SKIP = 2u, FD_NEW = 4u, FD_LAST = 8u;
-constexpr int BAR_SCREEN = 1, BAR_GROUP0 = 2;
 
 struct ChunkRec { int row, slot, n, pad; int ent[FCH]; float te[8]; };
 struct LaneState { int n, k, sub, row, slot, nchunks, pad0, pad1; };
 
 // control words in shared memory
-enum { C_HEAD = 0, C_TAIL, C_DONE, C_PUSHED, C_ISSUED, C_CLAIMQ /* 4 words */, C_NLIST = C_CLAIMQ + 4, C_NBLK, C_FAIL, C_FILL, C_WORDS = 16 };
+enum { C_HEAD = 0, C_RESERVE, C_DONE, C_PUSHED, C_ISSUED, C_FAIL, C_FILL, C_WORDS = 8 };
 
 template <int D, int TS, int NSTAGE, int G>
 struct FusedSmem {
@@ -86,18 +85,15 @@ struct FusedSmem {
     static constexpr int SBUF_OFF = NSTAGE * STAGE_BYTES;
     static constexpr int QBUF_OFF = SBUF_OFF + F_NSB * SBUF_BYTES;
     static constexpr int BAR_OFF = QBUF_OFF + F_GROUPS * NQB * QB_BYTES;       // full, empty, sbar
-    static constexpr int DESC_OFF = BAR_OFF + 8 * ((2 * NSTAGE + F_NSB + 1) & ~1);
+    static constexpr int DESC_OFF = BAR_OFF + 8 * ((2 * NSTAGE + F_NSB + F_GROUPS + 1) & ~1);
     static constexpr int HTE_OFF = DESC_OFF + 16 * NSTAGE;                     // float [groups][NQB][8]
     static constexpr int RING_OFF = HTE_OFF + 4 * F_GROUPS * NQB * 8;
     static constexpr int LST_OFF = RING_OFF + (int)sizeof(ChunkRec) * F_RING;
     static constexpr int LENT_OFF = LST_OFF + (int)sizeof(LaneState) * F_GROUPS;
     static constexpr int CTRL_OFF = LENT_OFF + 4 * F_GROUPS * FCH;
-    static constexpr int BOUND_OFF = CTRL_OFF + 4 * C_WORDS;                   // float [FSEG][G]
-    static constexpr int MN_OFF = BOUND_OFF + 4 * FSEG * G;
-    static constexpr int MASK_OFF = MN_OFF + 4 * FSEG;
-    static constexpr int LIST_OFF = MASK_OFF + FSEG;
-    static constexpr int WST_OFF = LIST_OFF + 4 * F_LIST;                      // int cnt[8], float best[8], int arg[8]
-    static constexpr int ML_OFF = WST_OFF + 96;                                // float [groups][2][F_WPG][8]
+    static constexpr int READY_OFF = CTRL_OFF + 4 * C_WORDS;                   // int [F_RING]: slot + 1 once its record is written
+    static constexpr int LIST_OFF = READY_OFF + 4 * F_RING;                    // int [F_SCR_WARPS][F_LIST]
+    static constexpr int ML_OFF = LIST_OFF + 4 * F_LIST * F_SCR_WARPS;         // float [groups][2][F_WPG][8]
     static constexpr int LEN_OFF = ML_OFF + 4 * F_GROUPS * 2 * F_WPG * 8;      // int len[rows], float te[rows * G]
     static size_t bytes(int rows) { return 1024 + LEN_OFF + (size_t)4 * rows * (1 + G); }
 };
@@ -118,6 +114,7 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::BAR_OFF);
     uint64_t* empty = full + NSTAGE;
     uint64_t* sbar = empty + NSTAGE;
+    uint64_t* flushbar = sbar + F_NSB;         // one per consumer group: its four warps meet here at the end of a chunk
     int4* desc = reinterpret_cast<int4*>(smem + L::DESC_OFF);
     float* hte = reinterpret_cast<float*>(smem + L::HTE_OFF);
     ChunkRec* ring = reinterpret_cast<ChunkRec*>(smem + L::RING_OFF);
@@ -139,10 +136,12 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], F_WPG); }
         for (int k = 0; k < F_NSB; ++k) mbar_init(&sbar[k], 1);
+        for (int k = 0; k < F_GROUPS; ++k) mbar_init(&flushbar[k], 32 * F_WPG);
         fence_barrier_init();
         prefetch_tmap(&tmK);
         prefetch_tmap(&tmV);
         for (int k = 0; k < C_WORDS; ++k) ctrl[k] = 0;
+        for (int k = 0; k < F_RING; ++k) reinterpret_cast<int*>(smem + L::READY_OFF)[k] = 0;
         for (int k = 0; k < (int)(sizeof(LaneState) / 4) * F_GROUPS; ++k) reinterpret_cast<int*>(lst)[k] = 0;
     }
     // sequence lengths are a caller input: they can be read while the previous kernel is still running
@@ -154,64 +153,38 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 
     if (warp >= F_SCR_WARP0) {
         // ======================================================================= screening warps
-        constexpr int LPR = D / 8;            // lanes sharing one record
-        constexpr int RPW = 32 / LPR;         // records per warp instruction
-        constexpr int NI = LPR / G;           // iterations whose partial sums are reduced together
-        constexpr int NV = 2 * LPR;           // partial sums per lane before the butterfly
-        constexpr int RB = RPW * NI;          // records per warp per batch
+        // Each warp works on items of its own: a lane per record.  A lane walks the head_dim of its record in
+        // 16-byte pieces, starting at a piece that depends on the lane so that the lanes of a quarter-warp always
+        // hit different banks, and keeps the two sums of Eq. dual_bound_eq for the G heads in registers.
         constexpr int REC_BYTES = L::REC_BYTES;
-        constexpr bool USE_Q2 = (G <= 4);
-        static_assert(NI >= 1, "group size too large for this head_dim");
-        float (*sbound)[G] = reinterpret_cast<float (*)[G]>(smem + L::BOUND_OFF);
-        float* smn = reinterpret_cast<float*>(smem + L::MN_OFF);
-        int* s_list = reinterpret_cast<int*>(smem + L::LIST_OFF);
-        int* w_cnt = reinterpret_cast<int*>(smem + L::WST_OFF);
-        float* w_best = reinterpret_cast<float*>(w_cnt + 8);
-        int* w_arg = w_cnt + 16;
-
-        const int stid = tid - 32 * F_SCR_WARP0, swarp = warp - F_SCR_WARP0;
-        const int cc = lane % LPR, rg = lane / LPR;
-        const int my_g = cc % G;
+        constexpr int NCH = D / 8;                      // 16-byte pieces per vector
+        int* s_list = reinterpret_cast<int*>(smem + L::LIST_OFF) + (warp - F_SCR_WARP0) * F_LIST;
+        int* ready = reinterpret_cast<int*>(smem + L::READY_OFF);
+        const int sw = warp - F_SCR_WARP0;
         const int P = gridDim.x, NC = a.n_claims;
+        const int NSWG = P * F_SCR_WARPS;               // screening warps of the whole grid
+        const int wg = blockIdx.x * F_SCR_WARPS + sw;
+        unsigned char* buf = smem + L::SBUF_OFF + sw * L::SBUF_BYTES;
+        const uint32_t rec_base = smem_u32(buf) + lane * REC_BYTES;
+        const uint32_t q_base = smem_u32(buf) + FSEG * REC_BYTES;
 
-        // the first three claims are fixed by the CTA's index; later ones come from the counter (or, on a workspace
-        // that does not carry the magic number yet, from the same fixed pattern)
+        // the first claim is fixed by the warp's index; later ones come from the counter (or, on a workspace that
+        // does not carry the magic number yet, from the same fixed pattern)
         bool dynamic = false;
-        int pend = NC;                    // thread 0: id of the claim three ahead of the current one
-        if (stid == 0) {
+        if (lane == 0) {
             const int m0 = ld_volatile(a.f_hdr), m1 = ld_volatile(a.f_hdr + 1);
             dynamic = ((uint32_t)m0 == F_MAGIC0 && (uint32_t)m1 == F_MAGIC1);
-            ctrl[C_CLAIMQ + 0] = blockIdx.x;
-            ctrl[C_CLAIMQ + 1] = blockIdx.x + P;
-            ctrl[C_CLAIMQ + 2] = blockIdx.x + 2 * P;
-            pend = dynamic ? 3 * P + atomicAdd(a.f_hdr + 2, 1) : blockIdx.x + 3 * P;
         }
-        named_barrier(BAR_SCREEN, F_SCR_THREADS);
+        dynamic = __shfl_sync(0xffffffffu, dynamic ? 1 : 0, 0) != 0;
 
-        struct Cur { int m, pos, row, it0, nit; bool valid; };
-        auto cur_load = [&](Cur& c) {
-            const int cid = ctrl[C_CLAIMQ + (c.m & 3)];
-            c.valid = cid < NC;
-            c.pos = 0; c.row = 0; c.it0 = 0; c.nit = 1;
-            if (c.valid) {
-                if (cid < a.rows) { c.row = cid; c.it0 = 0; c.nit = a.nwi; }
-                else { a.div_spr.divmod(cid - a.rows, c.row, c.it0); c.it0 += a.nwi; c.nit = 1; }
-            }
-        };
-        // A cursor moves lazily: the id of the next claim is looked up only when the cursor is used, which is when
-        // that id is certain to have been published (claim m + 2 is published as claim m starts).
-        auto cur_next = [&](Cur& c) { ++c.pos; };
-        auto cur_fix = [&](Cur& c) {
-            if (c.valid && c.pos >= c.nit) { ++c.m; cur_load(c); }
-        };
         struct Geom { int r, fit, i, hk, T, NB, j0, n_rec; };
-        auto geom_of = [&](const Cur& c) {
+        auto geom_of = [&](int row, int fit) {
             Geom g;
-            g.r = c.row; g.fit = c.it0 + c.pos;
-            a.div_hkv.divmod(g.r, g.i, g.hk);
-            g.T = s_len[g.r];
+            g.r = row; g.fit = fit;
+            a.div_hkv.divmod(row, g.i, g.hk);
+            g.T = s_len[row];
             g.NB = min(g.T >> a.b_shift, a.nb_cap);
-            g.j0 = g.fit * FSEG;
+            g.j0 = fit * FSEG;
             g.n_rec = max(0, min(FSEG, g.NB - g.j0));
             return g;
         };
@@ -226,321 +199,296 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             pdl_wait();
             waited = true;
         };
-        auto issue = [&](const Geom& g, int n) {          // thread 0: copies of item number n of this CTA
-            const int buf = n % F_NSB;
+        auto issue = [&](const Geom& g) {          // lane 0: copies of an item into this warp's buffer
             if (g.n_rec > 0) {
-                unsigned char* dst = smem + L::SBUF_OFF + buf * L::SBUF_BYTES;
                 const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
                                            ((int64_t)g.r * a.nb_cap + g.j0) * REC_BYTES;
-                mbar_arrive_expect_tx(&sbar[buf], g.n_rec * REC_BYTES + L::QB_BYTES);
-                tma_load_1d(dst, src, g.n_rec * REC_BYTES, &sbar[buf]);
-                tma_load_1d(dst + FSEG * REC_BYTES, a.q + ((int64_t)g.i * a.Hq + g.hk * G) * D, L::QB_BYTES, &sbar[buf]);
+                mbar_arrive_expect_tx(&sbar[sw], g.n_rec * REC_BYTES + L::QB_BYTES);
+                tma_load_1d(buf, src, g.n_rec * REC_BYTES, &sbar[sw]);
+                tma_load_1d(buf + FSEG * REC_BYTES, a.q + ((int64_t)g.i * a.Hq + g.hk * G) * D, L::QB_BYTES, &sbar[sw]);
             } else {
-                mbar_arrive(&sbar[buf]);
+                mbar_arrive(&sbar[sw]);
             }
         };
-        auto load_mn = [&](const Geom& g) {
-            return (stid < g.n_rec) ? __ldg(a.mnorm + (int64_t)g.r * a.nb_cap + g.j0 + stid) : 0.f;
+        auto load_mn = [&](const Geom& g) {        // this lane's record's largest key norm
+            return (lane < g.n_rec) ? __ldg(a.mnorm + (int64_t)g.r * a.nb_cap + g.j0 + lane) : 0.f;
         };
-
-        Cur cp, ce;                     // processing and look-ahead cursors
-        cp.m = 0; cur_load(cp);
-        ce = cp;
-        int n_enum = 0;                 // items enumerated (= copies started) so far
-        float mn0 = 0.f, mn1 = 0.f, mn2 = 0.f;    // max-norm entries of items n, n + 1, n + 2 (thread = record)
-        // start the copies of the first two items
-        for (int k = 0; k < 2; ++k) {
-            cur_fix(ce);
-            if (ce.valid) {
-                const Geom g = geom_of(ce);
-                if (!safe_item(g)) wait_pred();
-                if (stid == 0) issue(g, n_enum);
-                const float v = load_mn(g);
-                if (k == 0) mn0 = v; else mn1 = v;
-                ++n_enum;
-                cur_next(ce);
-            }
-        }
-
-        float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G], my_qn = 0.f;
-        int q_row = -1;
-        bool te_ready = false;
-
-        const int n_items_all = a.rows * a.nfs;
-        for (int n = 0;; ++n) {
-            cur_fix(cp);
-            if (!cp.valid) break;
-            if (n > n_items_all) { ctrl[C_FAIL] = 1; break; }     // cannot happen: no CTA has more items than there are
-            const Geom gc = geom_of(cp);
-            const int buf = n % F_NSB;
-            const bool first_of_claim = cp.pos == 0, last_of_claim = cp.pos + 1 == cp.nit;
-            const bool win_claim = cp.it0 == 0;       // the claim of a row's rescue window starts at item 0
-            const int r = gc.r, NB = gc.NB, j0 = gc.j0, n_rec = gc.n_rec;
-
-            if (pg && stid == 0) pg[1] = ((unsigned long long)n << 8) | 1;
-            if (xt && stid == 0 && n == 3) xt[1] = globaltimer_ns();
-            if (stid == 0) {
+        auto load_te = [&](const Geom& g) {        // lane g < G: effective threshold of head g of the item's group
+            if (lane >= G) return 0.f;
+            const int h = g.hk * G + lane;
+            return (a.tau ? __ldg(a.tau + (int64_t)g.i * a.Hq + h) : __ldg(a.head_const + h)) - a.a;
+        };
+        auto claim_items = [&](int cid, int& row, int& it0, int& nit) {
+            if (cid < a.rows) { row = cid; it0 = 0; nit = a.nwi; }
+            else { a.div_spr.divmod(cid - a.rows, row, it0); it0 += a.nwi; nit = 1; }
+        };
+        // id of the claim after the current one: asked for (lane 0) as an item starts, used when it ends
+        int n_claimed = 1;
+        auto ask_claim = [&]() {
+            int v = NC;
+            if (lane == 0) {
                 // pause while the producer has enough to issue: claims taken early are claims taken from others
                 for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
                     if (ld_volatile(ctrl + C_PUSHED) - ld_volatile(ctrl + C_ISSUED) < F_BACKLOG) break;
                     __nanosleep(100);
                 }
-                if (first_of_claim && cp.m >= 1) {
-                    // publish the claim two ahead (asked for one claim ago) and ask for the one after it
-                    ctrl[C_CLAIMQ + ((cp.m + 2) & 3)] = pend;
-                    pend = dynamic ? 3 * P + atomicAdd(a.f_hdr + 2, 1) : blockIdx.x + (cp.m + 3) * P;
+                v = dynamic ? NSWG + atomicAdd(a.f_hdr + 2, 1) : wg + n_claimed * NSWG;
+            }
+            ++n_claimed;
+            return v;
+        };
+
+        int cid = wg;
+        int row = 0, it0 = 0, nit = 1, pos = 0;
+        bool have = cid < NC;
+        Geom gc = {};
+        float mn_cur = 0.f, te_cur = 0.f;
+        bool te_have = false;
+        uint32_t n_items = 0;
+        if (have) {
+            claim_items(cid, row, it0, nit);
+            gc = geom_of(row, it0);
+            if (!safe_item(gc)) wait_pred();
+            if (lane == 0) issue(gc);
+            mn_cur = load_mn(gc);
+        }
+        // window statistics of a rescue-window claim (uniform across the warp)
+        int w_cnt[G], w_arg[G];
+        float w_best[G];
+
+        while (have) {
+            const bool first_of_claim = pos == 0, last_of_claim = pos + 1 == nit;
+            const bool win_claim = it0 == 0;
+            const int r = gc.r, NB = gc.NB, j0 = gc.j0, n_rec = gc.n_rec;
+            if (xt && sw == 0 && lane == 0 && n_items == 3) xt[1] = globaltimer_ns();
+            int pend = NC;
+            if (last_of_claim) pend = ask_claim();
+            if (first_of_claim && win_claim) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) { w_cnt[g] = 0; w_arg[g] = -1; w_best[g] = -INFINITY; }
+            }
+            if (xt && sw == 0 && lane == 0 && n_items == 3) xt[2] = globaltimer_ns();
+            bool ok = mbar_wait(&sbar[sw], n_items & 1);
+            if (!__all_sync(0xffffffffu, ok)) {
+                if (lane == 0) { ctrl[C_FAIL] = 1; if (tl) tl[7] = (1ull << 32) | n_items; }
+                break;
+            }
+            if (xt && sw == 0 && lane == 0 && n_items == 3) xt[3] = globaltimer_ns();
+
+            float bound[G];
+            if (n_rec > 0) {
+                // ||q_g||: the lanes of a half-warp split the pieces of q_g
+                float qn[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const uint4 v = lds128(q_base + g * 2 * D + (lane % NCH) * 16);
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                    float n2 = 0.f;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const float x0 = bf16_lo(w[kk]), x1 = bf16_hi(w[kk]);
+                        n2 = fmaf(x0, x0, n2);
+                        n2 = fmaf(x1, x1, n2);
+                    }
+#pragma unroll
+                    for (int s = 1; s < NCH; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+                    qn[g] = sqrtf(n2);
                 }
-            }
-            if (first_of_claim && win_claim && stid < 8) { w_cnt[stid] = 0; w_best[stid] = -INFINITY; w_arg[stid] = -1; }
-            if (stid < FSEG) smn[stid] = mn0;
-            if (pg && stid == 0) pg[1] = ((unsigned long long)n << 8) | 2;
-            if (xt && stid == 0 && n == 3) xt[2] = globaltimer_ns();
-            named_barrier(BAR_SCREEN, F_SCR_THREADS);
-            if (ctrl[C_FAIL]) break;          // a wait ran out somewhere in the previous item: every thread sees it here
-            if (pg && stid == 0) pg[1] = ((unsigned long long)n << 8) | 3;
-            if (xt && stid == 0 && n == 3) xt[3] = globaltimer_ns();
-
-            // look ahead: start the copies of item n + 2
-            cur_fix(ce);
-            if (ce.valid) {
-                const Geom g = geom_of(ce);
-                if (!safe_item(g)) wait_pred();
-                if (stid == 0) issue(g, n_enum);
-                mn2 = load_mn(g);
-                ++n_enum;
-                cur_next(ce);
-            } else {
-                mn2 = 0.f;
-            }
-
-
-            bool ok = true;
-            if (pg && stid == 0) pg[1] = ((unsigned long long)n << 8) | 4;
-            if (xt && stid == 0 && n == 3) xt[4] = globaltimer_ns();
-            if (!mbar_wait(&sbar[buf], (n / F_NSB) & 1)) { ok = false; ctrl[C_FAIL] = 1; if (tl) tl[7] = (1ull << 32) | (unsigned)n; }
-            if (n_rec > 0 && ok) {
-                const uint32_t rec_base = smem_u32(smem + L::SBUF_OFF + buf * L::SBUF_BYTES);
-                if (r != q_row) {
-                    q_row = r;
+                float dot[G], var[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) { dot[g] = 0.f; var[g] = 0.f; }
+#pragma unroll 2
+                for (int c = 0; c < NCH; ++c) {
+                    const int cc = (c + lane) % NCH;
+                    const uint4 m4 = lds128(rec_base + cc * 16), s4 = lds128(rec_base + 2 * D + cc * 16);
+                    const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw4[4] = {s4.x, s4.y, s4.z, s4.w};
+                    float mu[8], sg[8];
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw[kk]));
+                        const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw4[kk]));
+                        mu[2 * kk] = mf.x; mu[2 * kk + 1] = mf.y;
+                        sg[2 * kk] = sf.x; sg[2 * kk + 1] = sf.y;
+                    }
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
-                        const uint4 v = lds128(rec_base + FSEG * REC_BYTES + (g * D + cc * 8) * 2);
-                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                        float n2 = 0.f;
+                        const uint4 q4 = lds128(q_base + g * 2 * D + cc * 16);
+                        const uint32_t qw[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk) {
-                            qf[g][2 * kk] = bf16_lo(w[kk]);
-                            qf[g][2 * kk + 1] = bf16_hi(w[kk]);
+                            const float x0 = bf16_lo(qw[kk]), x1 = bf16_hi(qw[kk]);
+                            dot[g] = fmaf(x0, mu[2 * kk], dot[g]);
+                            dot[g] = fmaf(x1, mu[2 * kk + 1], dot[g]);
+                            const float t0 = x0 * sg[2 * kk], t1 = x1 * sg[2 * kk + 1];
+                            var[g] = fmaf(t0, t0, var[g]);
+                            var[g] = fmaf(t1, t1, var[g]);
                         }
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            n2 = fmaf(qf[g][kk], qf[g][kk], n2);
-                            if (USE_Q2) q2[g][kk] = qf[g][kk] * qf[g][kk];
-                        }
-#pragma unroll
-                        for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
-                        qn[g] = sqrtf(n2);
                     }
-                    my_qn = qn[0];
-#pragma unroll
-                    for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
                 }
-                for (int base = swarp * RB; base < n_rec; base += F_SCR_WARPS * RB) {
-                    float v[NV];
 #pragma unroll
-                    for (int it = 0; it < NI; ++it) {
-                        const int rec = base + it * RPW + rg;
-                        float mu[8], s2[8];
-                        if (rec < n_rec) {
-                            const uint32_t addr = rec_base + rec * REC_BYTES + cc * 16;
-                            const uint4 m4 = lds128(addr), s4 = lds128(addr + 2 * D);
-                            const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw[4] = {s4.x, s4.y, s4.z, s4.w};
+                for (int g = 0; g < G; ++g)
+                    bound[g] = a.scale * min_keep_nan(dot[g] + a.z * sqrtf(var[g]), qn[g] * mn_cur);
+            } else {
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk) {
-                                float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw[kk]));
-                                float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
-                                mu[2 * kk] = mf.x; mu[2 * kk + 1] = mf.y;
-                                s2[2 * kk] = USE_Q2 ? sf.x * sf.x : sf.x;
-                                s2[2 * kk + 1] = USE_Q2 ? sf.y * sf.y : sf.y;
-                            }
-                        } else {
+                for (int g = 0; g < G; ++g) bound[g] = 0.f;
+            }
+            if (xt && sw == 0 && lane == 0 && n_items == 3) xt[4] = globaltimer_ns();
+
+            // ---- the buffer is free: start the copies of the warp's next item
+            int nrow = row, nit0 = it0, nnit = nit, npos = pos + 1;
+            bool nhave = true;
+            if (last_of_claim) {
+                const int ncid = __shfl_sync(0xffffffffu, pend, 0);
+                nhave = ncid < NC;
+                npos = 0;
+                if (nhave) claim_items(ncid, nrow, nit0, nnit);
+            }
+            Geom gn = gc;
+            float mn_next = 0.f, te_next = 0.f;
+            bool te_next_have = false;
+            __syncwarp();
+            fence_proxy_async();          // this warp's reads of the buffer are ordered before the next copy into it
+            if (nhave) {
+                gn = geom_of(nrow, nit0 + npos);
+                if (!safe_item(gn)) wait_pred();
+                if (lane == 0) issue(gn);
+                mn_next = load_mn(gn);
+                if (waited) { te_next = load_te(gn); te_next_have = true; }
+            }
+            // the thresholds of this item, if they could not be fetched ahead (first item of the warp)
+            if (!te_have) { wait_pred(); te_cur = load_te(gc); te_have = true; }
+            if (xt && sw == 0 && lane == 0 && n_items == 3) xt[5] = globaltimer_ns();
+
+            // ---- admission bits, survivors in ascending order, window statistics
+            float te_g[G];
 #pragma unroll
-                            for (int kk = 0; kk < 8; ++kk) { mu[kk] = 0.f; s2[kk] = 0.f; }
-                        }
+            for (int g = 0; g < G; ++g) te_g[g] = __shfl_sync(0xffffffffu, te_cur, g);     // lane g holds head g's
+            unsigned m = 0;
+            if (lane < n_rec) {
+                const bool pinned = (j0 + lane) >= NB - a.lwb;
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    if (!(bound[g] < te_g[g]) || pinned) m |= 1u << g;
+            }
+            if (j0 + lane < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + lane] = (uint8_t)m;
+            const unsigned nz = __ballot_sync(0xffffffffu, m != 0);
+            if (m) s_list[__popc(nz & ((1u << lane) - 1u))] = (j0 + lane) | (int)(m << 24);
+            int nl = __popc(nz), nblk = nl;
+            if (win_claim) {
+                // rescue statistics of the part of the rescue window inside this item, per query head
+                const int Wr = min(a.rescue_window, NB);
+                const int nwin = min(n_rec, Wr - j0);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    int cnt = (lane < nwin) ? (int)((m >> g) & 1u) : 0;
+                    float best = (lane < nwin) ? bound[g] : -INFINITY;
+                    int arg = (lane < nwin) ? lane : 0x7fffffff;
+#pragma unroll
+                    for (int s = 16; s >= 1; s >>= 1) {
+                        cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
+                        const float ob = __shfl_xor_sync(0xffffffffu, best, s);
+                        const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
+                        if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+                    }
+                    if (nwin > 0) {
+                        w_cnt[g] += cnt;
+                        if (best > w_best[g] && arg != 0x7fffffff) { w_best[g] = best; w_arg[g] = j0 + arg; }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                if (win_claim && last_of_claim) {
+                    // top-1 rescue: a head with no admitted block in the window gets the window's best block
+                    const int Wr = min(a.rescue_window, NB);
+                    const int n0 = nl;
+                    if (Wr > 0) {
 #pragma unroll
                         for (int g = 0; g < G; ++g) {
-                            float dot = 0.f, var = 0.f;
-#pragma unroll
-                            for (int kk = 0; kk < 8; ++kk) {
-                                dot = fmaf(qf[g][kk], mu[kk], dot);
-                                if (USE_Q2) {
-                                    var = fmaf(q2[g][kk], s2[kk], var);
-                                } else {
-                                    const float t = qf[g][kk] * s2[kk];
-                                    var = fmaf(t, t, var);
-                                }
-                            }
-                            v[(it * G + g) * 2] = dot;
-                            v[(it * G + g) * 2 + 1] = var;
+                            if (w_cnt[g] != 0) continue;
+                            const int j = w_arg[g] < 0 ? 0 : w_arg[g];
+                            uint8_t* mp = a.sel_mask + (int64_t)r * a.nb_cap + j;
+                            const unsigned w = *reinterpret_cast<volatile uint8_t*>(mp);
+                            if (w == 0) ++nblk;
+                            *reinterpret_cast<volatile uint8_t*>(mp) = (uint8_t)(w | (1u << g));
+                            bool merged = false;
+                            for (int k = n0; k < nl; ++k)
+                                if ((s_list[k] & 0xffffff) == j) { s_list[k] |= 1 << (24 + g); merged = true; }
+                            if (!merged) s_list[nl++] = j | (1 << (24 + g));
                         }
                     }
-                    // transposed butterfly over the LPR lanes of a record: halves the values held at every step
-#pragma unroll
-                    for (int s = LPR / 2, nn = NV / 2; s >= 1; s >>= 1, nn >>= 1) {
-                        const bool upper = (lane & s) != 0;
-#pragma unroll
-                        for (int kk = 0; kk < nn; ++kk) {
-                            const float send = upper ? v[kk] : v[kk + nn];
-                            const float keep = upper ? v[kk + nn] : v[kk];
-                            v[kk] = keep + __shfl_xor_sync(0xffffffffu, send, s);
-                        }
-                    }
-                    // lane cc now holds (dot, var) of pair cc = it * G + g
-                    const int it = cc / G;
-                    const int rec = base + it * RPW + rg;
-                    const bool valid = rec < n_rec;
-                    const float mnv = valid ? smn[rec] : 0.f;
-                    const float bound = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * mnv);
-                    if (valid) sbound[rec][my_g] = bound;
+                }
+                // the row's tail rides with the item of the row's last full block
+                const int tail_fit = NB > 0 ? (NB - 1) / FSEG : 0;
+                if (gc.fit == tail_fit && gc.T > NB * a.b) s_list[nl++] = NB | (0xff << 24);
+                a.f_count[(int64_t)r * a.nfs + gc.fit] = nl | (nblk << 8);
+                if (gc.fit == 0 && a.status) {
+                    const int Traw = __ldg(a.seq_lens + gc.i);
+                    if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
+                    if (Traw <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
                 }
             }
-            if (pg && stid == 0) pg[1] = ((unsigned long long)n << 8) | 5;
-            if (xt && stid == 0 && n == 3) xt[5] = globaltimer_ns();
-            // the thresholds: read once, after the predictor is known to be complete
-            if (!te_ready) {
-                wait_pred();
-                for (int p = stid; p < a.rows * G; p += F_SCR_THREADS) {
-                    const int rr = p / G, g = p % G;
-                    int i2, hk2;
-                    a.div_hkv.divmod(rr, i2, hk2);
-                    const int h = hk2 * G + g;
-                    s_te[p] = (a.tau ? __ldg(a.tau + (int64_t)i2 * a.Hq + h) : __ldg(a.head_const + h)) - a.a;
-                }
-                te_ready = true;
-            }
-            named_barrier(BAR_SCREEN, F_SCR_THREADS);
+            nl = __shfl_sync(0xffffffffu, nl, 0);
+            if (xt && sw == 0 && lane == 0 && n_items == 3) xt[6] = globaltimer_ns();
 
-            if (pg && stid == 0) pg[1] = ((unsigned long long)n << 8) | 6;
-            if (xt && stid == 0 && n == 3) xt[6] = globaltimer_ns();
-            // admission bits, survivors in ascending order, window statistics
-            if (swarp == 0) {
-                const int rec = lane;
-                unsigned m = 0;
-                if (rec < n_rec) {
-                    const bool pinned = (j0 + rec) >= NB - a.lwb;
-#pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        const float bd = sbound[rec][g];
-                        if (!(bd < s_te[r * G + g]) || pinned) m |= 1u << g;
-                    }
-                }
-                if (j0 + rec < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + rec] = (uint8_t)m;
-                const unsigned nz = __ballot_sync(0xffffffffu, m != 0);
-                if (m) s_list[__popc(nz & ((1u << lane) - 1u))] = (j0 + rec) | (int)(m << 24);
-                if (lane == 0) { ctrl[C_NLIST] = __popc(nz); ctrl[C_NBLK] = __popc(nz); }
-                if (win_claim) {
-                    // rescue statistics of the part of the rescue window inside this item, per query head
-                    const int Wr = min(a.rescue_window, NB);
-                    const int nwin = min(n_rec, Wr - j0);
-#pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        int cnt = (rec < nwin) ? (int)((m >> g) & 1u) : 0;
-                        float best = (rec < nwin) ? sbound[rec][g] : -INFINITY;
-                        int arg = (rec < nwin) ? rec : 0x7fffffff;
-#pragma unroll
-                        for (int s = 16; s >= 1; s >>= 1) {
-                            cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
-                            const float ob = __shfl_xor_sync(0xffffffffu, best, s);
-                            const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
-                            if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
-                        }
-                        if (lane == 0 && nwin > 0) {
-                            w_cnt[g] += cnt;
-                            if (best > w_best[g] && arg != 0x7fffffff) { w_best[g] = best; w_arg[g] = j0 + arg; }
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) {
-                    int nl = ctrl[C_NLIST], nblk = nl;
-                    if (win_claim && last_of_claim) {
-                        // top-1 rescue: a head with no admitted block in the window gets the window's best block
-                        const int Wr = min(a.rescue_window, NB);
-                        const int n0 = nl;
-                        if (Wr > 0) {
-                            for (int g = 0; g < G; ++g) {
-                                if (w_cnt[g] != 0) continue;
-                                const int j = w_arg[g] < 0 ? 0 : w_arg[g];
-                                uint8_t* mp = a.sel_mask + (int64_t)r * a.nb_cap + j;
-                                const unsigned w = *reinterpret_cast<volatile uint8_t*>(mp);
-                                if (w == 0) ++nblk;
-                                *reinterpret_cast<volatile uint8_t*>(mp) = (uint8_t)(w | (1u << g));
-                                bool merged = false;
-                                for (int k = n0; k < nl; ++k)
-                                    if ((s_list[k] & 0xffffff) == j) { s_list[k] |= 1 << (24 + g); merged = true; }
-                                if (!merged) s_list[nl++] = j | (1 << (24 + g));
-                            }
-                        }
-                    }
-                    // the row's tail rides with the item of the row's last full block
-                    const int tail_fit = NB > 0 ? (NB - 1) / FSEG : 0;
-                    if (gc.fit == tail_fit && gc.T > NB * a.b) s_list[nl++] = NB | (0xff << 24);
-                    ctrl[C_NLIST] = nl;
-                    a.f_count[(int64_t)r * a.nfs + gc.fit] = nl | (nblk << 8);
-                    if (gc.fit == 0 && a.status) {
-                        const int Traw = __ldg(a.seq_lens + gc.i);
-                        if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
-                        if (Traw <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
-                    }
-                }
-                __syncwarp();
-                if (pg && stid == 0) pg[1] = ((unsigned long long)n << 8) | 7;
-            if (xt && stid == 0 && n == 3) xt[7] = globaltimer_ns();
-                // hand the list to the producer in chunks
-                const int nl = ctrl[C_NLIST];
-                for (int c0 = 0; c0 < nl && ok; c0 += FCH) {
+            // ---- hand the list to the producer in chunks: slots of the ring are reserved in order and filled
+            // independently; the producer takes a slot when its owner has marked it ready
+            if (nl > 0) {
+                const int nch = (nl + FCH - 1) / FCH;
+                int slot0 = 0;
+                if (lane == 0) slot0 = atomicAdd(ctrl + C_RESERVE, nch);
+                slot0 = __shfl_sync(0xffffffffu, slot0, 0);
+                bool pushed_ok = true;
+                for (int c = 0; c < nch && pushed_ok; ++c) {
+                    const int slot = slot0 + c, c0 = c * FCH;
                     const int cn = min(FCH, nl - c0);
-                    int tail = ctrl[C_TAIL];
                     if (lane == 0) {
                         bool room = false;
                         for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-                            if (tail - ld_volatile(ctrl + C_HEAD) < F_RING) { room = true; break; }
+                            if (slot - ld_volatile(ctrl + C_HEAD) < F_RING) { room = true; break; }
                             __nanosleep(100);
                         }
-                        if (!room) { ok = false; ctrl[C_FAIL] = 1; if (tl) tl[7] = (2ull << 32) | (unsigned)tail; }
+                        if (!room) { pushed_ok = false; ctrl[C_FAIL] = 1; if (tl) tl[7] = (2ull << 32) | (unsigned)slot; }
                     }
-                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                    if (!ok) break;
-                    ChunkRec* rec = &ring[tail % F_RING];
+                    pushed_ok = __shfl_sync(0xffffffffu, pushed_ok ? 1 : 0, 0) != 0;
+                    if (!pushed_ok) break;
+                    ChunkRec* rec = &ring[slot % F_RING];
                     if (lane < cn) rec->ent[lane] = s_list[c0 + lane];
-                    if (lane < 8) rec->te[lane] = (lane < G) ? s_te[r * G + lane] : 0.f;
+                    if (lane < 8) rec->te[lane] = (lane < G) ? te_cur : 0.f;
                     if (lane == 0) {
                         rec->row = r;
-                        rec->slot = (r * a.nfs + gc.fit) * FCPI + c0 / FCH;
+                        rec->slot = (r * a.nfs + gc.fit) * FCPI + c;
                         rec->n = cn;
                     }
                     __syncwarp();
                     if (lane == 0) {
                         __threadfence_block();
-                        st_volatile(ctrl + C_TAIL, tail + 1);
-                        st_volatile(ctrl + C_PUSHED, ctrl[C_PUSHED] + cn);
+                        st_volatile(ready + slot % F_RING, slot + 1);
+                        atomicAdd(ctrl + C_PUSHED, cn);
                     }
                     __syncwarp();
                 }
+                if (!pushed_ok) break;
             }
-            if (xt && stid == 0 && n == 3) xt[8] = globaltimer_ns();
-            mn0 = mn1; mn1 = mn2;
-            cur_next(cp);
+            if (xt && sw == 0 && lane == 0 && n_items == 3) xt[7] = globaltimer_ns();
+
+            have = nhave;
+            row = nrow; it0 = nit0; nit = nnit; pos = npos;
+            gc = gn;
+            mn_cur = mn_next;
+            te_cur = te_next;
+            te_have = te_next_have;
+            ++n_items;
+            if (n_items > (uint32_t)(a.rows * a.nfs)) { if (lane == 0) ctrl[C_FAIL] = 1; break; }     // cannot happen
         }
-        if (stid == 0) {
-            if (ctrl[C_FAIL]) {
+        if (lane == 0) {
+            if (ld_volatile(ctrl + C_FAIL)) {
                 if (a.status) atomicOr(a.status, ETA_DEV_TIMEOUT);
-                // copies already started must land before the CTA's shared memory can be released
-                for (int k = 0; k < F_NSB; ++k) mbar_wait(&sbar[k], 0);
+                mbar_wait(&sbar[sw], n_items & 1);      // a copy already started must land before the CTA can go
             }
             __threadfence_block();
-            st_volatile(ctrl + C_DONE, 1);
-            if (tl) tl[1] = globaltimer_ns();
+            atomicAdd(ctrl + C_DONE, 1);
+            if (tl && sw == 0) tl[1] = globaltimer_ns();
             if (pg) pg[1] = 0xffff;
         }
         return;
@@ -561,10 +509,11 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             bool skip = false;
             if (st->k >= st->n) {
                 // the lane needs a new chunk
-                const int done = ld_volatile(ctrl + C_DONE);       // read before the tail: a set flag means the tail is final
-                const int tail = ld_volatile(ctrl + C_TAIL);
-                if (head != tail) {
-                    __threadfence_block();             // the record was written before the tail moved
+                // read in this order: once every screening warp is done, the number of reserved slots is final
+                const bool done = ld_volatile(ctrl + C_DONE) == F_SCR_WARPS;
+                const int reserved = ld_volatile(ctrl + C_RESERVE);
+                if (ld_volatile(reinterpret_cast<int*>(smem + L::READY_OFF) + head % F_RING) == head + 1) {
+                    __threadfence_block();             // the record was written before its slot was marked ready
                     const ChunkRec* rec = &ring[head % F_RING];
                     const int qb = st->nchunks % NQB;
                     if (lane < FCH) lent[Lg * FCH + lane] = rec->ent[lane];
@@ -581,12 +530,12 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                     flags = FD_NEW | ((uint32_t)qb << 8);
                     idle = 0;
                 } else {
-                    if (done) done_mask |= 1 << Lg;
+                    if (done && head == reserved) done_mask |= 1 << Lg;
                     if (done_mask == (1 << F_GROUPS) - 1) break;
                     bool others = false;
 #pragma unroll
                     for (int k = 0; k < F_GROUPS; ++k) others = others || (k != Lg && lst[k].k < lst[k].n);
-                    if (!others && !done) {
+                    if (!others && !(done && head == reserved)) {
                         if (++idle > WAIT_LIMIT) { ok = false; if (tl && lane == 0) tl[6] = (3ull << 32) | fill; break; }
                         __nanosleep(100);
                         continue;
@@ -650,7 +599,7 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         pdl_trigger();
         if (pg && lane == 0) pg[2] = ((unsigned long long)fill << 8) | (ok ? 9 : 10);
         if (pg && lane == 0) pg[6] = ((unsigned long long)head << 32) | ((unsigned)done_mask << 16) | (unsigned)(idle & 0xffff);
-        if (pg && lane == 0) pg[7] = ((unsigned long long)ld_volatile(ctrl + C_TAIL) << 48) | ((unsigned long long)ld_volatile(ctrl + C_DONE) << 40) | ((unsigned long long)(ld_volatile(ctrl + C_PUSHED) & 0xfffff) << 20) | (unsigned)(ld_volatile(ctrl + C_ISSUED) & 0xfffff);
+        if (pg && lane == 0) pg[7] = ((unsigned long long)ld_volatile(ctrl + C_RESERVE) << 48) | ((unsigned long long)ld_volatile(ctrl + C_DONE) << 40) | ((unsigned long long)(ld_volatile(ctrl + C_PUSHED) & 0xfffff) << 20) | (unsigned)(ld_volatile(ctrl + C_ISSUED) & 0xfffff);
         // one end marker per group (no data): the next F_GROUPS fills reach every group exactly once
         for (int k = 0; k < F_GROUPS && ok; ++k) {
             const int stage = fill % NSTAGE;
@@ -710,6 +659,7 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     float o[HALVES][4][4];
     float m_run = -INFINITY, l_run = 0.f, te = 0.f;
     bool ok = true;
+    uint32_t flush_phase = 0;
 
     for (uint32_t fill = group;; fill += F_GROUPS) {
         const int stage = fill % NSTAGE;
@@ -727,7 +677,7 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 if ((uint32_t)ld_volatile(ctrl + C_FILL) > fill) { started = true; break; }
                 __nanosleep(40);
             }
-            if (!started) { ok = false; break; }
+            if (!started) { ok = false; if (tl && lane == 0 && wq == 0) tl[4] = (8ull << 32) | ((unsigned long long)group << 28) | fill; break; }
         }
         if (!mbar_wait(&full[stage], (fill / NSTAGE) & 1)) {
             if (pw && lane == 0) *pw = ((unsigned long long)fill << 8) | 2;
@@ -913,7 +863,9 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                     if (2 * t + 1 < G)
                         *reinterpret_cast<float2*>(stage_ptr + region_off(wq, (2 * t + 1) * D + dcol)) = make_float2(o[hf][mt][1], o[hf][mt][3]);
                 }
-            named_barrier(BAR_GROUP0 + group, 32 * F_WPG);
+            mbar_arrive(&flushbar[group]);
+            if (!mbar_wait(&flushbar[group], flush_phase)) { ok = false; if (tl && lane == 0) tl[4] = (6ull << 32) | fill; break; }
+            flush_phase ^= 1;
             if (pg && lane == 0 && wq == 0) pg[3 + group] = ((unsigned long long)fill << 8) | 8;
             const int64_t slot = ds.y;
             for (int idx = gtid; idx < G * D; idx += 32 * F_WPG) {
@@ -933,7 +885,9 @@ fused_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 a.part_o[(slot * G + hh) * D + dd] = acc;
                 if (dd == 0) a.part_ml[slot * G + hh] = make_float2(M, lacc);
             }
-            named_barrier(BAR_GROUP0 + group, 32 * F_WPG);
+            mbar_arrive(&flushbar[group]);
+            if (!mbar_wait(&flushbar[group], flush_phase)) { ok = false; if (tl && lane == 0) tl[4] = (7ull << 32) | fill; break; }
+            flush_phase ^= 1;
             fence_proxy_async();          // the scratch writes are ordered before the next copy into this stage
             if (lane == 0) mbar_arrive(&empty[stage]);
             if (pg && lane == 0 && wq == 0) pg[3 + group] = ((unsigned long long)fill << 8) | 9;
