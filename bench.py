@@ -192,9 +192,7 @@ def run_ours(args):
         into a CUDA graph and replayed, so the host costs one graph launch per step instead of six kernel launches
         through ctypes; the library calls are the same either way."""
         bias_d = torch.from_numpy(bias_np).to(dev)
-        path = {"auto": 0, "three": eb.ETA_FLAG_THREE_KERNELS, "single": eb.ETA_FLAG_SINGLE_KERNEL}[args.path]
-        params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window,
-                                 flags=flags if (flags & eb.ETA_FLAG_DENSE) else (flags | path),
+        params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags,
                                  ctas_per_sm=args.ctas_per_sm)
 
         def launch():
@@ -278,7 +276,6 @@ def run_ours(args):
     sampler.start()
     step_main = make_step(load_bias(sp.name, main_target))
     ms_main, wall_main = timed(step_main)
-    main_kernels = eb.eta_decode_kernel_count()
     ms_step = max_over_ranks(sum(ms_main) / len(ms_main), dist if world > 1 else None, dev)
     union_main = union_blocks_of(step_main)
     kt = kernel_times(load_bias(sp.name, main_target))
@@ -342,8 +339,7 @@ def run_ours(args):
                        "head_dim": sp.head_dim, "context": sp.context, "block_size": sp.block_size,
                        "target_union_sparsity": main_target, "measured_union_sparsity": 1 - union_main / nb_total,
                        "z": sp.z, "beta": sp.beta, "l2": "flushed between timed steps (384 MiB write)",
-                       "fresh_query_every_step": True, "replicas": world, "cuda_graph": bool(args.graph), "pdl": bool(args.pdl),
-                       "decode_kernels_per_call": eb.eta_decode_kernel_count()},
+                       "fresh_query_every_step": True, "replicas": world, "cuda_graph": bool(args.graph), "pdl": bool(args.pdl)},
             "attention_us_per_token": ms_step * 1e3,
             "achieved_gbs_all_kernels": ab["total"] / (ms_step * 1e-3) / 1e9,
             "frac_of_8tbs_nominal": ab["total"] / (ms_step * 1e-3) / 8e12,
@@ -351,7 +347,7 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": world * sp.batch / e2e_s, "unit": UNIT, "h2d_bytes_per_step": q_host[0].numel() * 2,
                     "d2h_bytes_per_step": out_host.numel() * 4},
-            "gpu_launches": args.steps * (2 + main_kernels),
+            "gpu_launches": args.steps * (2 + eb.eta_decode_kernel_count()),
             "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get((sp.name, main_target)), "traffic_unit": "bytes per launch",
@@ -434,8 +430,6 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch the kernels directly every step")
     ap.add_argument("--no-pdl", dest="pdl", action="store_false", help="fully serialise the kernel launches")
-    ap.add_argument("--path", default="auto", choices=["auto", "three", "single"],
-                    help="execution path of eta_decode: the library's choice, three kernels, or the single kernel")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--dry-run", action="store_true", help="exercise the multi-rank host logic on CPU (gloo)")

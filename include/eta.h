@@ -59,9 +59,6 @@ typedef enum eta_status {
 
 /* flags of eta_params.flags */
 #define ETA_FLAG_DENSE           1u  /* baseline: admit every block and switch the gate off (softmax attention) */
-#define ETA_FLAG_THREE_KERNELS   2u  /* run screening, streaming and merge as three kernels even where one would do */
-#define ETA_FLAG_SINGLE_KERNEL   4u  /* run the single screening+streaming kernel even on a small problem;
-                                        ETA_ERR_UNSUPPORTED where that path cannot run (see eta_decode) */
 /* flags of the summary builders */
 #define ETA_BUILD_SIGMA_ENVELOPE 1u  /* store the sub-block envelope (Eq. subblock_envelope_appx) instead of sigma */
 
@@ -85,22 +82,13 @@ typedef struct eta_params {
 } eta_params;
 
 /*
- * Bytes of scratch eta_decode wants for this cache shape (independent of the
+ * Bytes of scratch eta_decode needs for this cache shape (independent of the
  * sequence lengths).  The caller allocates it once, 256-byte aligned, and may
- * reuse it across calls on the same stream (calls that can overlap on the GPU
- * need a workspace each).  It needs no initialisation.  Between calls the library
- * keeps one thing in it: a claim counter guarded by a magic number, re-armed by
- * the last kernel of every call; a workspace without the magic number (first
- * use, or overwritten by the caller) is recognised and costs that one call its
- * dynamic load balance, nothing else.  Every other word is written before it is
- * read.  No device is touched by this function.
- *
- * eta_workspace_bytes_min is the smallest workspace eta_decode accepts: enough
- * for the three-kernel sequence, which keeps no state at all, and too small for
- * the single-kernel path (see eta_decode).
+ * reuse it across calls on the same stream; it carries no state between calls
+ * (every word is written before it is read) and needs no initialisation.
+ * No device is touched by this function.
  */
 int eta_workspace_bytes(const eta_cache_desc* desc, size_t* out_bytes);
-int eta_workspace_bytes_min(const eta_cache_desc* desc, size_t* out_bytes);
 
 /*
  * Section 3 (dual block index); appendix "End-to-end systems accounting"
@@ -166,22 +154,6 @@ int eta_score_dual(const eta_cache_desc* desc, const eta_params* params, const v
  * status_dev (nullable, uint32, caller-zeroed) device-side problems.
  * bf16 operands, fp32 scores / softmax statistics / accumulators; deterministic
  * for a given device and launch hint.  workspace: eta_workspace_bytes() bytes.
- *
- * Two execution paths give the same selection and, to rounding, the same output
- * (the paper has one fused kernel per chunk; neither split is the paper's):
- *   - a single persistent kernel that screens and streams side by side, followed
- *     by a merge kernel: CTAs claim runs of 32 block records from a counter, so
- *     the load balances itself, and every chunk of at most 8 surviving blocks
- *     leaves one partial that the merge adds in list order - the output does
- *     not depend on which CTA took which claim.  Used when the workspace has
- *     eta_workspace_bytes() bytes, the rescue window spans at most 256 blocks,
- *     nb_cap <= 32768, the group size is 1, 2, 4 (or 8 with head_dim 128 and
- *     block_size >= 64), batch * n_kv_heads fits its shared-memory tables (a
- *     few hundred rows) and the call has at least 4 claims per SM;
- *   - screening kernel, streaming kernel, merge kernel, with an exact split of
- *     the survivors over the streaming CTAs: everything else, ETA_FLAG_DENSE,
- *     and workspaces of eta_workspace_bytes_min() bytes.
- * ETA_FLAG_THREE_KERNELS / ETA_FLAG_SINGLE_KERNEL override the choice.
  */
 int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q,
                const void* K, const void* V, const int32_t* seq_lens,
@@ -200,9 +172,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
  * Same arguments, results and status codes as eta_decode, minus workspace / workspace_bytes.  The scratch is a
  * fixed array of ETA_STATIC_SCRATCH_BYTES (8 MiB) inside the library's CUDA module: every GPU that loads the
  * library holds it from load until the process exits.  The call allocates and frees nothing.
- *   - Limit: shapes for which eta_workspace_bytes_min() exceeds ETA_STATIC_SCRATCH_BYTES are refused with
+ *   - Limit: shapes for which eta_workspace_bytes() exceeds ETA_STATIC_SCRATCH_BYTES are refused with
  *     ETA_ERR_WORKSPACE before anything is launched (the five benchmark configurations need 0.8 - 3 MiB).
- *     The call always runs the three-kernel sequence of eta_decode.
  *   - Set-up: the first call on each device looks up the array's device address (with that device current).
  *     Make that first call ahead of any stream capture.
  *   - Sharing: all calls on a device use the same array, and it keeps the previous call's contents.  Nothing in
@@ -220,8 +191,7 @@ int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, cons
 /* Size of the built-in scratch of eta_decode_static, in bytes. */
 size_t eta_static_scratch_bytes(void);
 
-/* Number of kernels the most recent eta_decode call of this thread launched (3, or 2 on the single-kernel
- * path; 3 before any call), for launch accounting. */
+/* Number of kernels one eta_decode call launches (for launch accounting). */
 int eta_decode_kernel_count(void);
 
 /*
@@ -230,8 +200,7 @@ int eta_decode_kernel_count(void);
  * kernel launches on the call's stream (inside a stream capture they become nodes of the graph).
  * eta_profile_read waits for the most recent eta_decode to finish and writes the time from each launch to the
  * next, in milliseconds, to ms[0 .. count-1] (n >= 5), in the order append, predict, screen, decode, merge,
- * returning the count, or a negative status when no profiled eta_decode has run.  On the single-kernel path
- * "screen" is 0 and "decode" is the screening+streaming kernel.  The first two are 0
+ * returning the count, or a negative status when no profiled eta_decode has run.  The first two are 0
  * unless those calls were made, in that order, right before the eta_decode.  Not thread-safe; leave disabled
  * in production.
  */

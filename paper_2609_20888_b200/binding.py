@@ -16,12 +16,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libeta_b200.so")
 
 ETA_FLAG_DENSE = 1
-ETA_FLAG_THREE_KERNELS = 2
-ETA_FLAG_SINGLE_KERNEL = 4
 ETA_BUILD_SIGMA_ENVELOPE = 1
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
-EXPORTS = ("eta_workspace_bytes", "eta_workspace_bytes_min", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
+EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
            "eta_score_dual", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
            "eta_profile_kernel_name", "eta_set_pdl", "eta_debug_timeline", "eta_strerror", "eta_last_cuda_error")
 
@@ -41,7 +39,7 @@ class Params(ctypes.Structure):
 
 
 class EtaError(RuntimeError):
-    code = 0
+    pass
 
 
 _lib = None
@@ -58,7 +56,6 @@ def load() -> ctypes.CDLL:
         vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
         D, P = ctypes.POINTER(CacheDesc), ctypes.POINTER(Params)
         lib.eta_workspace_bytes.argtypes = [D, ctypes.POINTER(ctypes.c_size_t)]
-        lib.eta_workspace_bytes_min.argtypes = [D, ctypes.POINTER(ctypes.c_size_t)]
         lib.eta_build_block_summaries.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
         lib.eta_append_summary.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
         lib.eta_predict_threshold.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, f32p, f32p, f32p, vp]
@@ -88,9 +85,7 @@ def load() -> ctypes.CDLL:
 def _check(rc: int, what: str) -> None:
     if rc != 0:
         lib = load()
-        err = EtaError(f"{what}: {lib.eta_strerror(rc).decode()} ({rc}) {lib.eta_last_cuda_error().decode()}")
-        err.code = rc
-        raise err
+        raise EtaError(f"{what}: {lib.eta_strerror(rc).decode()} ({rc}) {lib.eta_last_cuda_error().decode()}")
 
 
 def _dev(t: torch.Tensor | None, dtype=None, name="tensor"):
@@ -137,12 +132,6 @@ def cache_desc(K: torch.Tensor, V: torch.Tensor, n_q_heads: int, block_size: int
 def eta_workspace_bytes(desc: CacheDesc) -> int:
     n = ctypes.c_size_t(0)
     _check(load().eta_workspace_bytes(ctypes.byref(desc), ctypes.byref(n)), "eta_workspace_bytes")
-    return n.value
-
-
-def eta_workspace_bytes_min(desc: CacheDesc) -> int:
-    n = ctypes.c_size_t(0)
-    _check(load().eta_workspace_bytes_min(ctypes.byref(desc), ctypes.byref(n)), "eta_workspace_bytes_min")
     return n.value
 
 

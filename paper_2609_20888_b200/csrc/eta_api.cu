@@ -83,18 +83,6 @@ WsLayout ws_layout(const eta_cache_desc* d) {
     L.part_ml = off;    off = align_up(off + sizeof(float2) * slots * G, 256);
     L.part_o = off;     off = align_up(off + sizeof(float) * slots * G * d->head_dim, 256);
     L.total = off;
-    // single-kernel path: per-item counts and per-chunk partials (skipped when they would be unreasonably large)
-    L.nfs = (d->nb_cap + FSEG - 1) / FSEG;
-    L.f_hdr = L.f_count = L.f_part_ml = L.f_part_o = 0;
-    L.total_fused = L.total;
-    const size_t fslots = (size_t)L.rows * L.nfs * FCPI;
-    if (L.nfs <= F_MAX_ITEMS_ROW && sizeof(float) * fslots * G * d->head_dim <= ((size_t)1 << 30)) {
-        L.f_hdr = off;      off = align_up(off + 4 * sizeof(int32_t), 256);
-        L.f_count = off;    off = align_up(off + sizeof(int32_t) * (size_t)L.rows * L.nfs, 256);
-        L.f_part_ml = off;  off = align_up(off + sizeof(float2) * fslots * G, 256);
-        L.f_part_o = off;   off = align_up(off + sizeof(float) * fslots * G * d->head_dim, 256);
-        L.total_fused = off;
-    }
     return L;
 }
 
@@ -103,14 +91,6 @@ WsLayout ws_layout(const eta_cache_desc* d) {
 extern "C" {
 
 int eta_workspace_bytes(const eta_cache_desc* desc, size_t* out_bytes) {
-    if (!out_bytes) return ETA_ERR_INVALID_ARG;
-    int rc = eta::validate_desc(desc);
-    if (rc != ETA_OK) return rc;
-    *out_bytes = eta::ws_layout(desc).total_fused;
-    return ETA_OK;
-}
-
-int eta_workspace_bytes_min(const eta_cache_desc* desc, size_t* out_bytes) {
     if (!out_bytes) return ETA_ERR_INVALID_ARG;
     int rc = eta::validate_desc(desc);
     if (rc != ETA_OK) return rc;

@@ -34,17 +34,6 @@ constexpr int MAX_CTAS = 256;        // upper bound on streaming CTAs (sizes the
 constexpr int MAX_ROWS = 1024;        // rows (batch * n_kv_heads) whose unit prefix a streaming CTA keeps in shared memory
 constexpr int DECODE_GROUPS = 3;     // consumer groups per streaming CTA, each with its own partial per piece
 
-// The single-kernel path (eta_fused.cu) screens items of FSEG block records and streams their survivors in
-// chunks of at most FCH list entries; a chunk yields one partial (m, l, O) per query head, stored in slot
-// item * FCPI + chunk.  An item's list holds its FSEG records' survivors, then up to 8 rescued blocks, then the
-// row's tail.
-constexpr int FSEG = 32;
-constexpr int FCH = 8;
-constexpr int FCPI = (FSEG + 8 + 1 + FCH - 1) / FCH;
-constexpr int F_MAXWIN = 8;          // items the rescue window of a row may span on this path
-constexpr int F_MAX_ITEMS_ROW = 1024;  // items per row the merge of this path tabulates in shared memory
-constexpr uint32_t F_MAGIC0 = 0x45544146u, F_MAGIC1 = 0x5a9c3be1u;
-
 // Scratch layout (byte offsets from a 256-byte aligned base).
 struct WsLayout {
     int rows;        // batch * n_kv_heads
@@ -60,24 +49,9 @@ struct WsLayout {
     size_t tau_eff;     // float [batch * n_q_heads]
     size_t part_ml;     // float2 [(MAX_CTAS + rows) * DECODE_GROUPS * G]
     size_t part_o;      // float [(MAX_CTAS + rows) * DECODE_GROUPS * G * d]
-    size_t total;       // bytes of everything above: what the three-kernel path needs
-    // single-kernel path (0 / absent when the shape is not eligible: total_fused == total)
-    int nfs;            // items per row
-    size_t f_hdr;       // int32[4]: magic (2 words), claim counter, pad - the only words that outlive a call
-    size_t f_count;     // int32 [rows * nfs]: list length | blocks fetched << 8
-    size_t f_part_ml;   // float2 [rows * nfs * FCPI * G]
-    size_t f_part_o;    // float [rows * nfs * FCPI * G * d]
-    size_t total_fused;
+    size_t total;
 };
 WsLayout ws_layout(const eta_cache_desc* d);
-
-// Single-kernel path (eta_fused.cu).
-bool fused_eligible(const eta_cache_desc* d, const eta_params* p, const WsLayout& L, size_t workspace_bytes);
-int fused_claims(const eta_cache_desc* d, const eta_params* p, const WsLayout& L);
-int launch_fused_decode(const eta_cache_desc* desc, const eta_params* params, const WsLayout& L, const void* q,
-                        const void* K, const void* V, const int32_t* seq_lens, const void* musig, const float* mnorm,
-                        const float* tau, const float* head_const, float* out, uint8_t* sel_mask, int32_t* stats,
-                        uint32_t* status_dev, unsigned char* ws, int n_ctas, cudaStream_t s);
 
 struct RescueRec { int cnt; float maxb; int arg; int pad; };
 
@@ -239,25 +213,6 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     return t;
 }
 
-__device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
-    return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
-}
-// token row inside an 8-row group that MMA column n reads: bits 0 and 2 of n swapped, so that the two
-// rows a quarter-warp touches in one 16-byte load sit in different halves of the swizzle pattern
-__device__ __forceinline__ int rho(int n) { return (n & 2) | ((n & 1) << 2) | ((n >> 2) & 1); }
-__device__ __forceinline__ float rcp_approx(float x) {
-    float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-// min that keeps a NaN (so that "not below the threshold" admits the block)
-__device__ __forceinline__ float min_keep_nan(float g, float s) {
-    return (g < s) ? g : ((s < g) ? s : ((g != g) ? g : s));
-}
-// barrier among `count` threads of the CTA (ids 1..15; 0 is __syncthreads)
-__device__ __forceinline__ void named_barrier(int id, int count) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
 __device__ __forceinline__ int ld_volatile(const int* p) { return *reinterpret_cast<const volatile int*>(p); }
 __device__ __forceinline__ void st_volatile(int* p, int v) { *reinterpret_cast<volatile int*>(p) = v; }
 

@@ -53,6 +53,18 @@ constexpr int PIECE_COST = 3;          // tiles a row boundary inside a CTA's ra
 constexpr int RESC_ROWS = 8;           // rows (from the CTA's first) whose rescue decisions stay in shared memory
 constexpr int PW = 256;                // entries of the unit prefix the producer keeps in shared memory
 
+__device__ __forceinline__ uint32_t u4_get(const uint4& v, int i) {
+    return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
+}
+// token row inside an 8-row group that MMA column n reads: bits 0 and 2 of n swapped, so that the two
+// rows a quarter-warp touches in one 16-byte load sit in different halves of the swizzle pattern
+__device__ __forceinline__ int rho(int n) { return (n & 2) | ((n & 1) << 2) | ((n >> 2) & 1); }
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 
 // Top-1 rescue of query head g of row r (Algorithm 3, rescue phase): if none of the first
 // Wr = min(rescue_window, NB) blocks was admitted for the head, the first block with the largest bound among them
@@ -965,7 +977,7 @@ static EncodeTiledFn encode_fn() {
 
 // K or V as a 5-D tensor (c within a 64-column half, t, half, hk, i) of bf16; a box is 64 columns x TS tokens x
 // all halves: in shared memory, one 128-byte-swizzled [TS][64] tile per half, back to back.
-int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d, int64_t sb, int64_t sh, int64_t st,
+static int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d, int64_t sb, int64_t sh, int64_t st,
                      int TS) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return ETA_ERR_CUDA;
@@ -1005,10 +1017,7 @@ static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const
 
 extern "C" {
 
-static thread_local int g_last_kernel_count = 3;
-// Whether eta_decode picks the single-kernel path by itself where it applies (it is always available on request).
-static bool fused_default() { return false; }
-int eta_decode_kernel_count(void) { return g_last_kernel_count; }
+int eta_decode_kernel_count(void) { return 3; }
 
 int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q, const void* K, const void* V,
                const int32_t* seq_lens, const void* musig, const float* mnorm, const float* tau,
@@ -1028,7 +1037,6 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     const WsLayout L = ws_layout(desc);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < L.total)
         return ETA_ERR_WORKSPACE;
-    if ((params->flags & ETA_FLAG_THREE_KERNELS) && (params->flags & ETA_FLAG_SINGLE_KERNEL)) return ETA_ERR_INVALID_ARG;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -1043,19 +1051,6 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     const int TS = b < 64 ? b : 64;
     int n_ctas = n_sm;                  // one persistent CTA per SM; the shared-memory ring fills the SM
     if (n_ctas > MAX_CTAS) n_ctas = MAX_CTAS;
-
-    // Two ways to run the call.  The single kernel overlaps screening with streaming and wins whenever there
-    // are enough claims to keep every CTA busy; the three-kernel sequence lays the survivors out exactly and
-    // serves small problems, the dense baseline, wide rescue windows and workspaces of the minimum size.
-    const bool can_fuse = !dense && !(params->flags & ETA_FLAG_THREE_KERNELS) &&
-                          fused_eligible(desc, params, L, workspace_bytes);
-    if ((params->flags & ETA_FLAG_SINGLE_KERNEL) && !can_fuse) return ETA_ERR_UNSUPPORTED;
-    if (can_fuse && ((params->flags & ETA_FLAG_SINGLE_KERNEL) || (fused_default() && fused_claims(desc, params, L) >= 4 * n_ctas))) {
-        g_last_kernel_count = 2;
-        return launch_fused_decode(desc, params, L, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,
-                                   stats, status_dev, ws, n_ctas, s);
-    }
-    g_last_kernel_count = 3;
 
     ScreenArgs sa;
     sa.q = static_cast<const __nv_bfloat16*>(q);

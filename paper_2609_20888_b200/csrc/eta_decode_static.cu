@@ -54,7 +54,7 @@ int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, cons
                       const float* tau, const float* head_const, float* out, uint8_t* sel_mask, int32_t* stats,
                       uint32_t* status_dev, void* stream) {
     size_t need = 0;
-    int rc = eta_workspace_bytes_min(desc, &need);
+    int rc = eta_workspace_bytes(desc, &need);
     if (rc != ETA_OK) return rc;
     if (need > eta::STATIC_SCRATCH_BYTES) return ETA_ERR_WORKSPACE;   // shape needs more scratch than is built in
     void* scratch = nullptr;
@@ -63,10 +63,7 @@ int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, cons
     // every word of the scratch that a kernel reads is written earlier in the same call (counts, lists and window
     // statistics by the screening kernel, partial slots by the streaming kernel), so nothing carried over from
     // the previous call is ever consumed
-    if (!params) return ETA_ERR_INVALID_ARG;
-    eta_params p3 = *params;
-    p3.flags = (p3.flags & ~ETA_FLAG_SINGLE_KERNEL) | ETA_FLAG_THREE_KERNELS;   // the path that keeps no state in its scratch
-    return eta_decode(desc, &p3, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask, stats,
+    return eta_decode(desc, params, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask, stats,
                       status_dev, scratch, eta::STATIC_SCRATCH_BYTES, stream);
 }
 

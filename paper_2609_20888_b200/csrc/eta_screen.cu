@@ -21,6 +21,11 @@
 
 namespace eta {
 
+// min that keeps a NaN (so that "not below the threshold" admits the block)
+__device__ __forceinline__ float min_keep_nan(float g, float s) {
+    return (g < s) ? g : ((s < g) ? s : ((g != g) ? g : s));
+}
+
 template <int D, int G>
 struct ScreenSmem {
     static constexpr int REC_BYTES = 4 * D;                    // fp16 mu[d] + fp16 sigma[d]

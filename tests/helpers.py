@@ -108,27 +108,6 @@ def calibrate_head_const(bound, seq_lens, b, sparsity_levels):
 # GPU side (used by the -m gpu tests only)
 # --------------------------------------------------------------------------
 
-# Which of eta_decode's two execution paths the decode tests force (set by the `decode_path` fixture of the GPU
-# test modules): 0 = the library's own choice, else ETA_FLAG_THREE_KERNELS / ETA_FLAG_SINGLE_KERNEL.
-DECODE_PATH = {"flags": 0}
-
-
-def path_flags(flags: int) -> int:
-    """Add the forced path to a call's flags (the dense baseline always runs as three kernels)."""
-    return flags if (flags & 1) else (flags | DECODE_PATH["flags"])
-
-
-def decode_or_skip(eb, *args, **kw):
-    """eta_decode; a shape the forced single-kernel path cannot run skips the test instead of failing it."""
-    import pytest
-    try:
-        return eb.eta_decode(*args, **kw)
-    except eb.EtaError as e:
-        if e.code == -2 and (DECODE_PATH["flags"] & 4):
-            pytest.skip("single-kernel path does not cover this shape")
-        raise
-
-
 def gpu_decode(q_t, K_t, V_t, seq_lens, block_size, musig_bits, mnorm, tau=None, head_const=None, **params):
     """Run eta_decode on cuda:0 with the given (oracle-built) summaries.
 
@@ -144,12 +123,10 @@ def gpu_decode(q_t, K_t, V_t, seq_lens, block_size, musig_bits, mnorm, tau=None,
     lens = torch.from_numpy(np.asarray(seq_lens, np.int32)).to(dev)
     tau_d = None if tau is None else torch.from_numpy(np.ascontiguousarray(tau, np.float32)).to(dev)
     hc_d = None if head_const is None else torch.from_numpy(np.ascontiguousarray(head_const, np.float32)).to(dev)
-    params = dict(params)
-    params["flags"] = path_flags(params.get("flags", 0))
     p = eb.DecodeParams(**params)
     st.out.fill_(float("nan"))
-    decode_or_skip(eb, st.desc, p, q, K, V, lens, st.musig, st.mnorm, tau_d, hc_d, st.out, st.sel_mask,
-                   st.workspace, stats=st.stats, status=st.status)
+    eb.eta_decode(st.desc, p, q, K, V, lens, st.musig, st.mnorm, tau_d, hc_d, st.out, st.sel_mask, st.workspace,
+                  stats=st.stats, status=st.status)
     torch.cuda.synchronize()
     return st.out.cpu().numpy(), st.sel_mask.cpu().numpy(), st.stats.cpu().numpy(), int(st.status.item())
 

@@ -14,19 +14,9 @@ import torch
 
 from oracle import eta_oracle as orc
 from paper_2609_20888_b200 import workloads as wl
-from tests.helpers import (bits, cache_of, compare_masks, decode_or_skip, fp16_ulp_distance, output_errors,
-                           path_flags)
+from tests.helpers import bits, cache_of, compare_masks, fp16_ulp_distance, output_errors
 
 pytestmark = pytest.mark.gpu
-
-
-@pytest.fixture(autouse=True, params=["three_kernels", "single_kernel"])
-def decode_path(request):
-    """Every test of this module runs once per execution path of eta_decode."""
-    from tests import helpers
-    helpers.DECODE_PATH["flags"] = 2 if request.param == "three_kernels" else 4
-    yield request.param
-    helpers.DECODE_PATH["flags"] = 0
 
 MAX_ABS, MEAN_ABS = 1e-2, 1e-3
 CALIB = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "workload_calibration.json")))
@@ -98,13 +88,12 @@ class Session:
                               lwb=sp.lwb, rescue_window=sp.rescue_window)
         st.musig.copy_(torch.from_numpy(musig.view(np.int16)).view(torch.float16).to(self.dev))
         st.mnorm.copy_(torch.from_numpy(mnorm).to(self.dev))
-        p = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window,
-                            flags=path_flags(flags))
+        p = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags)
         st.out.fill_(float("nan"))
-        decode_or_skip(eb, st.desc, p, q.to(self.dev), self.Kd, self.Vd, self.lens_d, st.musig, st.mnorm,
-                       None if tau is None else torch.from_numpy(tau).to(self.dev),
-                       None if head_const is None else torch.from_numpy(head_const).to(self.dev),
-                       st.out, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+        eb.eta_decode(st.desc, p, q.to(self.dev), self.Kd, self.Vd, self.lens_d, st.musig, st.mnorm,
+                      None if tau is None else torch.from_numpy(tau).to(self.dev),
+                      None if head_const is None else torch.from_numpy(head_const).to(self.dev),
+                      st.out, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
         torch.cuda.synchronize()
         assert int(st.status.item()) == 0
         out, sel = st.out.cpu().numpy(), st.sel_mask.cpu().numpy()

@@ -17,19 +17,10 @@ import torch
 
 from oracle import eta_oracle as orc
 from paper_2609_20888_b200 import workloads as wl
-from tests.helpers import (bits, cache_of, calibrate_bias, calibrate_head_const, compare_masks, decode_or_skip,
-                           fp16_ulp_distance, gpu_decode, output_errors, path_flags)
+from tests.helpers import (bits, cache_of, calibrate_bias, calibrate_head_const, compare_masks, fp16_ulp_distance,
+                           gpu_decode, output_errors)
 
 pytestmark = pytest.mark.gpu
-
-
-@pytest.fixture(autouse=True, params=["three_kernels", "single_kernel"])
-def decode_path(request):
-    """Every test of this module runs once per execution path of eta_decode."""
-    from tests import helpers
-    helpers.DECODE_PATH["flags"] = 2 if request.param == "three_kernels" else 4
-    yield request.param
-    helpers.DECODE_PATH["flags"] = 0
 
 MAX_ABS, MEAN_ABS = 1e-2, 1e-3
 
@@ -357,8 +348,8 @@ def test_strided_cache_layout_bthd():
         assert fp16_ulp_distance(got[i, :, :NBs[i]], musig[i, :, :NBs[i]]).max() <= 1
     st.musig.copy_(torch.from_numpy(musig.view(np.int16)).view(torch.float16).to(dev))
     st.mnorm.copy_(torch.from_numpy(mnorm).to(dev))
-    decode_or_skip(eb, st.desc, eb.DecodeParams(flags=path_flags(0)), q.to(dev), Kd, Vd, lens_d, st.musig, st.mnorm,
-                   torch.from_numpy(tau).to(dev), None, st.out, st.sel_mask, st.workspace, status=st.status)
+    eb.eta_decode(st.desc, eb.DecodeParams(), q.to(dev), Kd, Vd, lens_d, st.musig, st.mnorm,
+                  torch.from_numpy(tau).to(dev), None, st.out, st.sel_mask, st.workspace, status=st.status)
     torch.cuda.synchronize()
     assert int(st.status.item()) == 0
     near = compare_masks(st.sel_mask.cpu().numpy(), ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G,
@@ -401,8 +392,8 @@ def test_chained_gpu_path_and_multi_step_append():
         q = w.queries(step)
         qd = q.to(dev)
         eb.eta_predict_threshold(qd, Wd, bias_d, st.tau)
-        decode_or_skip(eb, st.desc, eb.DecodeParams(z=sp.z, beta=sp.beta, flags=path_flags(0)), qd, Kd, Vd, lens_d,
-                       st.musig, st.mnorm, st.tau, None, st.out, st.sel_mask, st.workspace, status=st.status)
+        eb.eta_decode(st.desc, eb.DecodeParams(z=sp.z, beta=sp.beta), qd, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau,
+                      None, st.out, st.sel_mask, st.workspace, status=st.status)
         torch.cuda.synchronize()
         assert int(st.status.item()) == 0
         c = orc.Cache(bits(K), bits(V), lens.copy(), sp.block_size)

@@ -29,7 +29,7 @@ def test_static_scratch_variant_matches_eta_decode_twice_in_a_row():
     st = eb.DecodeState(Kd, Vd, sp.n_q_heads, sp.block_size)
     lens_d = w.seq_lens.to(dev)
     eb.eta_build_block_summaries(st.desc, Kd, lens_d, st.musig, st.mnorm)
-    assert eb.eta_workspace_bytes_min(st.desc) <= eb.eta_static_scratch_bytes() == 8 << 20
+    assert eb.eta_workspace_bytes(st.desc) <= eb.eta_static_scratch_bytes() == 8 << 20
 
     out2 = torch.empty_like(st.out)
     sel2 = torch.empty_like(st.sel_mask)
@@ -61,7 +61,7 @@ def test_static_scratch_variant_refuses_shapes_beyond_its_limit():
     # 64 sequences x 8 KV heads x 512K tokens: needs far more than 8 MiB of scratch; refused before any launch
     T = 512 * 1024
     d = eb.CacheDesc(64, 32, 8, 128, 64, T, T // 64, 8 * T * 128, T * 128, 128, 8 * T * 128, T * 128, 128)
-    assert eb.eta_workspace_bytes_min(d) > eb.eta_static_scratch_bytes()
+    assert eb.eta_workspace_bytes(d) > eb.eta_static_scratch_bytes()
     p = eb.DecodeParams().c()
     one, null = ctypes.c_void_p(256), ctypes.c_void_p(None)
     rc = lib.eta_decode_static(ctypes.byref(d), ctypes.byref(p), one, one, one, one, one, one, one, null, one, one,
