@@ -275,13 +275,17 @@ void eta_oracle_score_dual(
  *   if none of the first Wr = min(rescue_window, NB) blocks is admitted, the
  *   first index attaining the largest bound among them is admitted
  *   (strict ">" update while scanning upwards).
+ * ungate_last (the diagonal case of Eq. mult_attn, M_ts = 1 for s = t, carried
+ * over to decoding, where the query's own token is the newest one): when the
+ * newest token closes a full block (T mod b == 0) that block is admitted for
+ * every head, since an ungated token must be attended.
  * sel[i,hk,j] gets bit g = h - hk*G set for every admitting head.
  * rescued[i,h] (nullable) is set to the rescued index or -1.
  */
 void eta_oracle_select(
     const double* bound, const float* tau, const float* head_const,
     int B, int Hq, int Hkv, int b, int NBcap, const int32_t* seq_lens,
-    double a, int lwb, int rescue_window,
+    double a, int lwb, int rescue_window, int ungate_last,
     uint8_t* sel, int32_t* rescued)
 {
     int G = Hq / Hkv;
@@ -302,6 +306,7 @@ void eta_oracle_select(
             for (int j = 0; j < NB; ++j) {
                 int admit = !(bd[j] < tau_eff);
                 if (j >= NB - lwb) admit = 1;
+                if (ungate_last && seq_lens[i] > 0 && seq_lens[i] % b == 0 && j == seq_lens[i] / b - 1) admit = 1;
                 if (admit) {
                     row[j] |= (uint8_t)(1u << g);
                     if (j < Wr) attended_in_window += 1;
@@ -349,6 +354,10 @@ double eta_oracle_gate(double S, double tau_eff, double beta) {
  * Z (nullable, [B,Hq]) receives log(sum_s w_s); n_tok (nullable) the number
  * of attended tokens.  A head never attends a block fetched only for a
  * sibling head of its GQA group.
+ * ungate_last: the newest token s = T_i - 1 (the query's own position) keeps
+ * its raw logit, S~ = S (Eq. mult_attn, M_ts = 1 for s = t; the "restore token
+ * diagonal" line of Algorithm 2).  Off, every token is gated (Algorithm 3 as
+ * printed).
  */
 void eta_oracle_gated_block_attention(
     const uint16_t* q,
@@ -356,7 +365,7 @@ void eta_oracle_gated_block_attention(
     const uint16_t* V, int64_t v_stride_b, int64_t v_stride_h, int64_t v_stride_t,
     const uint8_t* sel, const float* tau, const float* head_const,
     int B, int Hq, int Hkv, int d, int b, int NBcap, const int32_t* seq_lens,
-    double a, double beta, double s,
+    double a, double beta, double s, int ungate_last,
     double* out, double* logZ, int64_t* n_tok)
 {
     int G = Hq / Hkv;
@@ -385,6 +394,7 @@ void eta_oracle_gated_block_attention(
                 for (int c = 0; c < d; ++c)
                     dot += eta_oracle_bf16_to_double(qv[c]) * eta_oracle_bf16_to_double(Kh[p * k_stride_t + c]);
                 double Sg = eta_oracle_gate(s * dot, tau_eff, beta);
+                if (ungate_last && p == T - 1) Sg = s * dot;
                 St[p] = Sg;
                 if (Sg > mx) mx = Sg;
                 cnt += 1;

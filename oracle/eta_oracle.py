@@ -156,7 +156,8 @@ def score_dual(q, musig, mnorm, seq_lens, block_size, z, scale=None, parts=False
     return bound
 
 
-def select(bound, seq_lens, block_size, Hkv, tau=None, head_const=None, a=0.0, lwb=0, rescue_window=128):
+def select(bound, seq_lens, block_size, Hkv, tau=None, head_const=None, a=0.0, lwb=0, rescue_window=128,
+           ungate_last=False):
     """-> sel uint8 [B,Hkv,NBcap] (bit g = query head hk*G+g), rescued int32 [B,Hq]."""
     B, Hq, NBcap = bound.shape
     assert (tau is None) != (head_const is None)
@@ -166,13 +167,13 @@ def select(bound, seq_lens, block_size, Hkv, tau=None, head_const=None, a=0.0, l
     hc32 = None if head_const is None else np.ascontiguousarray(head_const, np.float32)
     lib().eta_oracle_select(
         _p(np.ascontiguousarray(bound), _f64), _p(tau32, _f32), _p(hc32, _f32), _I(B), _I(Hq), _I(Hkv),
-        _I(block_size), _I(NBcap), _p(seq_lens, _i32), _D(a), _I(lwb), _I(rescue_window), _p(sel, _u8),
-        _p(rescued, _i32))
+        _I(block_size), _I(NBcap), _p(seq_lens, _i32), _D(a), _I(lwb), _I(rescue_window), _I(int(ungate_last)),
+        _p(sel, _u8), _p(rescued, _i32))
     return sel, rescued
 
 
 def gated_block_attention(q, cache: Cache, sel, tau=None, head_const=None, a=0.0, beta=5.0, scale=None,
-                          extras=False):
+                          extras=False, ungate_last=False):
     """-> out float64 [B,Hq,d] (+ logZ [B,Hq], n_tok [B,Hq] when extras)."""
     B, Hq, d = q.shape
     s = (1.0 / np.sqrt(d)) if scale is None else scale
@@ -188,7 +189,7 @@ def gated_block_attention(q, cache: Cache, sel, tau=None, head_const=None, a=0.0
         _p(cache.V, _u16), _L(vs[0]), _L(vs[1]), _L(vs[2]),
         _p(np.ascontiguousarray(sel), _u8), _p(tau32, _f32), _p(hc32, _f32),
         _I(B), _I(Hq), _I(cache.Hkv), _I(d), _I(cache.block_size), _I(cache.NBcap), _p(cache.seq_lens, _i32),
-        _D(a), _D(beta), _D(s), _p(out, _f64), _p(logZ, _f64), _p(ntok, _i64))
+        _D(a), _D(beta), _D(s), _I(int(ungate_last)), _p(out, _f64), _p(logZ, _f64), _p(ntok, _i64))
     if extras:
         return out, logZ, ntok
     return out
@@ -219,13 +220,14 @@ def block_max_logit(q, cache: Cache, scale=None):
 
 
 def decode_step(q, cache: Cache, musig, mnorm, tau=None, head_const=None, z=1.0, a=0.0, beta=5.0, lwb=0,
-                rescue_window=128, scale=None):
+                rescue_window=128, scale=None, ungate_last=False):
     """The whole inference rule in the paper's order: bound -> select -> attend.
 
     -> dict(out, sel, bound, rescued).  `tau` / `head_const` are float32 inputs.
     """
     bound = score_dual(q, musig, mnorm, cache.seq_lens, cache.block_size, z, scale)
     sel, rescued = select(bound, cache.seq_lens, cache.block_size, cache.Hkv, tau=tau, head_const=head_const,
-                          a=a, lwb=lwb, rescue_window=rescue_window)
-    out = gated_block_attention(q, cache, sel, tau=tau, head_const=head_const, a=a, beta=beta, scale=scale)
+                          a=a, lwb=lwb, rescue_window=rescue_window, ungate_last=ungate_last)
+    out = gated_block_attention(q, cache, sel, tau=tau, head_const=head_const, a=a, beta=beta, scale=scale,
+                                ungate_last=ungate_last)
     return {"out": out, "sel": sel, "bound": bound, "rescued": rescued}

@@ -526,3 +526,44 @@ def test_decode_step_composes_the_three_stages():
     sel, _ = orc.select(bound, c.seq_lens, 16, 2, tau=tau, lwb=2, rescue_window=8)
     assert np.array_equal(res["sel"], sel)
     np.testing.assert_array_equal(res["out"], orc.gated_block_attention(q, c, sel, tau=tau))
+
+
+def test_ungated_newest_token_closed_forms():
+    """Eq. mult_attn leaves the diagonal s = t ungated; at decode time that is the newest token."""
+    _, c, q = _attn_case(seed=21)
+    B, Hq, d, T = 2, 4, 16, int(c.seq_lens[0])
+    Kv, Vv, qv = bf16_values(c.K), bf16_values(c.V), bf16_values(q)
+    full = np.full((B, 2, c.NBcap), 0b11, np.uint8)
+    # tau = -inf: every gate is open already, the flag changes nothing (textbook softmax either way)
+    a0 = orc.gated_block_attention(q, c, full, tau=np.full((B, Hq), -np.inf), ungate_last=False)
+    a1 = orc.gated_block_attention(q, c, full, tau=np.full((B, Hq), -np.inf), ungate_last=True)
+    np.testing.assert_array_equal(a0, a1)
+    # tau = +inf: every gated logit is 0 (weight 1); the newest token keeps its raw logit S, so
+    #   out = (sum of the other values + e^S v_last) / (T - 1 + e^S)
+    out = orc.gated_block_attention(q, c, full, tau=np.full((B, Hq), np.inf), ungate_last=True)
+    for i in range(B):
+        for h in range(Hq):
+            S = (qv[i, h] @ Kv[i, h // 2, T - 1]) / math.sqrt(d)
+            num = Vv[i, h // 2, :T - 1].sum(axis=0) + math.exp(S) * Vv[i, h // 2, T - 1]
+            np.testing.assert_allclose(out[i, h], num / (T - 1 + math.exp(S)), rtol=1e-12, atol=1e-14)
+    # beta = 0: the others sit at half scale, the newest token at full scale
+    out = orc.gated_block_attention(q, c, full, tau=np.full((B, Hq), 0.3), beta=0.0, ungate_last=True)
+    for i in range(B):
+        for h in range(Hq):
+            S = (Kv[i, h // 2, :T] @ qv[i, h]) / math.sqrt(d)
+            w = np.exp(np.concatenate([0.5 * S[:-1], S[-1:]]))
+            np.testing.assert_allclose(out[i, h], (w[:, None] * Vv[i, h // 2, :T]).sum(0) / w.sum(), rtol=1e-11, atol=1e-13)
+
+
+def test_ungated_newest_token_forces_its_block_when_it_closes_one():
+    rng = np.random.default_rng(5)
+    B, Hq, Hkv, b, NB = 2, 4, 2, 16, 6
+    bound = rng.standard_normal((B, Hq, NB))
+    tau = np.full((B, Hq), 10.0, np.float32)                 # nothing passes the screen
+    lens = np.array([NB * b, NB * b - 3], np.int32)          # sequence 0 ends on a block boundary, sequence 1 in a tail
+    sel0, _ = orc.select(bound, lens, b, Hkv, tau=tau, rescue_window=2)
+    sel1, _ = orc.select(bound, lens, b, Hkv, tau=tau, rescue_window=2, ungate_last=True)
+    assert np.all(sel1[0, :, NB - 1] == 0b11)                # the block holding token T-1, for every head
+    sel1_rest = sel1.copy(); sel1_rest[0, :, NB - 1] = sel0[0, :, NB - 1]
+    np.testing.assert_array_equal(sel1_rest, sel0)           # nothing else changes
+    np.testing.assert_array_equal(sel1[1], sel0[1])          # newest token in the tail: already attended
