@@ -59,6 +59,10 @@ typedef enum eta_status {
 
 /* flags of eta_params.flags */
 #define ETA_FLAG_DENSE           1u  /* baseline: admit every block and switch the gate off (softmax attention) */
+#define ETA_FLAG_UNGATE_LAST     2u  /* Eq. mult_attn leaves the diagonal s = t ungated; at decode time the query's own
+                                        token is the newest one: it keeps its raw logit (S~ = S), and when it closes a
+                                        full block that block is admitted for every head.  Off: Algorithm 3 as
+                                        printed, every token gated */
 /* flags of the summary builders */
 #define ETA_BUILD_SIGMA_ENVELOPE 1u  /* store the sub-block envelope (Eq. subblock_envelope_appx) instead of sigma */
 

@@ -16,6 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libeta_b200.so")
 
 ETA_FLAG_DENSE = 1
+ETA_FLAG_UNGATE_LAST = 2
 ETA_BUILD_SIGMA_ENVELOPE = 1
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 

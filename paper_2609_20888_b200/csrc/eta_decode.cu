@@ -43,6 +43,7 @@ struct DecodeArgs {
     uint32_t* status;
     float beta, scale;
     int Hq, Hkv, G, b, t_cap, nb_cap, nseg, entries, rows, rescue_window;
+    int ungate_last;     // the newest token of every sequence keeps its raw logit (ETA_FLAG_UNGATE_LAST)
     FastDiv div_nseg, div_epr, div_hkv, div_g;
     unsigned long long* timeline;
 };
@@ -483,10 +484,16 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     } else {
                         ent = NB | (0xff << 24);           // the tail: every head attends it
                         nrows = T - NB * a.b;
+                        if (a.ungate_last) nrows |= 0x10000;      // its last token is the sequence's newest
                     }
                 } else {
                     ent = __ldg(a.seg_list + ((int64_t)r * a.nseg + sg) * LSTRIDE + (uu - pwin[k]));
                     nrows = a.b;
+                    if (a.ungate_last) {
+                        int T = __ldg(a.seq_lens + a.div_hkv.div(r));
+                        T = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
+                        if (((ent & 0xffffff) + 1) * a.b == T) nrows |= 0x10000;   // the block the newest token closes
+                    }
                 }
             }
         };
@@ -508,7 +515,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             for (int k = 0; k < nb && ok; ++k) {
                 const int r = __shfl_sync(0xffffffffu, c_row, k);
                 const int ent = __shfl_sync(0xffffffffu, c_ent, k);
-                const int nrows = __shfl_sync(0xffffffffu, c_nrows, k);
+                const int nrows_raw = __shfl_sync(0xffffffffu, c_nrows, k);
+                const int nrows = nrows_raw & 0xffff;
+                const bool holds_newest = (nrows_raw >> 16) != 0;
                 const int j = ent & 0xffffff;
                 const int hmask = (ent >> 24) & 0xff;
                 int i, hk;
@@ -527,7 +536,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                             ok = false;
                         } else {
                             if (SHARED_STAGES) st_volatile(&s_fill_started, (int)fill + 1);
-                            desc[stage] = make_int4(r, piece << 1, hmask, nvalid);
+                            // bits 8..15: row of the tile whose token stays ungated, 0xff: none
+                            const int urow = (holds_newest && (sub + 1) * TS >= nrows) ? nvalid - 1 : 0xff;
+                            desc[stage] = make_int4(r, piece << 1, hmask | (urow << 8), nvalid);
                             unsigned char* st = smem + stage * L::STAGE_BYTES;
                             mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
                             const int y = j * a.b + sub * TS;
@@ -692,7 +703,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             break;
         }
 
-        const int hmask = ds.z, nvalid = ds.w;
+        const int hmask = ds.z & 0xff, urow = (ds.z >> 8) & 0xff, nvalid = ds.w;
         const uint32_t kbase = smem_u32(smem + stage * L::STAGE_BYTES);
         const uint32_t vbase = kbase + HALVES * L::TILE_BYTES;
 
@@ -759,6 +770,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     const float x = (a.beta == 0.f) ? 0.f : a.beta * (S - te);
                     gated = S * rcp_approx(1.f + exp2f(-x * LOG2E));      // S * sigmoid(x); exp2(+inf) -> rcp -> 0
                 }
+                if (trow == urow) gated = S;          // the query's own token (Eq. mult_attn, s = t)
                 gated = (head_on && trow < nvalid) ? gated : -INFINITY;
                 sg[nt][c] = gated;
                 bmax = fmaxf(bmax, gated);
@@ -1097,6 +1109,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.Hq = desc->n_q_heads; da.Hkv = desc->n_kv_heads; da.G = G; da.b = b; da.t_cap = desc->t_cap;
     da.nseg = L.nseg; da.entries = L.entries; da.rows = L.rows; da.nb_cap = desc->nb_cap;
     da.rescue_window = params->rescue_window;
+    da.ungate_last = (!dense && (params->flags & ETA_FLAG_UNGATE_LAST)) ? 1 : 0;
     da.div_nseg = FastDiv(L.nseg); da.div_epr = FastDiv(L.nseg + 2); da.div_hkv = FastDiv(desc->n_kv_heads);
     da.div_g = FastDiv(G);
     da.timeline = debug_timeline();

@@ -139,7 +139,8 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     for (int item = it0; item < it1; ++item) {
         const int k = item - it0, buf = k & 1;
         const int r = gc.r, seg = gc.seg, i = gc.i, hk = gc.hk, T = gc.T, NB = gc.NB, j0 = gc.j0, n_rec = gc.n_rec;
-        (void)T;
+        // an ungated newest token must be attended: when it closes a full block, that block counts as pinned
+        const int lwb_item = ((a.flags & ETA_FLAG_UNGATE_LAST) && T > 0 && (T & (a.b - 1)) == 0 && a.lwb < 1) ? 1 : a.lwb;
         Geom gn = gc;
         float mn_next = 0.f, te_next = 0.f;
         bool next_issued = false, next_te = false;
@@ -256,7 +257,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                     const bool valid = rec < n_rec;
                     const float mnv = valid ? smn[rec] : 0.f;
                     const float bound = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * mnv);
-                    const bool pinned = (j0 + rec) >= NB - a.lwb;
+                    const bool pinned = (j0 + rec) >= NB - lwb_item;
                     if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }     // first item only
                     const bool admit = valid && (!(bound < my_te) || pinned || !ok);
                     if (valid) sbound[rec][my_g] = bound;

@@ -159,9 +159,13 @@ def _decode_case(w, q, tau=None, head_const=None, **params):
     sp = w.spec
     c = cache_of(w)
     musig, mnorm = orc.block_summaries(c)
+    params = dict(params)
+    ungate = params.pop("ungate_last", False)
     ref = orc.decode_step(bits(q), c, musig, mnorm, tau=tau, head_const=head_const, z=params.get("z", 1.0),
                           a=params.get("a", 0.0), beta=params.get("beta", 5.0), lwb=params.get("lwb", 0),
-                          rescue_window=params.get("rescue_window", 128))
+                          rescue_window=params.get("rescue_window", 128), ungate_last=ungate)
+    if ungate:
+        params["flags"] = params.get("flags", 0) | _eb().ETA_FLAG_UNGATE_LAST
     out, sel, stats, status = gpu_decode(q, w.K, w.V, c.seq_lens, sp.block_size, musig, mnorm, tau=tau,
                                          head_const=head_const, **params)
     assert status == 0
@@ -217,6 +221,28 @@ def test_decode_matches_oracle_on_scaled_configs(name, ctx, batch, params):
         kw.update(params)
         (mx, mean), near, ref = _decode_case(w, q, tau=tau, **kw)
         print(f"{name} ctx={ctx} target={target}: max {mx:.2e} mean {mean:.2e} near-ties {len(near)}")
+
+
+@pytest.mark.parametrize("name,ctx,batch", [("c2_32k", 4096, 2), ("c2_32k", 4096 + 77, 2), ("c4_512k", 16384, 1),
+                                            ("c4_512k", 16384 + 100, 1), ("c1_tiny", 2048 + 16, 1), ("c1_tiny", 2048, 1)])
+def test_ungated_newest_token(name, ctx, batch):
+    """ETA_FLAG_UNGATE_LAST: the newest token keeps its raw logit; when it closes a block the block is admitted.
+    Contexts that end on a block boundary and in a tail, one and two tiles per block."""
+    _eb()
+    sp = wl.CONFIGS[name].scaled(ctx, batch=batch)
+    w = wl.make_workload(sp)
+    q = w.queries(0)
+    tau, _ = _calibrated_tau(w, q, 0.9)
+    (mx, mean), near, ref = _decode_case(w, q, tau=tau, z=sp.z, beta=sp.beta, ungate_last=True)
+    if ctx % sp.block_size == 0:
+        NB = ctx // sp.block_size
+        assert np.all(ref["sel"][:, :, NB - 1] == (1 << sp.gqa) - 1)
+    # an infinite threshold closes every other gate: the newest token then dominates in closed form (oracle pin);
+    # here: both sides agree on it
+    inf = np.full_like(tau, np.inf)
+    (_, _), _, r1 = _decode_case(w, q, tau=inf, z=sp.z, beta=sp.beta, ungate_last=True)
+    (_, _), _, r0 = _decode_case(w, q, tau=inf, z=sp.z, beta=sp.beta)
+    assert np.abs(r1["out"] - r0["out"]).max() > 1e-6            # here the flag does change the result
 
 
 def test_frozen_constants_against_predicted_mode_on_the_same_cache():
