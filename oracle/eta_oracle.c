@@ -496,3 +496,91 @@ void eta_oracle_block_max_logit(
         }
     }
 }
+
+/* ------------------------------------------------------------------------ */
+/* Offline threshold calibration (appendix "Offline Threshold Calibration via */
+/* 1/t-Weighted Histograms", Algorithm "Density-Matched Offline Threshold     */
+/* Calibration")                                                              */
+/* ------------------------------------------------------------------------ */
+
+static double oracle_sigmoid(double x) {
+    if (x >= 0) return 1.0 / (1.0 + exp(-x));
+    double e = exp(x);
+    return e / (1.0 + e);
+}
+
+/* g(c) = sum_b H[b] sigmoid(beta (s_b - c)): the head's density under a static
+ * threshold c, from the normalised 1/t-weighted score histogram. */
+double eta_oracle_calibration_density(const double* hist, int n_bins, double s_min, double s_max,
+                                      double beta, double c)
+{
+    double w = (s_max - s_min) / n_bins, g = 0.0;
+    for (int b = 0; b < n_bins; ++b) g += hist[b] * oracle_sigmoid(beta * (s_min + (b + 0.5) * w - c));
+    return g;
+}
+
+/*
+ * The calibration pass over a split of n_seq sequences of T tokens, per query
+ * head h (GQA: KV head h / G), with raw causal scores S_ts = s <q_t, k_s>,
+ * s <= t, and the dynamic thresholds tau[x,h,t] of the predictor:
+ *   target density   dbar_h = 1/(n_seq T) sum_x sum_t (1/t) sum_{s<=t} sigmoid(beta (S_ts - tau_t))
+ *   histogram        H_h[bin(S_ts)] += 1/t    (t counted from 1), then H_h /= sum_b H_h[b]
+ *   constant         c_h = root of g(c) = dbar_h by bisection (g decreases from 1 to 0)
+ * Bins: n_bins equal bins on [s_min, s_max], centre s_b = s_min + (b + 1/2) w;
+ * a score outside the range goes to the first / last bin (the paper fixes
+ * neither range nor edge rule).  The bin of a score is decided on the score
+ * rounded to binary32, the precision the GPU path computes scores in.
+ * Bisection: `iters` halvings of [s_min - 40/beta, s_max + 40/beta].
+ * hist [Hq, n_bins], dbar [Hq], head_const [Hq], residual [Hq] (= g(c) - dbar).
+ */
+void eta_oracle_calibrate(
+    const uint16_t* Q, const uint16_t* K, const float* tau,
+    int n_seq, int Hq, int Hkv, int T, int d, double beta, double s,
+    int n_bins, double s_min, double s_max, int iters,
+    double* hist, double* dbar, double* head_const, double* residual)
+{
+    int G = Hq / Hkv;
+    double w = (s_max - s_min) / n_bins;
+    #pragma omp parallel for schedule(dynamic)
+    for (int h = 0; h < Hq; ++h) {
+        double* H = hist + (int64_t)h * n_bins;
+        for (int b = 0; b < n_bins; ++b) H[b] = 0.0;
+        double dsum = 0.0;
+        for (int x = 0; x < n_seq; ++x) {
+            const uint16_t* Qh = Q + (((int64_t)x * Hq + h) * T) * d;
+            const uint16_t* Kh = K + (((int64_t)x * Hkv + h / G) * T) * d;
+            for (int t = 0; t < T; ++t) {
+                double inv_t = 1.0 / (double)(t + 1);
+                double th = (double)tau[((int64_t)x * Hq + h) * T + t];
+                double rowsum = 0.0;
+                for (int sidx = 0; sidx <= t; ++sidx) {
+                    double dot = 0.0;
+                    for (int c = 0; c < d; ++c)
+                        dot += eta_oracle_bf16_to_double(Qh[(int64_t)t * d + c]) *
+                               eta_oracle_bf16_to_double(Kh[(int64_t)sidx * d + c]);
+                    double S = s * dot;
+                    rowsum += oracle_sigmoid(beta * (S - th));
+                    double Sf = (double)(float)S;
+                    int b = (int)floor((Sf - s_min) / w);
+                    if (b < 0) b = 0;
+                    if (b >= n_bins) b = n_bins - 1;
+                    H[b] += inv_t;
+                }
+                dsum += rowsum * inv_t;
+            }
+        }
+        double tot = 0.0;
+        for (int b = 0; b < n_bins; ++b) tot += H[b];
+        for (int b = 0; b < n_bins; ++b) H[b] = tot > 0.0 ? H[b] / tot : 0.0;
+        double target = dsum / ((double)n_seq * (double)T);
+        double lo = s_min - 40.0 / beta, hi = s_max + 40.0 / beta;
+        for (int it = 0; it < iters; ++it) {
+            double mid = 0.5 * (lo + hi);
+            if (eta_oracle_calibration_density(H, n_bins, s_min, s_max, beta, mid) > target) lo = mid; else hi = mid;
+        }
+        double c = 0.5 * (lo + hi);
+        dbar[h] = target;
+        head_const[h] = c;
+        if (residual) residual[h] = eta_oracle_calibration_density(H, n_bins, s_min, s_max, beta, c) - target;
+    }
+}

@@ -219,6 +219,31 @@ def block_max_logit(q, cache: Cache, scale=None):
     return out
 
 
+def calibration_density(hist, s_min, s_max, beta, c):
+    """g(c) of the calibration appendix for one head's normalised histogram."""
+    h = np.ascontiguousarray(hist, np.float64)
+    f = lib().eta_oracle_calibration_density
+    f.restype = ctypes.c_double
+    return f(_p(h, _f64), _I(h.shape[0]), _D(s_min), _D(s_max), _D(beta), _D(c))
+
+
+def calibrate(Q, K, tau, beta=5.0, scale=None, n_bins=2048, s_min=-8.0, s_max=8.0, iters=80):
+    """Density-matched static thresholds.  Q uint16 (bf16 bits) [n_seq, Hq, T, d], K [n_seq, Hkv, T, d],
+    tau float32 [n_seq, Hq, T]  ->  dict(hist [Hq, n_bins], dbar [Hq], head_const [Hq], residual [Hq])."""
+    n_seq, Hq, T, d = Q.shape
+    Hkv = K.shape[1]
+    s = (1.0 / np.sqrt(d)) if scale is None else scale
+    hist = np.zeros((Hq, n_bins), np.float64)
+    dbar = np.zeros(Hq, np.float64)
+    hc = np.zeros(Hq, np.float64)
+    res = np.zeros(Hq, np.float64)
+    lib().eta_oracle_calibrate(
+        _p(np.ascontiguousarray(Q), _u16), _p(np.ascontiguousarray(K), _u16),
+        _p(np.ascontiguousarray(tau, np.float32), _f32), _I(n_seq), _I(Hq), _I(Hkv), _I(T), _I(d), _D(beta), _D(s),
+        _I(n_bins), _D(s_min), _D(s_max), _I(iters), _p(hist, _f64), _p(dbar, _f64), _p(hc, _f64), _p(res, _f64))
+    return {"hist": hist, "dbar": dbar, "head_const": hc, "residual": res}
+
+
 def decode_step(q, cache: Cache, musig, mnorm, tau=None, head_const=None, z=1.0, a=0.0, beta=5.0, lwb=0,
                 rescue_window=128, scale=None, ungate_last=False):
     """The whole inference rule in the paper's order: bound -> select -> attend.

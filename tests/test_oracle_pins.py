@@ -567,3 +567,82 @@ def test_ungated_newest_token_forces_its_block_when_it_closes_one():
     sel1_rest = sel1.copy(); sel1_rest[0, :, NB - 1] = sel0[0, :, NB - 1]
     np.testing.assert_array_equal(sel1_rest, sel0)           # nothing else changes
     np.testing.assert_array_equal(sel1[1], sel0[1])          # newest token in the tail: already attended
+
+
+# ---------------------------------------------------------------------------------------------------
+# offline threshold calibration (1/t-weighted histogram + bisection)
+# ---------------------------------------------------------------------------------------------------
+
+def _calib_case(seed=3, n_seq=2, Hq=4, Hkv=2, T=40, d=16):
+    rng = np.random.default_rng(seed)
+    Q = bf16_bits_from_f64(rng.standard_normal((n_seq, Hq, T, d)))
+    K = bf16_bits_from_f64(rng.standard_normal((n_seq, Hkv, T, d)))
+    return rng, Q, K
+
+
+def test_calibration_hand_example_of_the_causal_row_weights():
+    # one sequence, one head, T = 2, d = 1: scores S11 = 1*1, S21 = 2*1, S22 = 2*3 (scale 1)
+    Q = bf16_bits_from_f64(np.array([1.0, 2.0]).reshape(1, 1, 2, 1))
+    K = bf16_bits_from_f64(np.array([1.0, 3.0]).reshape(1, 1, 2, 1))
+    tau = np.array([0.5, 4.0], np.float32).reshape(1, 1, 2)
+    r = orc.calibrate(Q, K, tau, beta=2.0, scale=1.0, n_bins=8, s_min=0.0, s_max=8.0)
+    # bins of width 1: S11 = 1 -> bin 1 (weight 1), S21 = 2 -> bin 2 (1/2), S22 = 6 -> bin 6 (1/2); total 2
+    expect = np.zeros(8); expect[1], expect[2], expect[6] = 0.5, 0.25, 0.25
+    np.testing.assert_allclose(r["hist"][0], expect, rtol=0, atol=1e-15)
+    sig = lambda x: 1.0 / (1.0 + math.exp(-x))
+    dbar = 0.5 * (sig(2.0 * (1 - 0.5)) + 0.5 * (sig(2.0 * (2 - 4.0)) + sig(2.0 * (6 - 4.0))))
+    np.testing.assert_allclose(r["dbar"][0], dbar, rtol=1e-14)
+    # the root solves 0.5 s(1.5-c) + 0.25 s(2.5-c) + 0.25 s(6.5-c) = dbar (bin centres), to the stated residual
+    g = 0.5 * sig(2 * (1.5 - r["head_const"][0])) + 0.25 * sig(2 * (2.5 - r["head_const"][0])) + 0.25 * sig(2 * (6.5 - r["head_const"][0]))
+    assert abs(g - dbar) < 5e-16 and abs(r["residual"][0]) < 5e-16          # machine precision, as the paper states
+
+
+def test_calibration_constant_scores_give_a_closed_form_constant():
+    n_seq, Hq, T, d = 2, 2, 24, 8
+    Q = bf16_bits_from_f64(np.tile(np.eye(1, d) * 1.5, (n_seq, Hq, T, 1)))
+    K = bf16_bits_from_f64(np.tile(np.eye(1, d) * 2.0, (n_seq, Hq, T, 1)))
+    S0, tau0, beta = 3.0 * 0.5, 0.9, 4.0                      # scale 0.5
+    r = orc.calibrate(Q, K, np.full((n_seq, Hq, T), tau0, np.float32), beta=beta, scale=0.5, n_bins=64, s_min=-4, s_max=4)
+    w = 8.0 / 64
+    s_b = -4 + (math.floor((S0 + 4) / w) + 0.5) * w          # centre of the bin that holds every score
+    tau0f = float(np.float32(tau0))
+    np.testing.assert_allclose(r["dbar"], 1.0 / (1.0 + math.exp(-beta * (S0 - tau0f))), rtol=1e-13)
+    np.testing.assert_allclose(r["head_const"], s_b - (S0 - tau0f), rtol=0, atol=1e-12)
+
+
+def test_calibration_reproduces_a_static_threshold_and_matches_brute_force_density():
+    rng, Q, K = _calib_case()
+    n_seq, Hq, T, d = Q.shape
+    beta, n_bins, s_min, s_max = 5.0, 1024, -6.0, 6.0
+    w = (s_max - s_min) / n_bins
+    tau = np.full((n_seq, Hq, T), 0.25, np.float32)
+    r = orc.calibrate(Q, K, tau, beta=beta, n_bins=n_bins, s_min=s_min, s_max=s_max)
+    assert np.all(np.abs(r["residual"]) < 5e-16)                        # machine precision (the paper: < 2e-16)
+    assert np.all(np.abs(r["head_const"] - 0.25) < w)                   # a constant predictor calibrates to itself
+    np.testing.assert_allclose(r["hist"].sum(axis=1), 1.0, rtol=1e-13)
+    # g(c) from the histogram against g(c) from the raw scores: sigmoid is beta/4-Lipschitz, scores move <= w/2
+    Qv, Kv = bf16_values(Q), bf16_values(K)
+    for h in range(Hq):
+        for c in (-1.0, 0.1, 0.25, 2.0):
+            tot = 0.0
+            for x in range(n_seq):
+                S = (Qv[x, h] @ Kv[x, h // 2].T) / math.sqrt(d)
+                for t in range(T):
+                    tot += (1.0 / (1.0 + np.exp(-beta * (S[t, :t + 1] - c)))).sum() / (t + 1)
+            g_raw = tot / (n_seq * T)
+            g_hist = orc.calibration_density(r["hist"][h], s_min, s_max, beta, c)
+            assert abs(g_raw - g_hist) <= beta * w / 8 + 1e-12
+    # g decreases in c
+    gs = [orc.calibration_density(r["hist"][0], s_min, s_max, beta, c) for c in np.linspace(-8, 8, 33)]
+    assert all(a > b for a, b in zip(gs, gs[1:])) and gs[0] > 0.999 and gs[-1] < 1e-3
+
+
+def test_calibration_matches_a_dynamic_predictor_in_density():
+    rng, Q, K = _calib_case(seed=8)
+    n_seq, Hq, T, d = Q.shape
+    tau = (0.2 + 0.5 * rng.standard_normal((n_seq, Hq, T))).astype(np.float32)     # token-dependent thresholds
+    r = orc.calibrate(Q, K, tau, beta=5.0, n_bins=2048, s_min=-6, s_max=6)
+    # the static constant yields the dynamic predictor's density on the split (that is its definition)
+    for h in range(Hq):
+        assert abs(orc.calibration_density(r["hist"][h], -6, 6, 5.0, r["head_const"][h]) - r["dbar"][h]) < 5e-16
+    assert np.all((r["dbar"] > 0.05) & (r["dbar"] < 0.95))
