@@ -141,6 +141,34 @@ int eta_score_dual(const eta_cache_desc* desc, const eta_params* params, const v
                    float* bound, void* stream);
 
 /*
+ * Appendix "Offline Threshold Calibration via 1/t-Weighted Histograms", Algorithm
+ * "Density-Matched Offline Threshold Calibration": replaces the dynamic predictor
+ * by one constant per query head with the same density on a calibration split.
+ * For every head h (KV head h / G), over n_seq sequences of seq_len tokens, with
+ * raw causal scores S_ts = s <q_t, k_s>, s <= t (t counted from 1):
+ *   dbar_h = 1/(n_seq seq_len) sum_x sum_t (1/t) sum_{s<=t} sigmoid(beta (S_ts - tau[x,h,t]))
+ *   H_h[bin(S_ts)] += 1/t, then H_h normalised to sum 1
+ *   head_const[h] = root of  sum_b H_h[b] sigmoid(beta (s_b - c)) = dbar_h  (bisection, double precision).
+ * Bins: n_bins (<= 4096) equal bins on [s_min, s_max], s_b the bin centre; scores
+ * outside the range go to the first / last bin (the paper fixes neither).
+ * Q bf16 [n_seq, n_q_heads, seq_len, head_dim], K bf16 [n_seq, n_kv_heads, seq_len,
+ * head_dim], tau fp32 [n_seq, n_q_heads, seq_len] (the predictor's thresholds),
+ * head_const fp32 [n_q_heads] (out), dbar fp32 [n_q_heads] (out, nullable); all
+ * device pointers.  Scores are computed in fp32 from the bf16 operands; the row
+ * weights are accumulated as integers, so the result does not depend on the
+ * order of the atomic updates.  head_dim 64 or 128; n_seq * seq_len <= 2^22.
+ * workspace: eta_calibration_workspace_bytes() bytes, 256-byte aligned, no
+ * initialisation needed.  Prefill-side tool: not part of a decode step.
+ */
+int eta_calibration_workspace_bytes(int32_t n_seq, int32_t seq_len, int32_t n_q_heads, int32_t n_bins,
+                                    size_t* out_bytes);
+int eta_calibrate_head_const(int32_t n_seq, int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads,
+                             int32_t head_dim, const void* Q, const void* K, const float* tau,
+                             float beta, float scale, int32_t n_bins, float s_min, float s_max,
+                             float* head_const, float* dbar, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/*
  * Algorithm 3 (screen, top-1 rescue, tail phase, chunk merge) with the
  * GQA-grouped execution of the fused-kernel appendix, for one decode query per
  * sequence.  Per query head h, with tau_eff = (tau[i,h] or head_const[h]) - a:

@@ -21,7 +21,7 @@ ETA_BUILD_SIGMA_ENVELOPE = 1
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
 EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
-           "eta_score_dual", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
+           "eta_score_dual", "eta_calibration_workspace_bytes", "eta_calibrate_head_const", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
            "eta_profile_kernel_name", "eta_set_pdl", "eta_debug_timeline", "eta_strerror", "eta_last_cuda_error")
 
 
@@ -61,6 +61,10 @@ def load() -> ctypes.CDLL:
         lib.eta_append_summary.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
         lib.eta_predict_threshold.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, f32p, f32p, f32p, vp]
         lib.eta_score_dual.argtypes = [D, P, vp, i32p, vp, f32p, f32p, vp]
+        i32 = ctypes.c_int32
+        lib.eta_calibration_workspace_bytes.argtypes = [i32, i32, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        lib.eta_calibrate_head_const.argtypes = [i32, i32, i32, i32, i32, vp, vp, f32p, ctypes.c_float, ctypes.c_float,
+                                                 i32, ctypes.c_float, ctypes.c_float, f32p, f32p, vp, ctypes.c_size_t, vp]
         lib.eta_decode.argtypes = [D, P, vp, vp, vp, i32p, vp, f32p, f32p, f32p, f32p, vp, i32p, vp, vp,
                                    ctypes.c_size_t, vp]
         lib.eta_decode_static.argtypes = [D, P, vp, vp, vp, i32p, vp, f32p, f32p, f32p, f32p, vp, i32p, vp, vp]
@@ -169,6 +173,28 @@ def eta_score_dual(desc, params: DecodeParams, q, seq_lens, musig, mnorm, bound)
                                  _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
                                  _dev(mnorm, torch.float32, "mnorm"), _dev(bound, torch.float32, "bound"), _stream()),
            "eta_score_dual")
+
+
+def eta_calibrate_head_const(Q, K, tau, head_const, dbar=None, beta=5.0, scale=0.0, n_bins=2048, s_min=-8.0,
+                             s_max=8.0, workspace=None):
+    """Q bf16 [n_seq, Hq, T, d], K bf16 [n_seq, Hkv, T, d], tau fp32 [n_seq, Hq, T] -> head_const fp32 [Hq]
+    (and dbar fp32 [Hq]).  Allocates the scratch with torch when none is given; returns it for reuse."""
+    n_seq, Hq, T, d = Q.shape
+    Hkv = K.shape[1]
+    need = ctypes.c_size_t(0)
+    _check(load().eta_calibration_workspace_bytes(n_seq, T, Hq, n_bins, ctypes.byref(need)),
+           "eta_calibration_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need.value + 256, dtype=torch.uint8, device=Q.device)
+        off = (-workspace.data_ptr()) % 256
+        workspace = workspace[off:off + need.value]
+    _check(load().eta_calibrate_head_const(n_seq, T, Hq, Hkv, d, _dev(Q, torch.bfloat16, "Q"),
+                                           _dev(K, torch.bfloat16, "K"), _dev(tau, torch.float32, "tau"), beta, scale,
+                                           n_bins, s_min, s_max, _dev(head_const, torch.float32, "head_const"),
+                                           _dev(dbar, torch.float32, "dbar"), _dev(workspace, torch.uint8, "workspace"),
+                                           workspace.numel(), _stream()),
+           "eta_calibrate_head_const")
+    return workspace
 
 
 def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,
