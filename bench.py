@@ -179,6 +179,28 @@ def run_ours(args):
     build_ms = ev0.elapsed_time(ev1)
     k_bytes = sum(int(t) // sp.block_size for t in lens) * sp.n_kv_heads * sp.block_size * sp.head_dim * 2
 
+    # offline calibration (prefill-side tool, timed on its own): 16 sequences of 1024 tokens at this head geometry
+    cal = None
+    if rank == 0 and world == 1:
+        gcal = torch.Generator(device=dev).manual_seed(208880)
+        cq = torch.randn((16, sp.n_q_heads, 1024, sp.head_dim), generator=gcal, device=dev).to(torch.bfloat16)
+        ck = torch.randn((16, sp.n_kv_heads, 1024, sp.head_dim), generator=gcal, device=dev).to(torch.bfloat16)
+        ctau = torch.full((16, sp.n_q_heads, 1024), 0.5, device=dev)
+        chc = torch.empty(sp.n_q_heads, device=dev)
+        cws = eb.eta_calibrate_head_const(cq, ck, ctau, chc, None, beta=sp.beta, n_bins=2048)
+        torch.cuda.synchronize()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for _ in range(5):
+            eb.eta_calibrate_head_const(cq, ck, ctau, chc, None, beta=sp.beta, n_bins=2048, workspace=cws)
+        c1.record()
+        torch.cuda.synchronize()
+        cal_ms = c0.elapsed_time(c1) / 5
+        pairs = 16 * sp.n_q_heads * (1024 * 1025 // 2)
+        cal = {"ms": cal_ms, "n_seq": 16, "seq_len": 1024, "n_bins": 2048,
+               "causal_pairs_per_s": pairs / (cal_ms * 1e-3), "max_abs_dev_from_0.5": float((chc - 0.5).abs().max())}
+        del cq, ck, ctau, cws
+
     n_q = args.steps + args.warmup
     q_host = [w.queries(s).pin_memory() for s in range(n_q)]
     q_dev = [q.to(dev) for q in q_host]
@@ -353,6 +375,7 @@ def run_ours(args):
                          "traffic": NCU_TRAFFIC_BYTES.get((sp.name, main_target)), "traffic_unit": "bytes per launch",
                          "algorithmic_bytes_per_launch": ab["decode"]},
             "prefill_build": {"ms": build_ms, "gbs": k_bytes / (build_ms * 1e-3) / 1e9},
+            "calibration": cal,
             "sweep": sweep,
             "cpu_baseline": cpu,
             "setup_s": {"generate": round(gen_s, 1)},
