@@ -26,22 +26,27 @@ __device__ __forceinline__ float min_keep_nan(float g, float s) {
     return (g < s) ? g : ((s < g) ? s : ((g != g) ? g : s));
 }
 
+constexpr int SCR_GROUP = 8;       // items whose bounds are kept before their admission is decided: one per warp
+
 template <int D, int G>
 struct ScreenSmem {
     static constexpr int REC_BYTES = 4 * D;                    // fp16 mu[d] + fp16 sigma[d]
     static constexpr int BUF_BYTES = SEG * REC_BYTES + G * D * 2;   // a segment's records, then the group's queries
     static constexpr int BAR_OFF = 2 * BUF_BYTES;
-    static constexpr int BOUND_OFF = BAR_OFF + 16;
-    static constexpr int MN_OFF = BOUND_OFF + 4 * SEG * G;
-    static constexpr int MASK_OFF = MN_OFF + 4 * SEG;
-    static constexpr int MISC_OFF = MASK_OFF + SEG;            // int s_last, int warp sums[8]
-    static constexpr int LEN_OFF = MISC_OFF + 64;              // int32 clamped sequence lengths [MAX_ROWS]
+    static constexpr int BOUND_OFF = BAR_OFF + 16;             // float [SCR_GROUP][SEG][G]: bounds of a group's items
+    static constexpr int MN_OFF = BOUND_OFF + SCR_GROUP * 4 * SEG * G;   // float [2][SEG]: largest key norms
+    static constexpr int OK_OFF = MN_OFF + 2 * 4 * SEG;        // int [SCR_GROUP]: 0 where the wait for an item's records ran out
+    static constexpr int LEN_OFF = OK_OFF + 4 * SCR_GROUP;     // int32 clamped sequence lengths [MAX_ROWS]
     static constexpr int BYTES = LEN_OFF + 4 * MAX_ROWS + 128; // + slack for the 128-byte alignment of the base
 };
 
-// Persistent screening kernel: every CTA owns a contiguous range of (row, segment) items and double-buffers
-// them, so the records (and the group's queries) of the next item are in flight while the current one is
-// evaluated.
+// Persistent screening kernel.  Every CTA owns a contiguous range of (row, segment) items and works through it in
+// groups of up to SCR_GROUP items, in two phases.
+//   Phase 1, item by item: the records (and the group's queries) arrive by double-buffered 1-D bulk copies and
+//   the bound of every (record, head) pair is computed and kept in shared memory.  Nothing here needs the
+//   thresholds, so under programmatic dependent launch this phase runs while the predictor is still at work.
+//   Phase 2, a warp per item: admission against the thresholds, pinning, the user-visible mask, compaction of the
+//   union in ascending block order, and the rescue-window statistics.
 template <int D, int G>
 __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     using L = ScreenSmem<D, G>;
@@ -57,9 +62,9 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     extern __shared__ unsigned char scr_raw[];
     unsigned char* sm = scr_raw + ((128u - (smem_u32(scr_raw) & 127u)) & 127u);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::BAR_OFF);
-    float (*sbound)[G] = reinterpret_cast<float (*)[G]>(sm + L::BOUND_OFF);
-    float* smn = reinterpret_cast<float*>(sm + L::MN_OFF);
-    uint8_t* smask = sm + L::MASK_OFF;
+    float (*sbound_all)[G] = reinterpret_cast<float (*)[G]>(sm + L::BOUND_OFF);
+    float* smn_all = reinterpret_cast<float*>(sm + L::MN_OFF);
+    int* s_ok = reinterpret_cast<int*>(sm + L::OK_OFF);
     int* s_len = reinterpret_cast<int*>(sm + L::LEN_OFF);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -78,6 +83,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         mbar_init(&bars[1], 1);
         fence_barrier_init();
     }
+    if (tid < SCR_GROUP) s_ok[tid] = 1;
     // sequence lengths (a caller input) of every row, clamped, once: the per-item geometry then needs no global load
     for (int rr = tid; rr < a.rows; rr += 256) {
         const int T = a.seq_lens[rr / a.Hkv];
@@ -114,17 +120,12 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     // The summaries and thresholds may still be in the making when this kernel starts (programmatic dependent
     // launch): the append kernel writes the record and the norm of a block that has just filled up, the predictor
     // writes tau.  Everything else this kernel reads is final, so only an item that holds a row's newest block of
-    // a just-completed length must wait before its copies; the thresholds are fetched after the wait, which
-    // the first item reaches only when its bounds are already computed.
+    // a just-completed length must wait before its copies; the thresholds are read in phase 2, after the wait.
     auto safe_item = [&](const Geom& g) {
         return !(g.n_rec > 0 && (g.T & (a.b - 1)) == 0 && g.j0 + g.n_rec == g.NB);
     };
     auto load_mn = [&](const Geom& g) {        // largest-norm entry of record `tid` of the item
         return (tid < g.n_rec && !dense) ? __ldg(a.mnorm + (int64_t)g.r * a.nb_cap + g.j0 + tid) : 0.f;
-    };
-    auto load_te = [&](const Geom& g) {        // effective threshold of head my_g of the item's group
-        const int h = g.hk * G + my_g;
-        return dense ? -INFINITY : ((a.tau ? __ldg(a.tau + (int64_t)g.i * a.Hq + h) : __ldg(a.head_const + h)) - a.a);
     };
 
     float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G], my_qn = 0.f;
@@ -133,81 +134,70 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     Geom gc = item_geom(it0);
     if (!safe_item(gc)) { pdl_wait(); waited = true; }
     if (tid == 0) issue(gc, 0);
-    float mn_cur = load_mn(gc);
-    float te_cur = waited ? load_te(gc) : 0.f;
+    {
+        const float mn0 = load_mn(gc);
+        if (tid < SEG) smn_all[tid] = mn0;
+    }
+    __syncthreads();
 
-    for (int item = it0; item < it1; ++item) {
-        const int k = item - it0, buf = k & 1;
-        const int r = gc.r, seg = gc.seg, i = gc.i, hk = gc.hk, T = gc.T, NB = gc.NB, j0 = gc.j0, n_rec = gc.n_rec;
-        // an ungated newest token must be attended: when it closes a full block, that block counts as pinned
-        const int lwb_item = ((a.flags & ETA_FLAG_UNGATE_LAST) && T > 0 && (T & (a.b - 1)) == 0 && a.lwb < 1) ? 1 : a.lwb;
-        Geom gn = gc;
-        float mn_next = 0.f, te_next = 0.f;
-        bool next_issued = false, next_te = false;
-        if (item + 1 < it1) {
-            gn = item_geom(item + 1);
-            if (waited || safe_item(gn)) {
+    for (int gs = it0; gs < it1; gs += SCR_GROUP) {
+        const int ge = min(it1, gs + SCR_GROUP);
+        // ------------------------------------------------------------ phase 1: bounds of the group's items
+        for (int item = gs; item < ge; ++item) {
+            const int k = item - it0, buf = k & 1, slot = item - gs;
+            float (*sbound)[G] = sbound_all + slot * SEG;
+            const float* smn = smn_all + buf * SEG;
+            const int r = gc.r, n_rec = gc.n_rec;
+            Geom gn = gc;
+            float mn_next = 0.f;
+            if (item + 1 < it1) {
+                gn = item_geom(item + 1);
+                if (!waited && !safe_item(gn)) { pdl_wait(); waited = true; }
                 if (tid == 0) issue(gn, buf ^ 1);
                 mn_next = load_mn(gn);
-                next_issued = true;
             }
-            if (waited) { te_next = load_te(gn); next_te = true; }
-        }
-        float my_te = te_cur;
-        if (tid < SEG) smn[tid] = mn_cur;
-        if (seg == 0 && tid == 0 && a.status) {
-            const int Traw = __ldg(a.seq_lens + i);
-            if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
-            if (Traw <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
-        }
-        // mask entries of this segment that are not full blocks read as "not attended"
-        if (tid < SEG && tid >= n_rec && j0 + tid < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = 0;
-        if (n_rec == 0 && tid == 0) a.seg_count[r * a.nseg + seg] = 0;
+            if (tl && tid == 0 && item == it0 + 1) tl[6] = globaltimer_ns();
+            bool ok = mbar_wait(&bars[buf], (k >> 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok && lane == 0) s_ok[slot] = 0;
+            if (tl && tid == 0 && item == it0 + 1) tl[7] = globaltimer_ns();
 
-        if (tl && tid == 0 && item == it0 + 1) tl[6] = globaltimer_ns();
-        bool ok = mbar_wait(&bars[buf], (k >> 1) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        __syncthreads();       // smn visible
-        if (tl && tid == 0 && item == it0 + 1) tl[7] = globaltimer_ns();
-
-        if (n_rec > 0) {
-            const uint32_t rec_base = smem_u32(sm + buf * L::BUF_BYTES);
-            if (!dense) {
+            if (n_rec > 0 && !dense && ok) {
+                const uint32_t rec_base = smem_u32(sm + buf * L::BUF_BYTES);
                 // this lane's slice of the G query vectors, in fp32: kept across the items of one row
                 if (r != q_row) {
-                q_row = r;
+                    q_row = r;
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const uint4 v = lds128(rec_base + SEG * REC_BYTES + (g * D + cc * 8) * 2);
-                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                    float n2 = 0.f;
+                    for (int g = 0; g < G; ++g) {
+                        const uint4 v = lds128(rec_base + SEG * REC_BYTES + (g * D + cc * 8) * 2);
+                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                        float n2 = 0.f;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        qf[g][2 * kk] = bf16_lo(w[kk]);
-                        qf[g][2 * kk + 1] = bf16_hi(w[kk]);
+                        for (int kk = 0; kk < 4; ++kk) {
+                            qf[g][2 * kk] = bf16_lo(w[kk]);
+                            qf[g][2 * kk + 1] = bf16_hi(w[kk]);
+                        }
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            n2 = fmaf(qf[g][kk], qf[g][kk], n2);
+                            if (USE_Q2) q2[g][kk] = qf[g][kk] * qf[g][kk];
+                        }
+#pragma unroll
+                        for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+                        qn[g] = sqrtf(n2);
                     }
+                    my_qn = qn[0];
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        n2 = fmaf(qf[g][kk], qf[g][kk], n2);
-                        if (USE_Q2) q2[g][kk] = qf[g][kk] * qf[g][kk];
-                    }
-#pragma unroll
-                    for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
-                    qn[g] = sqrtf(n2);
-                }
-                my_qn = qn[0];
-#pragma unroll
-                for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
+                    for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
                 }
 
                 for (int base = warp * RB; base < n_rec; base += 8 * RB) {
-                    // a wait that ran out: admit everything (errs toward loading) - never seen in practice
                     float v[NV];
 #pragma unroll
                     for (int it = 0; it < NI; ++it) {
                         const int rec = base + it * RPW + rg;
                         float mu[8], s2[8];
-                        if (rec < n_rec && ok) {
+                        if (rec < n_rec) {
                             const uint32_t addr = rec_base + rec * REC_BYTES + cc * 16;
                             const uint4 m4 = lds128(addr), s4 = lds128(addr + 2 * D);
                             const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw[4] = {s4.x, s4.y, s4.z, s4.w};
@@ -254,83 +244,109 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                     // lane cc now holds (dot, var) of pair cc = it * G + g
                     const int it = cc / G;
                     const int rec = base + it * RPW + rg;
-                    const bool valid = rec < n_rec;
-                    const float mnv = valid ? smn[rec] : 0.f;
-                    const float bound = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * mnv);
-                    const bool pinned = (j0 + rec) >= NB - lwb_item;
-                    if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }     // first item only
-                    const bool admit = valid && (!(bound < my_te) || pinned || !ok);
-                    if (valid) sbound[rec][my_g] = bound;
-                    const unsigned bal = __ballot_sync(0xffffffffu, admit);
-                    if (valid && my_g == 0) smask[rec] = (uint8_t)((bal >> lane) & ((1u << G) - 1u));
+                    if (rec < n_rec)
+                        sbound[rec][my_g] = a.scale * min_keep_nan(v[0] + a.z * sqrtf(v[1]), my_qn * smn[rec]);
                 }
-            } else {
-                if (tid < n_rec) smask[tid] = (uint8_t)((1u << G) - 1u);
             }
-            if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }     // warps without a batch
+            // the next item's key norms (fetched at the top of this iteration) go to its parity before the barrier
+            if (item + 1 < it1 && tid < SEG) smn_all[(buf ^ 1) * SEG + tid] = mn_next;
+            // the one CTA-wide barrier of an item: its bounds are complete, and every read of the record buffer the
+            // next copy goes into (and of the norms two items back) is over
             __syncthreads();
             if (tl && tid == 0 && item == it0 + 1) tl[1] = globaltimer_ns();
+            gc = gn;
+        }
 
-            // user-visible admission bits
-            if (tid < n_rec) a.sel_mask[(int64_t)r * a.nb_cap + j0 + tid] = smask[tid];
-
+        // ------------------------------------------------------------ phase 2: a warp per item of the group
+        if (!waited) { pdl_wait(); waited = true; }       // the thresholds (and the newest summaries) are final now
+        if (gs + warp < ge) {
+            const int slot = warp;
+            const Geom g = item_geom(gs + slot);
+            const float (*sbound)[G] = sbound_all + slot * SEG;
+            const int r = g.r, seg = g.seg, NB = g.NB, j0 = g.j0, n_rec = g.n_rec;
+            const bool ok = s_ok[slot] != 0;
+            // an ungated newest token must be attended: when it closes a full block, that block counts as pinned
+            const int lwb_item = ((a.flags & ETA_FLAG_UNGATE_LAST) && g.T > 0 && (g.T & (a.b - 1)) == 0 && a.lwb < 1) ? 1 : a.lwb;
+            // lane gq < G fetches the effective threshold of head gq of the item's group
+            float te_l = -INFINITY;
+            if (!dense && lane < G) {
+                const int h = g.hk * G + lane;
+                te_l = (a.tau ? __ldg(a.tau + (int64_t)g.i * a.Hq + h) : __ldg(a.head_const + h)) - a.a;
+            }
+            float te_g[G];
+#pragma unroll
+            for (int gq = 0; gq < G; ++gq) te_g[gq] = __shfl_sync(0xffffffffu, te_l, gq);
+            if (seg == 0) {
+                if (lane < G) a.tau_eff[(int64_t)g.i * a.Hq + g.hk * G + lane] = te_l;
+                if (lane == 0 && a.status) {
+                    const int Traw = __ldg(a.seq_lens + g.i);
+                    if (Traw > a.t_cap) atomicOr(a.status, ETA_DEV_LEN_CLAMPED);
+                    if (Traw <= 0) atomicOr(a.status, ETA_DEV_EMPTY_ROW);
+                }
+            }
+            // admission bits of records lane and lane + 32
+            unsigned m[SEG / 32];
+#pragma unroll
+            for (int half = 0; half < SEG / 32; ++half) {
+                const int rec = half * 32 + lane;
+                m[half] = 0;
+                if (rec < n_rec) {
+                    const bool pinned = (j0 + rec) >= NB - lwb_item;
+#pragma unroll
+                    for (int gq = 0; gq < G; ++gq)
+                        if (dense || !ok || pinned || !(sbound[rec][gq] < te_g[gq])) m[half] |= 1u << gq;
+                }
+                // user-visible bits; entries of this segment that are not full blocks read as "not attended"
+                if (j0 + rec < a.nb_cap) a.sel_mask[(int64_t)r * a.nb_cap + j0 + rec] = (uint8_t)m[half];
+            }
             // segment-local compaction of the union (ballot + popc prefix), ascending block order
-            if (warp == 7) {
+            {
                 int carry = 0;
                 int32_t* list = a.seg_list + ((int64_t)r * a.nseg + seg) * LSTRIDE;
 #pragma unroll
                 for (int half = 0; half < SEG / 32; ++half) {
-                    const int rec = half * 32 + lane;
-                    const unsigned m = (rec < n_rec) ? smask[rec] : 0u;
-                    const unsigned nz = __ballot_sync(0xffffffffu, m != 0);
-                    if (m) list[carry + __popc(nz & ((1u << lane) - 1u))] = (j0 + rec) | (int)(m << 24);
+                    const unsigned nz = __ballot_sync(0xffffffffu, m[half] != 0);
+                    if (m[half]) list[carry + __popc(nz & ((1u << lane) - 1u))] = (j0 + half * 32 + lane) | (int)(m[half] << 24);
                     carry += __popc(nz);
                 }
                 if (lane == 0) a.seg_count[r * a.nseg + seg] = carry;
             }
-
             // rescue statistics of the part of the rescue window inside this segment, per query head
             const int Wr = min(a.rescue_window, NB);
-            if (j0 < Wr && warp < G) {
-                const int g = warp;
+            if (j0 < Wr && n_rec > 0) {
                 const int nwin = min(n_rec, Wr - j0);
-                int cnt = 0, arg = 0x7fffffff;
-                float best = -INFINITY;
 #pragma unroll
-                for (int half = 0; half < SEG / 32; ++half) {
-                    const int rec = half * 32 + lane;
-                    if (rec < nwin) {
-                        cnt += (smask[rec] >> g) & 1;
-                        const float bd = dense ? 0.f : sbound[rec][g];
-                        if (bd > best) { best = bd; arg = rec; }
+                for (int gq = 0; gq < G; ++gq) {
+                    int cnt = 0, arg = 0x7fffffff;
+                    float best = -INFINITY;
+#pragma unroll
+                    for (int half = 0; half < SEG / 32; ++half) {
+                        const int rec = half * 32 + lane;
+                        if (rec < nwin) {
+                            cnt += (m[half] >> gq) & 1;
+                            const float bd = (dense || !ok) ? 0.f : sbound[rec][gq];
+                            if (bd > best) { best = bd; arg = rec; }
+                        }
+                    }
+#pragma unroll
+                    for (int s = 16; s >= 1; s >>= 1) {
+                        cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
+                        const float ob = __shfl_xor_sync(0xffffffffu, best, s);
+                        const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
+                        if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+                    }
+                    if (lane == 0) {
+                        RescueRec rr;
+                        rr.cnt = cnt; rr.maxb = best; rr.arg = (arg == 0x7fffffff) ? -1 : (j0 + arg); rr.pad = 0;
+                        a.seg_resc[((int64_t)r * a.nseg + seg) * G + gq] = rr;
                     }
                 }
-#pragma unroll
-                for (int s = 16; s >= 1; s >>= 1) {
-                    cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
-                    const float ob = __shfl_xor_sync(0xffffffffu, best, s);
-                    const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
-                    if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
-                }
-                if (lane == 0) {
-                    RescueRec rr;
-                    rr.cnt = cnt; rr.maxb = best; rr.arg = (arg == 0x7fffffff) ? -1 : (j0 + arg); rr.pad = 0;
-                    a.seg_resc[((int64_t)r * a.nseg + seg) * G + g] = rr;
-                }
             }
-        }   // n_rec > 0
-        if (!waited) { pdl_wait(); waited = true; my_te = load_te(gc); }
-        if (seg == 0 && tid < G) a.tau_eff[(int64_t)i * a.Hq + hk * G + tid] = my_te;     // lane g < G holds head g
-        if (item + 1 < it1 && !next_issued) {
-            if (tid == 0) issue(gn, buf ^ 1);
-            mn_next = load_mn(gn);
         }
-        if (item + 1 < it1 && !next_te) te_next = load_te(gn);
-
-        __syncthreads();       // the item's shared-memory state may be overwritten from here on
-        mn_cur = mn_next;
-        te_cur = te_next;
-        gc = gn;
+        if (ge < it1) {
+            __syncthreads();          // the bounds of this group have been read: the next group may overwrite them
+            if (tid < SCR_GROUP) s_ok[tid] = 1;
+        }
     }
     if (tl && tid == 0) tl[5] = globaltimer_ns();
     pdl_trigger();
