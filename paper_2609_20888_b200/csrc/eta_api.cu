@@ -77,7 +77,6 @@ WsLayout ws_layout(const eta_cache_desc* d) {
     L.seg_resc = off;   off = align_up(off + sizeof(RescueRec) * (size_t)L.rows * L.nseg * G, 256);
     L.row_start = off;  off = align_up(off + sizeof(int32_t) * ((size_t)L.rows + 1), 256);
     L.cta_range = off;  off = align_up(off + sizeof(int2) * (size_t)MAX_CTAS, 256);
-    L.row_cand = off;   off = align_up(off + sizeof(int2) * (size_t)L.rows, 256);
     L.tau_eff = off;    off = align_up(off + sizeof(float) * (size_t)d->batch * d->n_q_heads, 256);
     size_t slots = ((size_t)MAX_CTAS + L.rows) * DECODE_GROUPS;
     L.part_ml = off;    off = align_up(off + sizeof(float2) * slots * G, 256);
@@ -134,9 +133,12 @@ int eta_profile_read(float* ms, int n) {
     cudaError_t e = cudaEventSynchronize(g_ev[5]);
     for (int k = 0; k < N_MARKS - 1 && e == cudaSuccess; ++k) {
         ms[k] = 0.f;
-        // append / predict are separate calls: timed only when they were made in the same profiled step
-        if (k < 2 && !((g_ev_seen >> k) & 1)) continue;
-        e = cudaEventElapsedTime(&ms[k], g_ev[k], g_ev[k + 1]);
+        // append / predict are separate calls: timed only when they were made in the same profiled step; an
+        // interval runs to the next mark that was recorded
+        if (!((g_ev_seen >> k) & 1)) continue;
+        int j = k + 1;
+        while (j < N_MARKS - 1 && !((g_ev_seen >> j) & 1)) ++j;
+        e = cudaEventElapsedTime(&ms[k], g_ev[k], g_ev[j]);
     }
     if (e != cudaSuccess) { set_cuda_error(e, "eta_profile_read"); return ETA_ERR_CUDA; }
     return N_MARKS - 1;

@@ -45,7 +45,6 @@ struct WsLayout {
     size_t seg_resc;    // {int cnt; float maxb; int arg; int pad} [rows * nseg * G]
     size_t row_start;   // int32 [rows + 1]: global unit prefix over rows (written by the streaming kernel)
     size_t cta_range;   // int2 [MAX_CTAS]: unit range of every streaming CTA (written by the streaming kernel)
-    size_t row_cand;    // int2 [rows]: first and last streaming CTA whose range meets the row
     size_t tau_eff;     // float [batch * n_q_heads]
     size_t part_ml;     // float2 [(MAX_CTAS + rows) * DECODE_GROUPS * G]
     size_t part_o;      // float [(MAX_CTAS + rows) * DECODE_GROUPS * G * d]
@@ -89,6 +88,7 @@ struct ScreenArgs {
     int lwb, rescue_window;
     uint32_t flags;
     int Hq, Hkv, b, b_shift, t_cap, nb_cap, nseg, rows;
+    int n_early, per_early, per_late;     // item split over the CTAs: the first n_early share per_early items evenly, the rest take per_late each
     FastDiv div_nseg, div_hkv;
     int32_t* seg_count;
     int32_t* seg_list;

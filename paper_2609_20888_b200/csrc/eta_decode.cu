@@ -36,7 +36,6 @@ struct DecodeArgs {
     int32_t* stats;
     int32_t* row_start;
     int2* cta_range;
-    int2* row_cand;
     int32_t* hdr;
     float2* part_ml;
     float* part_o;
@@ -313,27 +312,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         for (int rr = tid; rr <= a.rows; rr += 32 * (WARPS_PER_GROUP * NGROUPS + 1)) a.row_start[rr] = rowbase[rr];
         if (tid == 0) { a.hdr[0] = U; a.hdr[1] = P; }
     }
-    if (tid == 0) {
-        a.cta_range[blockIdx.x] = make_int2(u0, u1);      // read by the merge kernel
-        // the streaming CTAs whose ranges meet row rr, for the rows this CTA looks after: first CTA that ends
-        // after the row's first unit, last CTA that starts before the row's end
-        for (int rr = blockIdx.x; rr < a.rows; rr += P) {
-            const int ra = rowbase[rr], rb = rowbase[rr + 1];
-            int lo = 0, hi = P - 1;
-            while (lo < hi) {             // first c with u1(c) > ra
-                const int mid = (lo + hi) >> 1;
-                const int e1 = (mid + 1 == P) ? U : cost_to_unit(((mid + 1) * C) / P);
-                if (e1 > ra) hi = mid; else lo = mid + 1;
-            }
-            const int c_lo = lo;
-            lo = 0; hi = P - 1;
-            while (lo < hi) {             // last c with u0(c) < rb
-                const int mid = (lo + hi + 1) >> 1;
-                if (cost_to_unit((mid * C) / P) < rb) lo = mid; else hi = mid - 1;
-            }
-            a.row_cand[rr] = make_int2(c_lo, rb > ra ? lo : c_lo - 1);
-        }
-    }
+    if (tid == 0) a.cta_range[blockIdx.x] = make_int2(u0, u1);      // read by the merge kernel
     if (tl && tid == 0) tl[1] = globaltimer_ns();
     if (u0 >= u1) return;
     // row holding unit u0: last r with rowbase[r] <= u0
@@ -854,19 +833,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 struct MergeArgs {
     const int32_t* row_start;
     const int2* cta_range;
-    const int2* row_cand;
     const int32_t* hdr;
     const float2* part_ml;
     const float* part_o;
     float* out;
-    int Hq, Hkv, G, nseg, rows, ngroups;
+    int Hq, Hkv, G, nseg, rows, ngroups, n_ctas;
 };
 
 constexpr int MERGE_WARPS = 8;
 
 // One CTA per (row, query head).  The candidate parts are the (streaming CTA, consumer group) pairs of the
-// CTAs the streaming kernel listed for the row; a CTA whose range turns out not to meet the row, and a part
-// marked absent, weigh nothing.  Warp w takes a contiguous share of the candidates: a lane reads the statistics
+// streaming CTAs from the first whose unit range ends after the row's first unit to the last whose range starts
+// before the row's end (found by a vote over the CTA ranges, one thread per streaming CTA); a CTA whose range
+// turns out not to meet the row, and a part marked absent, weigh nothing.  Warp w takes a contiguous share of the candidates: a lane reads the statistics
 // of one candidate, the warp takes the largest m of its share, then weighs and adds the candidates' O rows, eight
 // loads in flight; the eight warps' (m, l, O) are combined in a fixed order:
 //   o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
@@ -879,12 +858,25 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
+    __shared__ int s_cand[2];
+    if (tid == 0) { s_cand[0] = 0x7fffffff; s_cand[1] = -1; }
+    __syncthreads();
     pdl_trigger();
     pdl_wait();          // every partial of the streaming kernel is in memory from here on
     const int ra = a.row_start[r], rbd = a.row_start[r + 1];
-    const int2 cand = a.row_cand[r];
-    const int c_lo = cand.x;
-    const int n_cand = (rbd > ra && cand.y >= cand.x) ? (cand.y - cand.x + 1) * a.ngroups : 0;
+    for (int c0 = 0; c0 < a.n_ctas; c0 += 32 * MERGE_WARPS) {
+        const int c = c0 + tid;
+        const int2 rg = (c < a.n_ctas) ? a.cta_range[c] : make_int2(0x7fffffff, -1);
+        const unsigned after = __ballot_sync(0xffffffffu, rg.y > ra);       // ranges that end after the row's start
+        const unsigned before = __ballot_sync(0xffffffffu, rg.x < rbd);     // ranges that start before the row's end
+        if (lane == 0) {
+            if (after) atomicMin(&s_cand[0], c + __ffs(after) - 1);
+            if (before) atomicMax(&s_cand[1], c + 31 - __clz(before));
+        }
+    }
+    __syncthreads();
+    const int c_lo = s_cand[0], c_hi = s_cand[1];
+    const int n_cand = (rbd > ra && c_hi >= c_lo) ? (c_hi - c_lo + 1) * a.ngroups : 0;
     float acc[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
@@ -1101,7 +1093,6 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.row_start = reinterpret_cast<int32_t*>(ws + L.row_start);
     da.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
     da.cta_range = reinterpret_cast<int2*>(ws + L.cta_range);
-    da.row_cand = reinterpret_cast<int2*>(ws + L.row_cand);
     da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
     da.part_o = reinterpret_cast<float*>(ws + L.part_o);
     da.status = status_dev;
@@ -1127,8 +1118,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     profile_mark(4, s);
 
     MergeArgs ma;
-    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.cta_range = da.cta_range; ma.row_cand = da.row_cand; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
-    ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS;
+    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.cta_range = da.cta_range; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
+    ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS; ma.n_ctas = n_ctas;
     const unsigned mgrid = (unsigned)(L.rows * G);
     cudaError_t me = (D == 128) ? launch_pdl(merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
                                 : launch_pdl(merge_kernel<64>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma);

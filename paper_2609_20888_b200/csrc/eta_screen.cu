@@ -17,6 +17,7 @@
 // segments: this kernel only leaves per-segment window statistics (admitted
 // count, largest bound and its index per head); the streaming kernel combines
 // them when it lays out its work.
+#include <stdlib.h>
 #include "eta_common.cuh"
 
 namespace eta {
@@ -73,8 +74,16 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     if (tl && tid == 0) tl[0] = globaltimer_ns();
 
     const int n_items = a.rows * a.nseg;
-    const int it0 = (int)(((int64_t)blockIdx.x * n_items) / gridDim.x);
-    const int it1 = (int)(((int64_t)(blockIdx.x + 1) * n_items) / gridDim.x);
+    const int c = blockIdx.x;
+    // a.per_early holds the number of items the first n_early CTAs share evenly; the others take per_late each
+    int it0, it1;
+    if (c < a.n_early) {
+        it0 = (int)(((int64_t)c * a.per_early) / a.n_early);
+        it1 = (int)(((int64_t)(c + 1) * a.per_early) / a.n_early);
+    } else {
+        it0 = min(n_items, a.per_early + (c - a.n_early) * a.per_late);
+        it1 = min(n_items, it0 + a.per_late);
+    }
     const int cc = lane % LPR, rg = lane / LPR;
     const int my_g = cc % G;
 
@@ -119,11 +128,9 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     };
     // The summaries and thresholds may still be in the making when this kernel starts (programmatic dependent
     // launch): the append kernel writes the record and the norm of a block that has just filled up, the predictor
-    // writes tau.  Everything else this kernel reads is final, so only an item that holds a row's newest block of
-    // a just-completed length must wait before its copies; the thresholds are read in phase 2, after the wait.
-    auto safe_item = [&](const Geom& g) {
-        return !(g.n_rec > 0 && (g.T & (a.b - 1)) == 0 && g.j0 + g.n_rec == g.NB);
-    };
+    // writes tau.  Everything else this kernel reads is final.  Phase 1 therefore never waits: the one record per
+    // row that may be stale (the newest block of a just-completed length) gets a bound there like any other, and
+    // the warp that handles its item in phase 2, after the wait, recomputes that bound from global memory.
     auto load_mn = [&](const Geom& g) {        // largest-norm entry of record `tid` of the item
         return (tid < g.n_rec && !dense) ? __ldg(a.mnorm + (int64_t)g.r * a.nb_cap + g.j0 + tid) : 0.f;
     };
@@ -132,7 +139,6 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     int q_row = -1;
     bool waited = false;
     Geom gc = item_geom(it0);
-    if (!safe_item(gc)) { pdl_wait(); waited = true; }
     if (tid == 0) issue(gc, 0);
     {
         const float mn0 = load_mn(gc);
@@ -152,7 +158,6 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
             float mn_next = 0.f;
             if (item + 1 < it1) {
                 gn = item_geom(item + 1);
-                if (!waited && !safe_item(gn)) { pdl_wait(); waited = true; }
                 if (tid == 0) issue(gn, buf ^ 1);
                 mn_next = load_mn(gn);
             }
@@ -271,11 +276,61 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
             float te_l = -INFINITY;
             if (!dense && lane < G) {
                 const int h = g.hk * G + lane;
-                te_l = (a.tau ? __ldg(a.tau + (int64_t)g.i * a.Hq + h) : __ldg(a.head_const + h)) - a.a;
+                te_l = (a.tau ? __ldcg(a.tau + (int64_t)g.i * a.Hq + h) : __ldg(a.head_const + h)) - a.a;
             }
             float te_g[G];
 #pragma unroll
             for (int gq = 0; gq < G; ++gq) te_g[gq] = __shfl_sync(0xffffffffu, te_l, gq);
+            // The record of a block that filled up with the newest token was possibly copied before the append kernel
+            // wrote it: its bound is computed again here, from global memory past the L1, with the arithmetic (and
+            // the order of the sums) of phase 1.
+            if (!dense && ok && n_rec > 0 && (g.T & (a.b - 1)) == 0 && j0 + n_rec == NB) {
+                const int rec = n_rec - 1;
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
+                                           ((int64_t)r * a.nb_cap + j0 + rec) * REC_BYTES;
+                const int cl = lane % LPR;
+                const uint4 m4 = __ldcg(reinterpret_cast<const uint4*>(src + cl * 16));
+                const uint4 s4 = __ldcg(reinterpret_cast<const uint4*>(src + 2 * D + cl * 16));
+                const float mn = __ldcg(a.mnorm + (int64_t)r * a.nb_cap + j0 + rec);
+                const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw[4] = {s4.x, s4.y, s4.z, s4.w};
+                float mu[8], s2[8];
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw[kk]));
+                    float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
+                    mu[2 * kk] = mf.x; mu[2 * kk + 1] = mf.y;
+                    s2[2 * kk] = USE_Q2 ? sf.x * sf.x : sf.x;
+                    s2[2 * kk + 1] = USE_Q2 ? sf.y * sf.y : sf.y;
+                }
+#pragma unroll
+                for (int gq = 0; gq < G; ++gq) {
+                    const uint4 qv = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)g.i * a.Hq + g.hk * G + gq) * D) + cl);
+                    const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
+                    float dot = 0.f, var = 0.f, n2 = 0.f;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const float x = (kk & 1) ? bf16_hi(qw[kk >> 1]) : bf16_lo(qw[kk >> 1]);
+                        n2 = fmaf(x, x, n2);
+                        dot = fmaf(x, mu[kk], dot);
+                        if (USE_Q2) {
+                            var = fmaf(x * x, s2[kk], var);
+                        } else {
+                            const float t = x * s2[kk];
+                            var = fmaf(t, t, var);
+                        }
+                    }
+#pragma unroll
+                    for (int sh = 1; sh < LPR; sh <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, sh);
+#pragma unroll
+                    for (int sh = LPR / 2; sh >= 1; sh >>= 1) {
+                        dot += __shfl_xor_sync(0xffffffffu, dot, sh);
+                        var += __shfl_xor_sync(0xffffffffu, var, sh);
+                    }
+                    if (lane == 0)
+                        sbound_all[slot * SEG + rec][gq] = a.scale * min_keep_nan(dot + a.z * sqrtf(var), sqrtf(n2) * mn);
+                }
+                __syncwarp();
+            }
             if (seg == 0) {
                 if (lane < G) a.tau_eff[(int64_t)g.i * a.Hq + g.hk * G + lane] = te_l;
                 if (lane == 0 && a.status) {
@@ -397,11 +452,26 @@ static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream
         if (e != cudaSuccess) { set_cuda_error(e, "screen smem attribute"); return ETA_ERR_CUDA; }
         configured = true;
     }
-    // every CTA gets the same number of items (the last ones one fewer): the slowest CTA sets the kernel's end
+    // The slowest CTA sets the kernel's end.  All CTAs are resident at once (two per SM), but under programmatic
+    // dependent launch the kernel starts while its predecessors (summary append, threshold predictor) still hold
+    // some SMs, where only one of the two CTAs fits until they exit: the CTAs dispatched last (the highest
+    // indices) start a few microseconds late, so they are given fewer items.
     const int n_items = rows * a.nseg;
     const int per_cta = (n_items + n_ctas - 1) / n_ctas;
-    const int grid = (n_items + per_cta - 1) / per_cta;
-    cudaError_t e = launch_pdl(screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, a);
+    int grid = (n_items + per_cta - 1) / per_cta;
+    ScreenArgs b2 = a;
+    int n_late = 0;
+    if (pdl_enabled() && !getenv("ETA_NO_LATE")) {
+        const int batch = rows / a.Hkv;
+        n_late = (rows + 3) / 4 + (a.tau ? 8 * batch : 0);      // CTAs of the append and of the predictor kernel
+        if (n_late > grid / 4) n_late = grid / 4;
+    }
+    b2.per_late = per_cta > 2 ? per_cta - 2 : 1;
+    if (n_late == 0 || per_cta < 3) { n_late = 0; b2.per_late = per_cta; }
+    b2.n_early = grid - n_late;
+    b2.per_early = n_items - n_late * b2.per_late;
+    if (b2.per_early < 0) { b2.per_early = n_items; b2.n_early = grid; }
+    cudaError_t e = launch_pdl(screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, b2);
     if (e != cudaSuccess) { set_cuda_error(e, "screen launch"); return ETA_ERR_CUDA; }
     return check_launch("screen");
 }
