@@ -187,8 +187,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     int* cnt32 = reinterpret_cast<int*>(smem);                 // [rows] surviving blocks of the row
     int* resc_j = cnt32 + MAX_ROWS;                            // [rows][8] rescued block per head, -1: none
     int* s_len = resc_j + 8 * MAX_ROWS;                        // [rows] clamped sequence length
-    uint8_t* cnt8 = reinterpret_cast<uint8_t*>(s_len + MAX_ROWS);   // [rows * nseg] survivors per segment
-    const bool counts_in_smem = (size_t)a.rows * a.nseg + 10 * 4 * MAX_ROWS <= (size_t)NSTAGE * L::STAGE_BYTES;
+    int* nzp = s_len + MAX_ROWS;                               // [rows] rows with at least one unit before the row
+    uint8_t* cnt8 = reinterpret_cast<uint8_t*>(nzp + MAX_ROWS);     // [rows * nseg] survivors per segment
+    const bool counts_in_smem = (size_t)a.rows * a.nseg + 11 * 4 * MAX_ROWS <= (size_t)NSTAGE * L::STAGE_BYTES;
     // sequence lengths are a caller input: they can be read while the previous kernel is still running
     for (int rr = tid; rr < a.rows; rr += NTHREADS) {
         const int T = __ldg(a.seq_lens + a.div_hkv.div(rr));
@@ -197,10 +198,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
     __syncthreads();
     pdl_wait();          // the screening kernel's lists, counts and window statistics are complete from here on
+    if (tl && tid == 0) tl[7] = globaltimer_ns();
 
     // ---- every CTA lays out the flattened unit sequence for itself: per row the surviving blocks of its
     // segments, then its rescued blocks, then its tail; a scan over the rows gives each row's first unit
-    int nz_rows = 0;      // rows that have at least one unit
+    __shared__ int s_lay[3];      // rows that have at least one unit; the CTA's unit range
     {
         __shared__ int s_wsum[32];
         // all loads of the layout are independent and issued together: segment counts (summed per row with
@@ -228,85 +230,119 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             resc_j[rr * 8 + g] = rescue_of(a.seg_resc, rr, g, a.G, a.nseg, min(a.rescue_window, NB));
         }
         __syncthreads();
-        for (int rr = tid; rr < a.rows; rr += NTHREADS) {
-            const int tailf = (s_len[rr] % a.b) ? 1 : 0;
-            // heads that rescue the same block share one unit
-            int resc = 0, extra = 0;
+        // units of row rr (surviving blocks, rescued blocks, tail); heads that rescue the same block share one unit
+        auto row_units = [&](int rr) {
+            const int tailf = (s_len[rr] & (a.b - 1)) ? 1 : 0;
+            int resc = 0;
             for (int g = 0; g < a.G; ++g) {
                 const int j = resc_j[rr * 8 + g];
                 if (j < 0) continue;
                 bool dup = false;
                 for (int g2 = 0; g2 < g; ++g2) dup = dup || (resc_j[rr * 8 + g2] == j);
                 if (!dup) ++resc;
-                if (blockIdx.x == 0) {
-                    // the first CTA publishes the rescued heads' admission bits
-                    uint8_t* mp = a.sel_mask + (int64_t)rr * a.nb_cap + j;
-                    const unsigned w = *mp;
-                    if (w == 0) ++extra;          // a block no head had admitted: one more block fetched
-                    *mp = (uint8_t)(w | (1u << g));
-                }
             }
             rowinfo[rr] = (uint8_t)(resc | (tailf << 7));
-            const int c = cnt32[rr];
-            rowbase[rr] = c + resc + tailf;          // units of the row; turned into the prefix below
-            if (blockIdx.x == 0 && a.stats) a.stats[rr] = c + extra;
-        }
-        __syncthreads();
-        // exclusive block scan over the rows: value of row rr from get(rr), prefix handed to put(rr, prefix)
-        auto scan_rows = [&](auto get, auto put) {
-            int carry = 0;
-            for (int r0 = 0; r0 < a.rows; r0 += NTHREADS) {
-                const int rr = r0 + tid;
-                const int c = (rr < a.rows) ? get(rr) : 0;
-                int incl = c;
+            return cnt32[rr] + resc + tailf;
+        };
+        if (a.rows <= 32) {
+            // one warp lays out up to 32 rows in registers: no block-wide barrier until the split is known
+            if (warp == 0) {
+                const int units = lane < a.rows ? row_units(lane) : 0;
+                const int nzf = units > 0 ? 1 : 0;
+                int iu = units, iz = nzf;
 #pragma unroll
                 for (int s = 1; s < 32; s <<= 1) {
-                    const int o = __shfl_up_sync(0xffffffffu, incl, s);
-                    if (lane >= s) incl += o;
+                    const int ou = __shfl_up_sync(0xffffffffu, iu, s);
+                    const int oz = __shfl_up_sync(0xffffffffu, iz, s);
+                    if (lane >= s) { iu += ou; iz += oz; }
                 }
-                if (lane == 31) s_wsum[warp] = incl;
-                __syncthreads();
-                int wbase = 0, tot = 0;
-                for (int w = 0; w < NWARPS; ++w) {
-                    const int v = s_wsum[w];
-                    if (w < warp) wbase += v;
-                    tot += v;
-                }
-                if (rr < a.rows) put(rr, carry + wbase + incl - c);
-                carry += tot;
-                __syncthreads();
+                if (lane < a.rows) { rowbase[lane] = iu - units; nzp[lane] = iz - nzf; }
+                if (lane == 31) { rowbase[a.rows] = iu; s_lay[0] = iz; }
             }
-            return carry;
-        };
-        // cnt32 (scratch) <- rows with at least one unit before row rr; rowbase <- units before row rr
-        const int nz_total = scan_rows([&](int rr) { return rowbase[rr] > 0 ? 1 : 0; },
-                                       [&](int rr, int p) { cnt32[rr] = p; });
-        const int u_total = scan_rows([&](int rr) { return rowbase[rr]; }, [&](int rr, int p) { rowbase[rr] = p; });
-        if (tid == 0) { rowbase[a.rows] = u_total; s_wsum[0] = nz_total; }
-        __syncthreads();
-        nz_rows = s_wsum[0];
+        } else {
+            for (int rr = tid; rr < a.rows; rr += NTHREADS) rowbase[rr] = row_units(rr);
+            __syncthreads();
+            // exclusive block scan over the rows: value of row rr from get(rr), prefix handed to put(rr, prefix)
+            auto scan_rows = [&](auto get, auto put) {
+                int carry = 0;
+                for (int r0 = 0; r0 < a.rows; r0 += NTHREADS) {
+                    const int rr = r0 + tid;
+                    const int c = (rr < a.rows) ? get(rr) : 0;
+                    int incl = c;
+#pragma unroll
+                    for (int s = 1; s < 32; s <<= 1) {
+                        const int o = __shfl_up_sync(0xffffffffu, incl, s);
+                        if (lane >= s) incl += o;
+                    }
+                    if (lane == 31) s_wsum[warp] = incl;
+                    __syncthreads();
+                    int wbase = 0, tot = 0;
+                    for (int w = 0; w < NWARPS; ++w) {
+                        const int v = s_wsum[w];
+                        if (w < warp) wbase += v;
+                        tot += v;
+                    }
+                    if (rr < a.rows) put(rr, carry + wbase + incl - c);
+                    carry += tot;
+                    __syncthreads();
+                }
+                return carry;
+            };
+            // nzp <- rows with at least one unit before row rr; rowbase <- units before row rr
+            const int nz_total = scan_rows([&](int rr) { return rowbase[rr] > 0 ? 1 : 0; },
+                                           [&](int rr, int p) { nzp[rr] = p; });
+            const int u_total = scan_rows([&](int rr) { return rowbase[rr]; }, [&](int rr, int p) { rowbase[rr] = p; });
+            if (tid == 0) { rowbase[a.rows] = u_total; s_lay[0] = nz_total; }
+            __syncthreads();
+        }
     }
-    const int U = rowbase[a.rows];
     const int P = gridDim.x;
     // Equal shares of COST, not of units: a row that starts inside a CTA's range costs that CTA a flush of its
     // partials and a query reload, worth about PIECE_COST tiles.  Row rr spans the cost interval
-    // [rowbase[rr] + PIECE_COST * cnt32[rr], +PIECE_COST (if it has units) + its units).
-    auto cost_to_unit = [&](int64_t x) {
-        int lo = 0, hi = a.rows;         // last rr in [0, rows] with cost_start(rr) <= x
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            const int nzb = (mid < a.rows) ? cnt32[mid] : nz_rows;
-            if ((int64_t)rowbase[mid] + (int64_t)PIECE_COST * nzb <= x) lo = mid; else hi = mid - 1;
+    // [rowbase[rr] + PIECE_COST * nzp[rr], +PIECE_COST (if it has units) + its units).  Two lanes of the first
+    // warp find the CTA's two range ends; everybody else picks them up after the barrier.
+    if (warp == 0) {
+        __syncwarp();
+        const int nz_rows = s_lay[0], U = rowbase[a.rows];
+        auto cost_to_unit = [&](int64_t x) {
+            int lo = 0, hi = a.rows;         // last rr in [0, rows] with cost_start(rr) <= x
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                const int nzb = (mid < a.rows) ? nzp[mid] : nz_rows;
+                if ((int64_t)rowbase[mid] + (int64_t)PIECE_COST * nzb <= x) lo = mid; else hi = mid - 1;
+            }
+            if (lo >= a.rows) return U;
+            const int units = rowbase[lo + 1] - rowbase[lo];
+            int64_t off = x - ((int64_t)rowbase[lo] + (int64_t)PIECE_COST * nzp[lo]) - (units > 0 ? PIECE_COST : 0);
+            off = off < 0 ? 0 : (off > units ? units : off);
+            return rowbase[lo] + (int)off;
+        };
+        if (lane < 2) {
+            const int64_t C = (int64_t)U + (int64_t)PIECE_COST * nz_rows;
+            const int c = blockIdx.x + lane;
+            s_lay[1 + lane] = (c == P) ? U : cost_to_unit((c * C) / P);
         }
-        if (lo >= a.rows) return U;
-        const int units = rowbase[lo + 1] - rowbase[lo];
-        int64_t off = x - ((int64_t)rowbase[lo] + (int64_t)PIECE_COST * cnt32[lo]) - (units > 0 ? PIECE_COST : 0);
-        off = off < 0 ? 0 : (off > units ? units : off);
-        return rowbase[lo] + (int)off;
-    };
-    const int64_t C = (int64_t)U + (int64_t)PIECE_COST * nz_rows;
-    const int u0 = cost_to_unit((blockIdx.x * C) / P);
-    const int u1 = (blockIdx.x + 1 == P) ? U : cost_to_unit(((blockIdx.x + 1) * C) / P);
+    }
+    if (blockIdx.x == 0 && warp >= 1) {
+        // the first CTA publishes the rescued heads' admission bits and the number of blocks fetched per row
+        for (int rr = tid - 32; rr < a.rows; rr += NTHREADS - 32) {
+            int extra = 0;
+            for (int g = 0; g < a.G; ++g) {
+                const int j = resc_j[rr * 8 + g];
+                if (j < 0) continue;
+                uint8_t* mp = a.sel_mask + (int64_t)rr * a.nb_cap + j;
+                const unsigned w = *mp;
+                bool dup = false;
+                for (int g2 = 0; g2 < g; ++g2) dup = dup || (resc_j[rr * 8 + g2] == j);
+                if (w == 0 && !dup) ++extra;      // a block no head had admitted: one more block fetched
+                *mp = (uint8_t)(w | (1u << g));
+            }
+            if (a.stats) a.stats[rr] = cnt32[rr] + extra;
+        }
+    }
+    __syncthreads();
+    const int U = rowbase[a.rows];
+    const int u0 = s_lay[1], u1 = s_lay[2];
     if (blockIdx.x == 0) {
         // the merge kernel reads the row ranges and the split from memory
         for (int rr = tid; rr <= a.rows; rr += 32 * (WARPS_PER_GROUP * NGROUPS + 1)) a.row_start[rr] = rowbase[rr];
@@ -484,7 +520,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         int nb = batch_size(u);
         int c_row, c_ent, c_nrows;
         fetch(u, nb, c_row, c_ent, c_nrows);
-        if (tl && lane == 0) tl[7] = globaltimer_ns() + (c_ent & 0);
         while (u < u1 && ok) {
             // the next batch is fetched once the first tiles of this batch are on their way, so that its loads
             // are in flight while the rest of this batch is issued

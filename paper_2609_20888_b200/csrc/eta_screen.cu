@@ -17,7 +17,6 @@
 // segments: this kernel only leaves per-segment window statistics (admitted
 // count, largest bound and its index per head); the streaming kernel combines
 // them when it lays out its work.
-#include <stdlib.h>
 #include "eta_common.cuh"
 
 namespace eta {
@@ -223,10 +222,12 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                             float dot = 0.f, var = 0.f;
 #pragma unroll
                             for (int kk = 0; kk < 8; ++kk) {
-                                dot = fmaf(qf[g][kk], mu[kk], dot);
                                 if (USE_Q2) {
-                                    var = fmaf(q2[g][kk], s2[kk], var);
+                                    // (dot, var) += (q, q^2) * (mu, sigma^2): one packed instruction, each half
+                                    // rounded like a scalar fma
+                                    fma2(dot, var, qf[g][kk], q2[g][kk], mu[kk], s2[kk]);
                                 } else {
+                                    dot = fmaf(qf[g][kk], mu[kk], dot);
                                     const float t = qf[g][kk] * s2[kk];
                                     var = fmaf(t, t, var);
                                 }
@@ -263,7 +264,9 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         }
 
         // ------------------------------------------------------------ phase 2: a warp per item of the group
+        if (tl && tid == 0 && !waited) tl[2] = globaltimer_ns();
         if (!waited) { pdl_wait(); waited = true; }       // the thresholds (and the newest summaries) are final now
+        if (tl && tid == 0 && gs == it0) tl[3] = globaltimer_ns();
         if (gs + warp < ge) {
             const int slot = warp;
             const Geom g = item_geom(gs + slot);
@@ -452,25 +455,38 @@ static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream
         if (e != cudaSuccess) { set_cuda_error(e, "screen smem attribute"); return ETA_ERR_CUDA; }
         configured = true;
     }
-    // The slowest CTA sets the kernel's end.  All CTAs are resident at once (two per SM), but under programmatic
-    // dependent launch the kernel starts while its predecessors (summary append, threshold predictor) still hold
-    // some SMs, where only one of the two CTAs fits until they exit: the CTAs dispatched last (the highest
-    // indices) start a few microseconds late, so they are given fewer items.
+    // The slowest CTA sets the kernel's end.  All CTAs are resident at once (n_ctas = two per SM), but under
+    // programmatic dependent launch the kernel starts while its predecessors (summary append, threshold predictor)
+    // still hold some SMs, where no CTA of this kernel fits until they exit: the CTAs dispatched last (the
+    // highest indices) start late and get two items fewer (measured at G = 4, D = 128: giving them three or four
+    // fewer evens out the mean end time but leaves some early CTAs with one item more, which ends later).
+    // With x items for an early CTA all end together when  n_early x + n_late (x - 2) = n_items.
     const int n_items = rows * a.nseg;
-    const int per_cta = (n_items + n_ctas - 1) / n_ctas;
-    int grid = (n_items + per_cta - 1) / per_cta;
     ScreenArgs b2 = a;
-    int n_late = 0;
-    if (pdl_enabled() && !getenv("ETA_NO_LATE")) {
+    int grid = 0, n_late = 0;
+    if (pdl_enabled()) {
         const int batch = rows / a.Hkv;
-        n_late = (rows + 3) / 4 + (a.tau ? 8 * batch : 0);      // CTAs of the append and of the predictor kernel
-        if (n_late > grid / 4) n_late = grid / 4;
+        n_late = 2 * ((rows + 3) / 4 + (a.tau ? 8 * batch : 0));      // two slots per CTA of the append / predictor kernel
+        if (n_late > n_ctas / 3) n_late = n_ctas / 3;
     }
-    b2.per_late = per_cta > 2 ? per_cta - 2 : 1;
-    if (n_late == 0 || per_cta < 3) { n_late = 0; b2.per_late = per_cta; }
-    b2.n_early = grid - n_late;
-    b2.per_early = n_items - n_late * b2.per_late;
-    if (b2.per_early < 0) { b2.per_early = n_items; b2.n_early = grid; }
+    const int x = (n_items + 2 * n_late + n_ctas - 1) / n_ctas;
+    if (n_late > 0 && x >= 3) {
+        grid = n_ctas;
+        b2.per_late = x - 2;
+        b2.n_early = grid - n_late;
+        b2.per_early = n_items - n_late * b2.per_late;       // shared evenly by the early CTAs
+        if (b2.per_early < b2.n_early) n_late = 0;
+    } else {
+        n_late = 0;
+    }
+    if (n_late == 0) {
+        // every CTA gets the same number of items (the last ones one fewer)
+        const int per_cta = (n_items + n_ctas - 1) / n_ctas;
+        grid = (n_items + per_cta - 1) / per_cta;
+        b2.per_late = per_cta;
+        b2.n_early = grid;
+        b2.per_early = n_items;
+    }
     cudaError_t e = launch_pdl(screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, b2);
     if (e != cudaSuccess) { set_cuda_error(e, "screen launch"); return ETA_ERR_CUDA; }
     return check_launch("screen");
