@@ -120,6 +120,19 @@ int eta_append_summary(const eta_cache_desc* desc, const void* K, const int32_t*
                        void* musig, float* mnorm, uint32_t flags, void* stream);
 
 /*
+ * Brings one step's queries (Algorithm 3, "Require: query q_t") from the host to the device with a kernel
+ * instead of a copy engine (deployment plumbing; the paper has no counterpart).  q_host: bf16
+ * [batch, n_q_heads, head_dim] in page-locked host memory that the device can address (cudaHostAlloc /
+ * cudaHostRegister; with unified addressing the host pointer itself); q_dev: the same shape in device memory.
+ * Both 16-byte aligned, the size a multiple of 16 bytes (else ETA_ERR_UNSUPPORTED).  Ordered like any kernel on
+ * `stream`; the calls that follow on the stream see the complete copy.  The host buffer must stay unchanged until
+ * the kernel has run.  In the same way `out` of eta_decode may be page-locked host memory: the merge kernel's
+ * stores then go straight to the host and are visible once the stream has been synchronised.
+ */
+int eta_stage_query(int32_t batch, int32_t n_q_heads, int32_t head_dim, const void* q_host, void* q_dev,
+                    void* stream);
+
+/*
  * Eq. tau_pred: tau[i, h] = sum_r qbar[i, r] * W[r, h] + bias[h], with qbar the
  * head-major concatenation of the n_q_heads post-RoPE query vectors of sequence
  * i (length n_q_heads * head_dim).  q bf16 [batch, n_q_heads, head_dim];

@@ -20,7 +20,7 @@ ETA_FLAG_UNGATE_LAST = 2
 ETA_BUILD_SIGMA_ENVELOPE = 1
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
-EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_predict_threshold",
+EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_stage_query", "eta_predict_threshold",
            "eta_score_dual", "eta_calibration_workspace_bytes", "eta_calibrate_head_const", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
            "eta_profile_kernel_name", "eta_set_pdl", "eta_debug_timeline", "eta_strerror", "eta_last_cuda_error")
 
@@ -60,6 +60,7 @@ def load() -> ctypes.CDLL:
         lib.eta_build_block_summaries.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
         lib.eta_append_summary.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
         lib.eta_predict_threshold.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, f32p, f32p, f32p, vp]
+        lib.eta_stage_query.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
         lib.eta_score_dual.argtypes = [D, P, vp, i32p, vp, f32p, f32p, vp]
         i32 = ctypes.c_int32
         lib.eta_calibration_workspace_bytes.argtypes = [i32, i32, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
@@ -101,6 +102,15 @@ def _dev(t: torch.Tensor | None, dtype=None, name="tensor"):
     if dtype is not None and t.dtype != dtype:
         raise EtaError(f"{name} must be {dtype}, got {t.dtype}")
     return ctypes.c_void_p(t.data_ptr())
+
+
+def _dev_or_pinned(t: torch.Tensor, dtype=None, name="tensor"):
+    """Device pointer of a CUDA tensor, or of a page-locked host tensor (addressable by the device as it is)."""
+    if t is not None and not t.is_cuda and t.is_pinned():
+        if dtype is not None and t.dtype != dtype:
+            raise EtaError(f"{name} must be {dtype}, got {t.dtype}")
+        return ctypes.c_void_p(t.data_ptr())
+    return _dev(t, dtype, name)
 
 
 def _stream():
@@ -160,6 +170,17 @@ def eta_append_summary(desc, K, seq_lens_after, musig, mnorm, flags: int = 0) ->
            "eta_append_summary")
 
 
+def eta_stage_query(q_host, q_dev) -> None:
+    """Copies a step's queries from a page-locked host tensor into `q_dev` with a kernel on the current stream."""
+    if q_host.is_cuda or not q_host.is_pinned():
+        raise EtaError("q_host must be a page-locked host tensor")
+    if q_host.shape != q_dev.shape or q_host.dtype != torch.bfloat16 or not q_host.is_contiguous() or not q_dev.is_contiguous():
+        raise EtaError("q_host and q_dev must be contiguous bf16 tensors of the same shape")
+    B, Hq, d = q_host.shape
+    _check(load().eta_stage_query(B, Hq, d, ctypes.c_void_p(q_host.data_ptr()), _dev(q_dev, torch.bfloat16, "q_dev"),
+                                  _stream()), "eta_stage_query")
+
+
 def eta_predict_threshold(q, W, bias, tau) -> None:
     B, Hq, d = q.shape
     _check(load().eta_predict_threshold(B, Hq, d, _dev(q, torch.bfloat16, "q"), _dev(W, torch.float32, "W"),
@@ -204,7 +225,7 @@ def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau,
                              _dev(K, torch.bfloat16, "K"), _dev(V, torch.bfloat16, "V"),
                              _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
                              _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
-                             _dev(head_const, torch.float32, "head_const"), _dev(out, torch.float32, "out"),
+                             _dev(head_const, torch.float32, "head_const"), _dev_or_pinned(out, torch.float32, "out"),
                              _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),
                              _dev(status, torch.int32, "status"), _dev(workspace, torch.uint8, "workspace"),
                              workspace.numel(), _stream()),
@@ -220,7 +241,7 @@ def eta_decode_static(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnor
                                     _dev(K, torch.bfloat16, "K"), _dev(V, torch.bfloat16, "V"),
                                     _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
                                     _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
-                                    _dev(head_const, torch.float32, "head_const"), _dev(out, torch.float32, "out"),
+                                    _dev(head_const, torch.float32, "head_const"), _dev_or_pinned(out, torch.float32, "out"),
                                     _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),
                                     _dev(status, torch.int32, "status"), _stream()),
            "eta_decode_static")

@@ -34,9 +34,8 @@ struct DecodeArgs {
     const RescueRec* seg_resc;
     uint8_t* sel_mask;
     int32_t* stats;
-    int32_t* row_start;
-    int2* cta_range;
-    int32_t* hdr;
+    int2* row_start;     // [rows + 1] (units, non-empty rows) before the row
+    int32_t* hdr;        // total units, CTAs that share them, non-empty rows
     float2* part_ml;
     float* part_o;
     uint32_t* status;
@@ -202,7 +201,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     // ---- every CTA lays out the flattened unit sequence for itself: per row the surviving blocks of its
     // segments, then its rescued blocks, then its tail; a scan over the rows gives each row's first unit
-    __shared__ int s_lay[3];      // rows that have at least one unit; the CTA's unit range
+    __shared__ int s_lay[4];      // rows that have at least one unit; the CTA's unit range; CTAs that share the units
     {
         __shared__ int s_wsum[32];
         // all loads of the layout are independent and issued together: segment counts (summed per row with
@@ -296,7 +295,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             __syncthreads();
         }
     }
-    const int P = gridDim.x;
     // Equal shares of COST, not of units: a row that starts inside a CTA's range costs that CTA a flush of its
     // partials and a query reload, worth about PIECE_COST tiles.  Row rr spans the cost interval
     // [rowbase[rr] + PIECE_COST * nzp[rr], +PIECE_COST (if it has units) + its units).  Two lanes of the first
@@ -318,9 +316,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             return rowbase[lo] + (int)off;
         };
         if (lane < 2) {
+            // At least four cost units per CTA (fewer CTAs take part in a tiny problem): then no CTA's range is
+            // empty, and the CTAs that meet a row are exactly those between two ends that follow from the row's
+            // cost interval in closed form (the merge kernel finds its candidates that way).
             const int64_t C = (int64_t)U + (int64_t)PIECE_COST * nz_rows;
+            const int P = (int)min((int64_t)gridDim.x, max((int64_t)1, C / 4));
             const int c = blockIdx.x + lane;
-            s_lay[1 + lane] = (c == P) ? U : cost_to_unit((c * C) / P);
+            s_lay[1 + lane] = (c >= P) ? U : cost_to_unit((c * C) / P);
+            if (lane == 0) s_lay[3] = P;
         }
     }
     if (blockIdx.x == 0 && warp >= 1) {
@@ -344,11 +347,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int U = rowbase[a.rows];
     const int u0 = s_lay[1], u1 = s_lay[2];
     if (blockIdx.x == 0) {
-        // the merge kernel reads the row ranges and the split from memory
-        for (int rr = tid; rr <= a.rows; rr += 32 * (WARPS_PER_GROUP * NGROUPS + 1)) a.row_start[rr] = rowbase[rr];
-        if (tid == 0) { a.hdr[0] = U; a.hdr[1] = P; }
+        // the merge kernel reads the rows' unit and non-empty-row prefixes and the split's parameters from memory
+        for (int rr = tid; rr <= a.rows; rr += NTHREADS)
+            a.row_start[rr] = make_int2(rowbase[rr], rr < a.rows ? nzp[rr] : s_lay[0]);
+        if (tid == 0) { a.hdr[0] = U; a.hdr[1] = s_lay[3]; a.hdr[2] = s_lay[0]; }
     }
-    if (tid == 0) a.cta_range[blockIdx.x] = make_int2(u0, u1);      // read by the merge kernel
     if (tl && tid == 0) tl[1] = globaltimer_ns();
     if (u0 >= u1) return;
     // row holding unit u0: last r with rowbase[r] <= u0
@@ -866,23 +869,25 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
 // Associative merge of the pieces of one (sequence, query head): Algorithm 3, global reduction.
 struct MergeArgs {
-    const int32_t* row_start;
-    const int2* cta_range;
+    const int2* row_start;
     const int32_t* hdr;
     const float2* part_ml;
     const float* part_o;
     float* out;
-    int Hq, Hkv, G, nseg, rows, ngroups, n_ctas;
+    int Hq, Hkv, G, nseg, rows, ngroups;
+    unsigned long long* timeline;
 };
 
 constexpr int MERGE_WARPS = 8;
 
 // One CTA per (row, query head).  The candidate parts are the (streaming CTA, consumer group) pairs of the
-// streaming CTAs from the first whose unit range ends after the row's first unit to the last whose range starts
-// before the row's end (found by a vote over the CTA ranges, one thread per streaming CTA); a CTA whose range
-// turns out not to meet the row, and a part marked absent, weigh nothing.  Warp w takes a contiguous share of the candidates: a lane reads the statistics
-// of one candidate, the warp takes the largest m of its share, then weighs and adds the candidates' O rows, eight
-// loads in flight; the eight warps' (m, l, O) are combined in a fixed order:
+// streaming CTAs that hold units of the row.  Those CTAs follow from the split in closed form: CTA c has the cost
+// interval [floor(c C / P), floor((c + 1) C / P)), the row the interval [cs, ce) whose first PIECE_COST units are
+// padding, and (every CTA having at least four cost units) c holds units of the row exactly when its interval
+// starts before ce and ends after the padding.  A part marked absent weighs nothing.  Warp w takes a contiguous
+// share of the candidates: a lane reads the statistics of one candidate while the candidates' O rows are already
+// on their way (eight in flight), the warp takes the largest m of its share, weighs and adds the rows; the eight
+// warps' (m, l, O) are combined in a fixed order:
 //   o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
 template <int D>
 __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs a) {
@@ -893,25 +898,24 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
-    __shared__ int s_cand[2];
-    if (tid == 0) { s_cand[0] = 0x7fffffff; s_cand[1] = -1; }
-    __syncthreads();
+    unsigned long long* tl = (a.timeline && blockIdx.x < 200) ? a.timeline + (size_t)(808 + blockIdx.x) * 8 : nullptr;
+    if (tl && tid == 0) tl[0] = globaltimer_ns();
     pdl_trigger();
     pdl_wait();          // every partial of the streaming kernel is in memory from here on
-    const int ra = a.row_start[r], rbd = a.row_start[r + 1];
-    for (int c0 = 0; c0 < a.n_ctas; c0 += 32 * MERGE_WARPS) {
-        const int c = c0 + tid;
-        const int2 rg = (c < a.n_ctas) ? a.cta_range[c] : make_int2(0x7fffffff, -1);
-        const unsigned after = __ballot_sync(0xffffffffu, rg.y > ra);       // ranges that end after the row's start
-        const unsigned before = __ballot_sync(0xffffffffu, rg.x < rbd);     // ranges that start before the row's end
-        if (lane == 0) {
-            if (after) atomicMin(&s_cand[0], c + __ffs(after) - 1);
-            if (before) atomicMax(&s_cand[1], c + 31 - __clz(before));
-        }
+    if (tl && tid == 0) tl[1] = globaltimer_ns();
+    const int2 r0 = a.row_start[r], r1 = a.row_start[r + 1];
+    const int U = a.hdr[0], P = a.hdr[1], nz_rows = a.hdr[2];
+    const int units = r1.x - r0.x;
+    int c_lo = 0, n_cand = 0;
+    if (units > 0) {
+        const int64_t C = (int64_t)U + (int64_t)PIECE_COST * nz_rows;
+        const int64_t cs = (int64_t)r0.x + (int64_t)PIECE_COST * r0.y, ce = cs + PIECE_COST + units;
+        const int c_hi = (int)((ce * P - 1) / C);
+        c_lo = (int)(((cs + PIECE_COST + 1) * P + C - 1) / C) - 1;
+        n_cand = (c_hi - c_lo + 1) * a.ngroups;
     }
-    __syncthreads();
-    const int c_lo = s_cand[0], c_hi = s_cand[1];
-    const int n_cand = (rbd > ra && c_hi >= c_lo) ? (c_hi - c_lo + 1) * a.ngroups : 0;
+    if (tl && tid == 0) tl[2] = globaltimer_ns() + (n_cand & 0);
+    auto slot_of = [&](int k) { return ((int64_t)(c_lo + k / a.ngroups) + r) * a.ngroups + k % a.ngroups; };
     float acc[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
@@ -920,15 +924,32 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     const int k_begin = warp * per, k_end = min(n_cand, k_begin + per);
     for (int k0 = k_begin; k0 < k_end; k0 += 32) {
         const int k = k0 + lane;
+        const int nk = min(32, k_end - k0);
         float m_k = -INFINITY, l_k = 0.f;
-        int64_t slot = 0;
         if (k < k_end) {
-            const int c = c_lo + k / a.ngroups;
-            slot = ((int64_t)c + r) * a.ngroups + k % a.ngroups;
-            const int2 rg = __ldg(a.cta_range + c);                // both loads are issued before either is used
-            const float2 ml = a.part_ml[slot * a.G + gq];
-            if (max(rg.x, ra) < min(rg.y, rbd)) { m_k = ml.x; l_k = ml.y; }
+            const float2 ml = a.part_ml[slot_of(k) * a.G + gq];
+            m_k = ml.x; l_k = ml.y;
         }
+        // the first eight O rows of the round do not wait for the statistics
+        float xv[8][VPL];
+        auto load_rows = [&](int j0) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) xv[u][v] = 0.f;
+                if (j0 + u < nk) {
+                    const float* po = a.part_o + (slot_of(k0 + j0 + u) * a.G + gq) * D + lane * VPL;
+                    if (VPL == 4) {
+                        const float4 x = __ldg(reinterpret_cast<const float4*>(po));
+                        xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
+                    } else {
+                        const float2 x = __ldg(reinterpret_cast<const float2*>(po));
+                        xv[u][0] = x.x; xv[u][1] = x.y;
+                    }
+                }
+            }
+        };
+        load_rows(0);
         float m_round = m_k;
 #pragma unroll
         for (int s = 16; s >= 1; s >>= 1) m_round = fmaxf(m_round, __shfl_xor_sync(0xffffffffu, m_round, s));
@@ -943,35 +964,19 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
         for (int s = 16; s >= 1; s >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, s);
         l_w = l_w * rescale + lw;
         m_w = m_new;
-        const int nk = min(32, k_end - k0);
         for (int j0 = 0; j0 < nk; j0 += 8) {
-            float wv[8];
-            float xv[8][VPL];
+            if (j0 > 0) load_rows(j0);
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const int src = min(j0 + u, 31);
-                const float wk = __shfl_sync(0xffffffffu, w, src);
-                const int64_t sk = __shfl_sync(0xffffffffu, slot, src);
-                wv[u] = (j0 + u < nk) ? wk : 0.f;
+                const float wk = __shfl_sync(0xffffffffu, w, min(j0 + u, 31));
+                if (j0 + u < nk && wk != 0.f) {       // an absent part's row is stale memory: never touch it
 #pragma unroll
-                for (int v = 0; v < VPL; ++v) xv[u][v] = 0.f;
-                if (wv[u] != 0.f) {
-                    const float* po = a.part_o + (sk * a.G + gq) * D + lane * VPL;
-                    if (VPL == 4) {
-                        const float4 x = __ldg(reinterpret_cast<const float4*>(po));
-                        xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
-                    } else {
-                        const float2 x = __ldg(reinterpret_cast<const float2*>(po));
-                        xv[u][0] = x.x; xv[u][1] = x.y;
-                    }
+                    for (int v = 0; v < VPL; ++v) acc[v] = fmaf(xv[u][v], wk, acc[v]);
                 }
             }
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-#pragma unroll
-                for (int v = 0; v < VPL; ++v) acc[v] = fmaf(xv[u][v], wv[u], acc[v]);
         }
     }
+    if (tl && tid == 0) tl[3] = globaltimer_ns() + (__float_as_int(acc[0]) & 0);
 #pragma unroll
     for (int v = 0; v < VPL; ++v) s_acc[warp][lane * VPL + v] = acc[v];
     if (lane == 0) { s_l[warp] = l_w; s_m[warp] = m_w; }
@@ -991,6 +996,7 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
         }
         a.out[((int64_t)i * a.Hq + hk * a.G + gq) * D + tid] = l > 0.f ? o / l : 0.f;
     }
+    if (tl && tid == 0) tl[4] = globaltimer_ns();
 }
 
 // ------------------------------------------------------------------ host side
@@ -1125,9 +1131,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     DecodeArgs da;
     da.q = sa.q; da.seq_lens = seq_lens; da.tau_eff = sa.tau_eff; da.seg_list = sa.seg_list;
     da.seg_count = sa.seg_count; da.seg_resc = sa.seg_resc; da.sel_mask = sel_mask; da.stats = stats;
-    da.row_start = reinterpret_cast<int32_t*>(ws + L.row_start);
+    da.row_start = reinterpret_cast<int2*>(ws + L.row_start);
     da.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
-    da.cta_range = reinterpret_cast<int2*>(ws + L.cta_range);
     da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
     da.part_o = reinterpret_cast<float*>(ws + L.part_o);
     da.status = status_dev;
@@ -1153,8 +1158,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     profile_mark(4, s);
 
     MergeArgs ma;
-    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.cta_range = da.cta_range; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
-    ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS; ma.n_ctas = n_ctas;
+    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
+    ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS; ma.timeline = debug_timeline();
     const unsigned mgrid = (unsigned)(L.rows * G);
     cudaError_t me = (D == 128) ? launch_pdl(merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
                                 : launch_pdl(merge_kernel<64>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma);

@@ -10,6 +10,8 @@
 // on scheduling.
 #include <cooperative_groups.h>
 
+#include <stdint.h>
+
 #include "eta_common.cuh"
 
 namespace cg = cooperative_groups;
@@ -69,7 +71,32 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     if (threadIdx.x == 0) pdl_wait();
 }
 
+// Copy of a step's queries from page-locked host memory to device memory by a kernel: for a few tens of
+// kilobytes a kernel's loads over the interconnect cost less than setting up a copy engine.  The kernel never
+// signals its dependents early, so whatever follows it in the stream starts after the copy is complete.
+__global__ void __launch_bounds__(256) stage_query_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n16) {
+    for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n16; k += gridDim.x * blockDim.x) {
+        uint4 v;
+        asm volatile("ld.global.cv.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(src + k));
+        dst[k] = v;
+    }
+}
+
 }  // namespace eta
+
+extern "C" int eta_stage_query(int32_t batch, int32_t n_q_heads, int32_t head_dim, const void* q_host, void* q_dev,
+                               void* stream) {
+    if (!q_host || !q_dev || batch <= 0 || n_q_heads <= 0 || head_dim <= 0) return ETA_ERR_INVALID_ARG;
+    const size_t bytes = (size_t)batch * n_q_heads * head_dim * 2;
+    if (bytes % 16 || ((uintptr_t)q_host & 15) || ((uintptr_t)q_dev & 15)) return ETA_ERR_UNSUPPORTED;
+    if (bytes / 16 > 0x7fffffffu) return ETA_ERR_UNSUPPORTED;
+    const int n16 = (int)(bytes / 16);
+    int grid = (n16 + 255) / 256;
+    if (grid > 296) grid = 296;
+    eta::stage_query_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(q_host),
+                                                                                 static_cast<uint4*>(q_dev), n16);
+    return eta::check_launch("eta_stage_query");
+}
 
 extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t head_dim, const void* q,
                                      const float* W, const float* bias, float* tau, void* stream) {

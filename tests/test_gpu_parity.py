@@ -449,3 +449,40 @@ def test_run_to_run_determinism():
     for o in outs[1:]:
         assert np.array_equal(o[0].view(np.int32), outs[0][0].view(np.int32))
         assert np.array_equal(o[1], outs[0][1])
+
+
+def test_query_staged_from_pinned_memory_and_output_written_to_it():
+    """The host-facing variant of a step: the query is fetched from page-locked host memory by eta_stage_query and
+    the merge kernel stores the output into page-locked host memory.  Same bits as the device-resident step, and the
+    same agreement with the oracle."""
+    eb = _eb()
+    dev = torch.device("cuda:0")
+    sp = wl.CONFIGS["c2_32k"].scaled(4096 + 33, batch=2)
+    w = wl.make_workload(sp)
+    q = w.queries(0)
+    tau, _ = _calibrated_tau(w, q, 0.85)
+    c = cache_of(w)
+    musig, mnorm = orc.block_summaries(c)
+    ref_out, ref_sel, _, status = gpu_decode(q, w.K, w.V, c.seq_lens, sp.block_size, musig, mnorm, tau=tau)
+    assert status == 0
+
+    K, V = w.K.to(dev), w.V.to(dev)
+    st = eb.DecodeState(K, V, sp.n_q_heads, sp.block_size)
+    st.musig.copy_(torch.from_numpy(musig.view(np.int16)).view(torch.float16).to(dev))
+    st.mnorm.copy_(torch.from_numpy(mnorm).to(dev))
+    lens = torch.from_numpy(np.asarray(c.seq_lens, np.int32)).to(dev)
+    tau_d = torch.from_numpy(np.ascontiguousarray(tau, np.float32)).to(dev)
+    q_host = q.contiguous().pin_memory()
+    q_dev = torch.zeros_like(q_host, device=dev)
+    out_host = torch.full((sp.batch, sp.n_q_heads, sp.head_dim), float("nan"), dtype=torch.float32).pin_memory()
+    eb.eta_stage_query(q_host, q_dev)
+    eb.eta_decode(st.desc, eb.DecodeParams(), q_dev, K, V, lens, st.musig, st.mnorm, tau_d, None, out_host,
+                  st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    assert torch.equal(q_dev.cpu().view(torch.int16), q_host.view(torch.int16))
+    assert np.array_equal(out_host.numpy().view(np.int32), ref_out.view(np.int32))
+    assert np.array_equal(st.sel_mask.cpu().numpy(), ref_sel)
+    # and the unaligned / wrong-kind arguments are refused
+    with pytest.raises(eb.EtaError):
+        eb.eta_stage_query(q.contiguous(), q_dev)           # pageable host memory
