@@ -71,11 +71,10 @@ WsLayout ws_layout(const eta_cache_desc* d) {
     L.nseg = (d->nb_cap + SEG - 1) / SEG;
     L.entries = L.rows * (L.nseg + 2);
     size_t off = 0;
-    L.hdr = off;        off = align_up(off + 8 * sizeof(int32_t), 256);
     L.seg_count = off;  off = align_up(off + sizeof(int32_t) * (size_t)L.rows * L.nseg, 256);
     L.seg_list = off;   off = align_up(off + sizeof(int32_t) * (size_t)L.rows * L.nseg * LSTRIDE, 256);
     L.seg_resc = off;   off = align_up(off + sizeof(RescueRec) * (size_t)L.rows * L.nseg * G, 256);
-    L.row_start = off;  off = align_up(off + sizeof(int2) * ((size_t)L.rows + 1), 256);
+    L.row_span = off;   off = align_up(off + sizeof(int2) * (size_t)L.rows, 256);
     L.tau_eff = off;    off = align_up(off + sizeof(float) * (size_t)d->batch * d->n_q_heads, 256);
     size_t slots = ((size_t)MAX_CTAS + L.rows) * DECODE_GROUPS;
     L.part_ml = off;    off = align_up(off + sizeof(float2) * slots * G, 256);

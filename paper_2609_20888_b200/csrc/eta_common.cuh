@@ -39,11 +39,10 @@ struct WsLayout {
     int rows;        // batch * n_kv_heads
     int nseg;        // segments per row
     int entries;     // rows * (nseg + 2): per row its segments, a rescue pseudo-entry and a tail pseudo-entry
-    size_t hdr;         // int32[8]: [0] total units U, [1] streaming CTAs that share them, [2] non-empty rows (written by the streaming kernel)
     size_t seg_count;   // int32 [rows * nseg]
     size_t seg_list;    // int32 [rows * nseg * LSTRIDE]: block index | head bits << 24
     size_t seg_resc;    // {int cnt; float maxb; int arg; int pad} [rows * nseg * G]
-    size_t row_start;   // int2 [rows + 1]: (units, non-empty rows) before each row (written by the streaming kernel)
+    size_t row_span;    // int2 [rows]: first streaming CTA that holds units of the row, number of such CTAs (written by the streaming kernel)
     size_t tau_eff;     // float [batch * n_q_heads]
     size_t part_ml;     // float2 [(MAX_CTAS + rows) * DECODE_GROUPS * G]
     size_t part_o;      // float [(MAX_CTAS + rows) * DECODE_GROUPS * G * d]

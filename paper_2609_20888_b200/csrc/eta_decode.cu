@@ -34,8 +34,7 @@ struct DecodeArgs {
     const RescueRec* seg_resc;
     uint8_t* sel_mask;
     int32_t* stats;
-    int2* row_start;     // [rows + 1] (units, non-empty rows) before the row
-    int32_t* hdr;        // total units, CTAs that share them, non-empty rows
+    int2* row_span;      // [rows] first streaming CTA that holds units of the row, number of such CTAs
     float2* part_ml;
     float* part_o;
     uint32_t* status;
@@ -347,10 +346,23 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int U = rowbase[a.rows];
     const int u0 = s_lay[1], u1 = s_lay[2];
     if (blockIdx.x == 0) {
-        // the merge kernel reads the rows' unit and non-empty-row prefixes and the split's parameters from memory
-        for (int rr = tid; rr <= a.rows; rr += NTHREADS)
-            a.row_start[rr] = make_int2(rowbase[rr], rr < a.rows ? nzp[rr] : s_lay[0]);
-        if (tid == 0) { a.hdr[0] = U; a.hdr[1] = s_lay[3]; a.hdr[2] = s_lay[0]; }
+        // For the merge kernel: the streaming CTAs that hold units of each row.  CTA c has the cost interval
+        // [floor(c C / P), floor((c + 1) C / P)), row rr the interval [cs, ce) whose first PIECE_COST units are
+        // padding, and (every CTA having at least four cost units) c holds units of the row exactly when its
+        // interval starts before ce and ends after the padding.
+        const int64_t C = (int64_t)U + (int64_t)PIECE_COST * s_lay[0];
+        const int64_t P = s_lay[3];
+        for (int rr = tid; rr < a.rows; rr += NTHREADS) {
+            const int units = rowbase[rr + 1] - rowbase[rr];
+            int c_lo = 0, n_span = 0;
+            if (units > 0) {
+                const int64_t cs = (int64_t)rowbase[rr] + (int64_t)PIECE_COST * nzp[rr], ce = cs + PIECE_COST + units;
+                const int c_hi = (int)((ce * P - 1) / C);
+                c_lo = (int)(((cs + PIECE_COST + 1) * P + C - 1) / C) - 1;
+                n_span = c_hi - c_lo + 1;
+            }
+            a.row_span[rr] = make_int2(c_lo, n_span);
+        }
     }
     if (tl && tid == 0) tl[1] = globaltimer_ns();
     if (u0 >= u1) return;
@@ -869,8 +881,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
 // Associative merge of the pieces of one (sequence, query head): Algorithm 3, global reduction.
 struct MergeArgs {
-    const int2* row_start;
-    const int32_t* hdr;
+    const int2* row_span;
     const float2* part_ml;
     const float* part_o;
     float* out;
@@ -881,13 +892,10 @@ struct MergeArgs {
 constexpr int MERGE_WARPS = 8;
 
 // One CTA per (row, query head).  The candidate parts are the (streaming CTA, consumer group) pairs of the
-// streaming CTAs that hold units of the row.  Those CTAs follow from the split in closed form: CTA c has the cost
-// interval [floor(c C / P), floor((c + 1) C / P)), the row the interval [cs, ce) whose first PIECE_COST units are
-// padding, and (every CTA having at least four cost units) c holds units of the row exactly when its interval
-// starts before ce and ends after the padding.  A part marked absent weighs nothing.  Warp w takes a contiguous
-// share of the candidates: a lane reads the statistics of one candidate while the candidates' O rows are already
-// on their way (eight in flight), the warp takes the largest m of its share, weighs and adds the rows; the eight
-// warps' (m, l, O) are combined in a fixed order:
+// streaming CTAs that hold units of the row, which the streaming kernel lists per row; a part marked absent weighs
+// nothing.  Warp w takes a contiguous share of the candidates: a lane reads the statistics of one candidate while
+// the candidates' O rows are already on their way (eight in flight), the warp takes the largest m of its share,
+// weighs and adds the rows; the eight warps' (m, l, O) are combined in a fixed order:
 //   o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
 template <int D>
 __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs a) {
@@ -903,17 +911,8 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     pdl_trigger();
     pdl_wait();          // every partial of the streaming kernel is in memory from here on
     if (tl && tid == 0) tl[1] = globaltimer_ns();
-    const int2 r0 = a.row_start[r], r1 = a.row_start[r + 1];
-    const int U = a.hdr[0], P = a.hdr[1], nz_rows = a.hdr[2];
-    const int units = r1.x - r0.x;
-    int c_lo = 0, n_cand = 0;
-    if (units > 0) {
-        const int64_t C = (int64_t)U + (int64_t)PIECE_COST * nz_rows;
-        const int64_t cs = (int64_t)r0.x + (int64_t)PIECE_COST * r0.y, ce = cs + PIECE_COST + units;
-        const int c_hi = (int)((ce * P - 1) / C);
-        c_lo = (int)(((cs + PIECE_COST + 1) * P + C - 1) / C) - 1;
-        n_cand = (c_hi - c_lo + 1) * a.ngroups;
-    }
+    const int2 span = a.row_span[r];
+    const int c_lo = span.x, n_cand = span.y * a.ngroups;
     if (tl && tid == 0) tl[2] = globaltimer_ns() + (n_cand & 0);
     auto slot_of = [&](int k) { return ((int64_t)(c_lo + k / a.ngroups) + r) * a.ngroups + k % a.ngroups; };
     float acc[VPL];
@@ -1131,8 +1130,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     DecodeArgs da;
     da.q = sa.q; da.seq_lens = seq_lens; da.tau_eff = sa.tau_eff; da.seg_list = sa.seg_list;
     da.seg_count = sa.seg_count; da.seg_resc = sa.seg_resc; da.sel_mask = sel_mask; da.stats = stats;
-    da.row_start = reinterpret_cast<int2*>(ws + L.row_start);
-    da.hdr = reinterpret_cast<int32_t*>(ws + L.hdr);
+    da.row_span = reinterpret_cast<int2*>(ws + L.row_span);
     da.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
     da.part_o = reinterpret_cast<float*>(ws + L.part_o);
     da.status = status_dev;
@@ -1158,7 +1156,7 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     profile_mark(4, s);
 
     MergeArgs ma;
-    ma.row_start = da.row_start; ma.hdr = da.hdr; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
+    ma.row_span = da.row_span; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
     ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS; ma.timeline = debug_timeline();
     const unsigned mgrid = (unsigned)(L.rows * G);
     cudaError_t me = (D == 128) ? launch_pdl(merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
