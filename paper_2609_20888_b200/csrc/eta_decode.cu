@@ -687,6 +687,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             if (end) tl[4] = globaltimer_ns();
         }
 
+        // the next piece's query is requested before the finished piece is flushed: the flush does not read the
+        // query registers, and its barriers and stores hide the load's latency
+        if (!end && new_piece != piece && ds.x != q_row) load_q(ds.x);
         if ((end || new_piece != piece) && piece >= 0) {
             // ---- this group's part of a piece is complete: combine its four warps and store (m, l, O) per head
             float lsum = l_run + __shfl_xor_sync(0xffffffffu, l_run, 1);
