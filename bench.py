@@ -15,6 +15,7 @@ to one GPU and has no exchange step, so scaling is weak by construction.
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import math
 import os
@@ -211,7 +212,7 @@ def run_ours(args):
 
     q_stage = torch.empty_like(q_host[0]).pin_memory()      # fixed page-locked buffer the end-to-end step reads its query from
 
-    def make_step(bias_np, flags=0, profiled=False, host_io=False):
+    def make_step(bias_np, flags=0, profiled=False, host_io=False, host_q=None, host_out=None):
         """One decode step on the query in `static_q`.  With --graph (default) the launches are captured once
         into a CUDA graph and replayed, so the host costs one graph launch per step instead of several kernel
         launches through ctypes; the library calls are the same either way.  With host_io the step starts by
@@ -221,13 +222,16 @@ def run_ours(args):
         params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags,
                                  ctas_per_sm=args.ctas_per_sm)
 
+        host_q = host_io if host_q is None else host_q
+        host_out = host_io if host_out is None else host_out
+
         def launch():
-            if host_io:
+            if host_q:
                 eb.eta_stage_query(q_stage, static_q)
             eb.eta_append_summary(st.desc, Kd, lens_d, st.musig, st.mnorm)
             eb.eta_predict_threshold(static_q, Wd, bias_d, st.tau)
             eb.eta_decode(st.desc, params, static_q, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau, None,
-                          out_host if host_io else st.out, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+                          out_host if host_out else st.out, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
 
         graph = None
         if args.graph or profiled:
@@ -322,14 +326,23 @@ def run_ours(args):
     # first kernel reads the query over the interconnect (eta_stage_query) and the merge kernel stores the output
     # into pinned host memory, which costs less than two copy-engine transfers of a few tens of kilobytes.  Each
     # step is bracketed by events on the launching stream and followed by a host synchronise.
-    step_e2e = make_step(load_bias(sp.name, main_target), host_io=True)
+    io_q = args.e2e_io in ("kernel", "stage")
+    io_out = args.e2e_io in ("kernel", "hostout")
+    step_e2e = make_step(load_bias(sp.name, main_target), host_q=io_q, host_out=io_out) if (io_q or io_out) else step_main
     e2e_ms = 0.0
     for k in range(args.steps):
         flush.fill_(k & 0xff)
         a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a_ev.record()
-        q_stage.copy_(q_host[args.warmup + k])       # this step's query, host to host, into the buffer the graph reads
+        if io_q:
+            # this step's query, host to host, into the buffer the graph reads (a plain memmove: a tensor copy of
+            # more than 32 K elements would wake a thread pool)
+            ctypes.memmove(q_stage.data_ptr(), q_host[args.warmup + k].data_ptr(), q_stage.numel() * 2)
+        else:
+            static_q.copy_(q_host[args.warmup + k], non_blocking=True)
         step_e2e()
+        if not io_out:
+            out_host.copy_(st.out, non_blocking=True)
         b_ev.record()
         torch.cuda.synchronize()
         e2e_ms += a_ev.elapsed_time(b_ev)
@@ -469,6 +482,9 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch the kernels directly every step")
     ap.add_argument("--no-pdl", dest="pdl", action="store_false", help="fully serialise the kernel launches")
+    ap.add_argument("--e2e-io", default="kernel", choices=["kernel", "copy", "stage", "hostout"],
+                    help="end-to-end leg: the step's kernels read the query from / write the output to pinned host "
+                         "memory themselves (kernel), or two copy-engine transfers bracket the device-resident step (copy)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--dry-run", action="store_true", help="exercise the multi-rank host logic on CPU (gloo)")
