@@ -42,7 +42,7 @@ PEAKS = os.path.join(ROOT, "MEASURED_PEAKS.json")
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per launch of the streaming kernel from the ncu capture summarised in
 # profiles/decode_kernel_c3_128k_s90.md (mean of the two captured launches), keyed by (workload, target sparsity).
-NCU_TRAFFIC_BYTES = {("c3_128k", 0.90): 217.0e6}
+NCU_TRAFFIC_BYTES = {("c3_128k", 0.90): 218.2e6}
 
 
 def load_bias(name: str, target: float) -> np.ndarray:
@@ -92,7 +92,7 @@ class ClockSampler(threading.Thread):
 
 
 def algorithmic_bytes(sp, lens, union_blocks: float):
-    """Bytes one step must move ('algorithmic bytes'): summaries of every full block, K and V of the
+    """Algorithmic bytes of one step, i.e. what the method must move: summaries of every full block, K and V of the
     union of surviving blocks and of the tails, queries, thresholds, mask, output.  Split by kernel."""
     d, b, G = sp.head_dim, sp.block_size, sp.gqa
     nb = sum(int(t) // b for t in lens) * sp.n_kv_heads
