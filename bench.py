@@ -169,6 +169,24 @@ def run_ours(args):
     lens_d = w.seq_lens.to(dev)
     Wd = w.W.to(dev)
 
+    # --paged: the same cache scattered over a pool of pages of one block each by a seeded permutation; the step
+    # then runs through the paged entry points (same results bit for bit; tests/test_gpu_paged.py)
+    pdesc = pages = Kp = Vp = None
+    if args.paged:
+        B_, H_, T_, d_ = Kd.shape
+        b_ = sp.block_size
+        assert T_ % b_ == 0, "--paged needs a token capacity that is a multiple of the block size"
+        nbp = T_ // b_
+        gperm = torch.Generator(device=dev).manual_seed(sp.seed + 99)
+        perm = torch.randperm(B_ * nbp, generator=gperm, device=dev)
+        Kp, Vp = torch.empty((B_ * nbp, H_, b_, d_), dtype=Kd.dtype, device=dev), None
+        Kp[perm] = Kd.view(B_, H_, nbp, b_, d_).permute(0, 2, 1, 3, 4).reshape(B_ * nbp, H_, b_, d_)
+        Vp = torch.empty_like(Kp)
+        Vp[perm] = Vd.view(B_, H_, nbp, b_, d_).permute(0, 2, 1, 3, 4).reshape(B_ * nbp, H_, b_, d_)
+        table = perm.view(B_, nbp).to(torch.int32).contiguous()
+        pdesc = eb.paged_cache_desc(Kp, Vp, sp.batch, sp.n_q_heads, t_cap=T_, nb_cap=st.desc.nb_cap)
+        pages = eb.page_table(table, B_ * nbp)
+
     # prefill-side index build (once per sequence; timed on its own, not part of a decode step)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     eb.eta_build_block_summaries(st.desc, Kd, lens_d, st.musig, st.mnorm)
@@ -228,10 +246,17 @@ def run_ours(args):
         def launch():
             if host_q:
                 eb.eta_stage_query(q_stage, static_q)
+            o = out_host if host_out else st.out
+            if pages is not None:
+                eb.eta_append_summary_paged(pdesc, pages, Kp, lens_d, st.musig, st.mnorm)
+                eb.eta_predict_threshold(static_q, Wd, bias_d, st.tau)
+                eb.eta_decode_paged(pdesc, pages, params, static_q, Kp, Vp, lens_d, st.musig, st.mnorm, st.tau, None,
+                                    o, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+                return
             eb.eta_append_summary(st.desc, Kd, lens_d, st.musig, st.mnorm)
             eb.eta_predict_threshold(static_q, Wd, bias_d, st.tau)
             eb.eta_decode(st.desc, params, static_q, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau, None,
-                          out_host if host_out else st.out, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+                          o, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
 
         graph = None
         if args.graph or profiled:
@@ -390,7 +415,8 @@ def run_ours(args):
                        "head_dim": sp.head_dim, "context": sp.context, "block_size": sp.block_size,
                        "target_union_sparsity": main_target, "measured_union_sparsity": 1 - union_main / nb_total,
                        "z": sp.z, "beta": sp.beta, "l2": "flushed between timed steps (384 MiB write)",
-                       "fresh_query_every_step": True, "replicas": world, "cuda_graph": bool(args.graph), "pdl": bool(args.pdl)},
+                       "fresh_query_every_step": True, "replicas": world, "cuda_graph": bool(args.graph), "pdl": bool(args.pdl),
+                       "paged_cache": bool(args.paged), "e2e_io": args.e2e_io},
             "attention_us_per_token": ms_step * 1e3,
             "achieved_gbs_all_kernels": ab["total"] / (ms_step * 1e-3) / 1e9,
             "frac_of_8tbs_nominal": ab["total"] / (ms_step * 1e-3) / 8e12,
@@ -485,6 +511,7 @@ def main():
     ap.add_argument("--e2e-io", default="kernel", choices=["kernel", "copy", "stage", "hostout"],
                     help="end-to-end leg: the step's kernels read the query from / write the output to pinned host "
                          "memory themselves (kernel), or two copy-engine transfers bracket the device-resident step (copy)")
+    ap.add_argument("--paged", action="store_true", help="run the step on a paged copy of the cache (pages scattered by a seeded permutation)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--dry-run", action="store_true", help="exercise the multi-rank host logic on CPU (gloo)")

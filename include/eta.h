@@ -233,6 +233,36 @@ int eta_decode_static(const eta_cache_desc* desc, const eta_params* params, cons
                       const float* tau, const float* head_const,
                       float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev, void* stream);
 
+/*
+ * Paged KV cache (Section 3: the block summaries live "in a held-out table compatible with paged caching").
+ * K and V are pools of pages of block_size tokens; page p of KV head hk, token t of the page, is at
+ * K + p * k_stride_b + hk * k_stride_h + t * k_stride_t (the descriptor's sequence stride becomes the page
+ * stride; same for V).  block_table (device, int32 [batch, table_stride], table_stride >= ceil(t_cap /
+ * block_size)) gives, for sequence i and j >= 0, the page that holds tokens [j * block_size, (j + 1) * block_size)
+ * of the sequence; entries for j up to floor((T_i - 1) / block_size) must be valid page numbers in [0, n_pages)
+ * (the last of them is the partly filled tail page), the others are never read.  The summaries (musig, mnorm) and
+ * sel_mask stay indexed by (sequence, KV head, block) as in the contiguous case: they are the held-out table.
+ * The three calls compute exactly what their contiguous counterparts compute on the gathered cache, bit for bit.
+ * Ownership, alignment, error behaviour: as for the contiguous calls; a NULL table, table_stride too small or
+ * n_pages <= 0 return ETA_ERR_INVALID_ARG.  Page numbers are not range-checked on the device.
+ */
+typedef struct eta_page_table {
+    const int32_t* block_table;
+    int32_t table_stride;
+    int32_t n_pages;
+} eta_page_table;
+
+int eta_build_block_summaries_paged(const eta_cache_desc* desc, const eta_page_table* pages, const void* K_pool,
+                                    const int32_t* seq_lens, void* musig, float* mnorm, uint32_t flags, void* stream);
+int eta_append_summary_paged(const eta_cache_desc* desc, const eta_page_table* pages, const void* K_pool,
+                             const int32_t* seq_lens_after, void* musig, float* mnorm, uint32_t flags, void* stream);
+int eta_decode_paged(const eta_cache_desc* desc, const eta_page_table* pages, const eta_params* params, const void* q,
+                     const void* K_pool, const void* V_pool, const int32_t* seq_lens,
+                     const void* musig, const float* mnorm,
+                     const float* tau, const float* head_const,
+                     float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
 /* Size of the built-in scratch of eta_decode_static, in bytes. */
 size_t eta_static_scratch_bytes(void);
 

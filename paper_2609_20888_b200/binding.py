@@ -20,7 +20,8 @@ ETA_FLAG_UNGATE_LAST = 2
 ETA_BUILD_SIGMA_ENVELOPE = 1
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
-EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_stage_query", "eta_predict_threshold",
+EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_build_block_summaries_paged",
+           "eta_append_summary_paged", "eta_decode_paged", "eta_stage_query", "eta_predict_threshold",
            "eta_score_dual", "eta_calibration_workspace_bytes", "eta_calibrate_head_const", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
            "eta_profile_kernel_name", "eta_set_pdl", "eta_debug_timeline", "eta_strerror", "eta_last_cuda_error")
 
@@ -37,6 +38,10 @@ class Params(ctypes.Structure):
     _fields_ = [("z", ctypes.c_float), ("a", ctypes.c_float), ("beta", ctypes.c_float), ("scale", ctypes.c_float),
                 ("lwb", ctypes.c_int32), ("rescue_window", ctypes.c_int32), ("flags", ctypes.c_uint32),
                 ("ctas_per_sm", ctypes.c_int32)]
+
+
+class PageTable(ctypes.Structure):
+    _fields_ = [("block_table", ctypes.c_void_p), ("table_stride", ctypes.c_int32), ("n_pages", ctypes.c_int32)]
 
 
 class EtaError(RuntimeError):
@@ -59,6 +64,11 @@ def load() -> ctypes.CDLL:
         lib.eta_workspace_bytes.argtypes = [D, ctypes.POINTER(ctypes.c_size_t)]
         lib.eta_build_block_summaries.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
         lib.eta_append_summary.argtypes = [D, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
+        PT = ctypes.POINTER(PageTable)
+        lib.eta_build_block_summaries_paged.argtypes = [D, PT, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
+        lib.eta_append_summary_paged.argtypes = [D, PT, vp, i32p, vp, f32p, ctypes.c_uint32, vp]
+        lib.eta_decode_paged.argtypes = [D, PT, P, vp, vp, vp, i32p, vp, f32p, f32p, f32p, f32p, vp, i32p, vp, vp,
+                                         ctypes.c_size_t, vp]
         lib.eta_predict_threshold.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, f32p, f32p, f32p, vp]
         lib.eta_stage_query.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
         lib.eta_score_dual.argtypes = [D, P, vp, i32p, vp, f32p, f32p, vp]
@@ -144,6 +154,25 @@ def cache_desc(K: torch.Tensor, V: torch.Tensor, n_q_heads: int, block_size: int
                      V.stride(0), V.stride(1), V.stride(2))
 
 
+def paged_cache_desc(K_pool: torch.Tensor, V_pool: torch.Tensor, batch: int, n_q_heads: int, t_cap: int,
+                     nb_cap: int | None = None) -> CacheDesc:
+    """Describe a paged cache: pools of logical shape [n_pages, n_kv_heads, block_size, head_dim] (any strides with
+    unit stride along head_dim); the page size is the block size, the stride of the first axis the page stride."""
+    n_pages, Hkv, b, d = K_pool.shape
+    if K_pool.stride(3) != 1 or V_pool.stride(3) != 1 or V_pool.shape != K_pool.shape:
+        raise EtaError("K_pool and V_pool must have the same shape and unit stride along head_dim")
+    nb = nb_cap if nb_cap is not None else (t_cap + b - 1) // b
+    return CacheDesc(batch, n_q_heads, Hkv, d, b, t_cap, nb, K_pool.stride(0), K_pool.stride(1), K_pool.stride(2),
+                     V_pool.stride(0), V_pool.stride(1), V_pool.stride(2))
+
+
+def page_table(block_table: torch.Tensor, n_pages: int) -> PageTable:
+    """block_table: int32 CUDA tensor [batch, table_stride], page of every block of tokens of every sequence."""
+    if block_table.dim() != 2 or block_table.stride(1) != 1:
+        raise EtaError("block_table must be a 2-D tensor with unit stride along its second axis")
+    return PageTable(_dev(block_table, torch.int32, "block_table"), block_table.stride(0), n_pages)
+
+
 def eta_workspace_bytes(desc: CacheDesc) -> int:
     n = ctypes.c_size_t(0)
     _check(load().eta_workspace_bytes(ctypes.byref(desc), ctypes.byref(n)), "eta_workspace_bytes")
@@ -168,6 +197,22 @@ def eta_append_summary(desc, K, seq_lens_after, musig, mnorm, flags: int = 0) ->
                                      _dev(seq_lens_after, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
                                      _dev(mnorm, torch.float32, "mnorm"), flags, _stream()),
            "eta_append_summary")
+
+
+def eta_build_block_summaries_paged(desc, pages: PageTable, K_pool, seq_lens, musig, mnorm, flags: int = 0) -> None:
+    _check(load().eta_build_block_summaries_paged(ctypes.byref(desc), ctypes.byref(pages), _dev(K_pool, torch.bfloat16, "K_pool"),
+                                                  _dev(seq_lens, torch.int32, "seq_lens"),
+                                                  _dev(musig, torch.float16, "musig"), _dev(mnorm, torch.float32, "mnorm"),
+                                                  flags, _stream()),
+           "eta_build_block_summaries_paged")
+
+
+def eta_append_summary_paged(desc, pages: PageTable, K_pool, seq_lens_after, musig, mnorm, flags: int = 0) -> None:
+    _check(load().eta_append_summary_paged(ctypes.byref(desc), ctypes.byref(pages), _dev(K_pool, torch.bfloat16, "K_pool"),
+                                           _dev(seq_lens_after, torch.int32, "seq_lens"),
+                                           _dev(musig, torch.float16, "musig"), _dev(mnorm, torch.float32, "mnorm"),
+                                           flags, _stream()),
+           "eta_append_summary_paged")
 
 
 def eta_stage_query(q_host, q_dev) -> None:
@@ -230,6 +275,20 @@ def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau,
                              _dev(status, torch.int32, "status"), _dev(workspace, torch.uint8, "workspace"),
                              workspace.numel(), _stream()),
            "eta_decode")
+
+
+def eta_decode_paged(desc, pages: PageTable, params: DecodeParams, q, K_pool, V_pool, seq_lens, musig, mnorm, tau,
+                     head_const, out, sel_mask, workspace, stats=None, status=None) -> None:
+    p = params.c()
+    _check(load().eta_decode_paged(ctypes.byref(desc), ctypes.byref(pages), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
+                                   _dev(K_pool, torch.bfloat16, "K_pool"), _dev(V_pool, torch.bfloat16, "V_pool"),
+                                   _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                   _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
+                                   _dev(head_const, torch.float32, "head_const"), _dev_or_pinned(out, torch.float32, "out"),
+                                   _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),
+                                   _dev(status, torch.int32, "status"), _dev(workspace, torch.uint8, "workspace"),
+                                   workspace.numel(), _stream()),
+           "eta_decode_paged")
 
 
 def eta_decode_static(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,

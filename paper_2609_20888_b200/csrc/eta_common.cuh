@@ -22,6 +22,7 @@ inline int check_launch(const char* where) {
     return ETA_OK;
 }
 int validate_desc(const eta_cache_desc* d);
+int validate_pages(const eta_cache_desc* desc, const eta_page_table* pages);
 // Measurement aid: when profiling is enabled, records timing event k on the stream (see eta_profile_enable).
 void profile_mark(int k, cudaStream_t s);
 

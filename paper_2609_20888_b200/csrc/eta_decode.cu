@@ -41,6 +41,8 @@ struct DecodeArgs {
     float beta, scale;
     int Hq, Hkv, G, b, t_cap, nb_cap, nseg, entries, rows, rescue_window;
     int ungate_last;     // the newest token of every sequence keeps its raw logit (ETA_FLAG_UNGATE_LAST)
+    const int32_t* block_table;   // paged cache: [batch, table_stride] page of every block of tokens; null: contiguous
+    int table_stride;
     FastDiv div_nseg, div_epr, div_hkv, div_g;
     unsigned long long* timeline;
 };
@@ -464,8 +466,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
         };
         // per-lane description of unit ub + lane (row < 0: no such unit in this batch)
-        auto fetch = [&](int ub, int nb, int& row, int& ent, int& nrows) {
-            row = -1; ent = 0; nrows = 0;
+        auto fetch = [&](int ub, int nb, int& row, int& ent, int& nrows, int& page) {
+            row = -1; ent = 0; nrows = 0; page = 0;
             if (lane < nb) {
                 const int uu = ub + lane;
                 const int k = search(uu);
@@ -525,6 +527,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                         if (((ent & 0xffffff) + 1) * a.b == T) nrows |= 0x10000;   // the block the newest token closes
                     }
                 }
+                // paged cache: the page that holds the unit's block of tokens (one more dependent load per batch,
+                // hidden like the list fetch behind the tiles already on their way)
+                if (a.block_table)
+                    page = __ldg(a.block_table + (int64_t)a.div_hkv.div(r) * a.table_stride + (ent & 0xffffff));
             }
         };
 
@@ -533,18 +539,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         if (tl && lane == 0) tl[6] = globaltimer_ns();
         int u = u0;
         int nb = batch_size(u);
-        int c_row, c_ent, c_nrows;
-        fetch(u, nb, c_row, c_ent, c_nrows);
+        int c_row, c_ent, c_nrows, c_page;
+        fetch(u, nb, c_row, c_ent, c_nrows, c_page);
         while (u < u1 && ok) {
             // the next batch is fetched once the first tiles of this batch are on their way, so that its loads
             // are in flight while the rest of this batch is issued
             const int un = u + nb;
-            int nbn = 0, n_row = -1, n_ent = 0, n_nrows = 0;
+            int nbn = 0, n_row = -1, n_ent = 0, n_nrows = 0, n_page = 0;
             const int k_prefetch = min(nb, NSTAGE) - 1;
             for (int k = 0; k < nb && ok; ++k) {
                 const int r = __shfl_sync(0xffffffffu, c_row, k);
                 const int ent = __shfl_sync(0xffffffffu, c_ent, k);
                 const int nrows_raw = __shfl_sync(0xffffffffu, c_nrows, k);
+                const int page = __shfl_sync(0xffffffffu, c_page, k);
                 const int nrows = nrows_raw & 0xffff;
                 const bool holds_newest = (nrows_raw >> 16) != 0;
                 const int j = ent & 0xffffff;
@@ -570,10 +577,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                             desc[stage] = make_int4(r, piece << 1, hmask | (urow << 8), nvalid);
                             unsigned char* st = smem + stage * L::STAGE_BYTES;
                             mbar_arrive_expect_tx(&full[stage], L::STAGE_BYTES);
-                            const int y = j * a.b + sub * TS;
-                            // one copy per tile: 64 columns x TS tokens x HALVES half tiles, each half swizzled
-                            tma_load_5d(st, &tmK, 0, y, 0, hk, i, &full[stage]);
-                            tma_load_5d(st + HALVES * L::TILE_BYTES, &tmV, 0, y, 0, hk, i, &full[stage]);
+                            // one copy per tile: 64 columns x TS tokens x HALVES half tiles, each half swizzled.  The
+                            // outermost coordinate is the sequence (contiguous cache: token offset in the sequence) or
+                            // the page (paged cache: token offset in the page)
+                            const int y = a.block_table ? sub * TS : j * a.b + sub * TS;
+                            const int w4 = a.block_table ? page : i;
+                            tma_load_5d(st, &tmK, 0, y, 0, hk, w4, &full[stage]);
+                            tma_load_5d(st + HALVES * L::TILE_BYTES, &tmV, 0, y, 0, hk, w4, &full[stage]);
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -581,11 +591,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 }
                 if (k == k_prefetch && un < u1) {
                     nbn = batch_size(un);
-                    fetch(un, nbn, n_row, n_ent, n_nrows);
+                    fetch(un, nbn, n_row, n_ent, n_nrows, n_page);
                 }
             }
             u = un;
-            nb = nbn; c_row = n_row; c_ent = n_ent; c_nrows = n_nrows;
+            nb = nbn; c_row = n_row; c_ent = n_ent; c_nrows = n_nrows; c_page = n_page;
         }
         close_piece();
         pdl_trigger();       // everything is issued: the merge kernel may start to set up
@@ -1024,12 +1034,15 @@ static EncodeTiledFn encode_fn() {
 
 // K or V as a 5-D tensor (c within a 64-column half, t, half, hk, i) of bf16; a box is 64 columns x TS tokens x
 // all halves: in shared memory, one 128-byte-swizzled [TS][64] tile per half, back to back.
+// Tensor map of a K or V cache: 64 columns x tokens x column halves x KV heads x sequences, or, for a paged cache
+// (n_pages > 0), ... x tokens of a page x ... x pages, with sb the stride between pages.
 static int make_tmap(CUtensorMap* tm, const void* base, const eta_cache_desc* d, int64_t sb, int64_t sh, int64_t st,
-                     int TS) {
+                     int TS, int n_pages) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return ETA_ERR_CUDA;
     const cuuint32_t halves = (cuuint32_t)(d->head_dim / 64);
-    cuuint64_t dims[5] = {64, (cuuint64_t)d->t_cap, halves, (cuuint64_t)d->n_kv_heads, (cuuint64_t)d->batch};
+    cuuint64_t dims[5] = {64, (cuuint64_t)(n_pages > 0 ? d->block_size : d->t_cap), halves, (cuuint64_t)d->n_kv_heads,
+                          (cuuint64_t)(n_pages > 0 ? n_pages : d->batch)};
     cuuint64_t strides[4] = {(cuuint64_t)st * 2, 128, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
     cuuint32_t box[5] = {64, (cuuint32_t)TS, halves, 1, 1};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
@@ -1060,19 +1073,14 @@ static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const
     return check_launch("decode");
 }
 
-}  // namespace eta
-
-extern "C" {
-
-int eta_decode_kernel_count(void) { return 3; }
-
-int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q, const void* K, const void* V,
-               const int32_t* seq_lens, const void* musig, const float* mnorm, const float* tau,
-               const float* head_const, float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev,
-               void* workspace, size_t workspace_bytes, void* stream) {
-    using namespace eta;
+// eta_decode and eta_decode_paged: `pages` null selects the contiguous cache
+static int decode_impl(const eta_cache_desc* desc, const eta_page_table* pages, const eta_params* params, const void* q,
+                       const void* K, const void* V, const int32_t* seq_lens, const void* musig, const float* mnorm,
+                       const float* tau, const float* head_const, float* out, uint8_t* sel_mask, int32_t* stats,
+                       uint32_t* status_dev, void* workspace, size_t workspace_bytes, void* stream) {
     int rc = validate_desc(desc);
     if (rc != ETA_OK) return rc;
+    if (pages && (rc = validate_pages(desc, pages)) != ETA_OK) return rc;
     if (!params || !q || !K || !V || !seq_lens || !out || !sel_mask) return ETA_ERR_INVALID_ARG;
     const bool dense = (params->flags & ETA_FLAG_DENSE) != 0;
     if (!dense && (!musig || !mnorm)) return ETA_ERR_INVALID_ARG;
@@ -1125,9 +1133,10 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     if (rc != ETA_OK) return rc;
 
     CUtensorMap tmK, tmV;
-    rc = make_tmap(&tmK, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t, TS);
+    const int n_pages = pages ? pages->n_pages : 0;
+    rc = make_tmap(&tmK, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t, TS, n_pages);
     if (rc != ETA_OK) return rc;
-    rc = make_tmap(&tmV, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_t, TS);
+    rc = make_tmap(&tmV, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_t, TS, n_pages);
     if (rc != ETA_OK) return rc;
 
     DecodeArgs da;
@@ -1142,6 +1151,8 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     da.nseg = L.nseg; da.entries = L.entries; da.rows = L.rows; da.nb_cap = desc->nb_cap;
     da.rescue_window = params->rescue_window;
     da.ungate_last = (!dense && (params->flags & ETA_FLAG_UNGATE_LAST)) ? 1 : 0;
+    da.block_table = pages ? pages->block_table : nullptr;
+    da.table_stride = pages ? pages->table_stride : 0;
     da.div_nseg = FastDiv(L.nseg); da.div_epr = FastDiv(L.nseg + 2); da.div_hkv = FastDiv(desc->n_kv_heads);
     da.div_g = FastDiv(G);
     da.timeline = debug_timeline();
@@ -1167,6 +1178,29 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
     if (me != cudaSuccess) { set_cuda_error(me, "merge launch"); return ETA_ERR_CUDA; }
     profile_mark(5, s);
     return check_launch("merge");
+}
+
+}  // namespace eta
+
+extern "C" {
+
+int eta_decode_kernel_count(void) { return 3; }
+
+int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q, const void* K, const void* V,
+               const int32_t* seq_lens, const void* musig, const float* mnorm, const float* tau,
+               const float* head_const, float* out, uint8_t* sel_mask, int32_t* stats, uint32_t* status_dev,
+               void* workspace, size_t workspace_bytes, void* stream) {
+    return eta::decode_impl(desc, nullptr, params, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask, stats,
+                            status_dev, workspace, workspace_bytes, stream);
+}
+
+int eta_decode_paged(const eta_cache_desc* desc, const eta_page_table* pages, const eta_params* params, const void* q,
+                     const void* K_pool, const void* V_pool, const int32_t* seq_lens, const void* musig,
+                     const float* mnorm, const float* tau, const float* head_const, float* out, uint8_t* sel_mask,
+                     int32_t* stats, uint32_t* status_dev, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!pages) return ETA_ERR_INVALID_ARG;
+    return eta::decode_impl(desc, pages, params, q, K_pool, V_pool, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,
+                            stats, status_dev, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

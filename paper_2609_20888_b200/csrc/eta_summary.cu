@@ -140,7 +140,7 @@ template <int D>
 __global__ void __launch_bounds__(128) build_summaries_kernel(
     const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
     int nb_max, int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
-    float* __restrict__ mnorm) {
+    float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride) {
     const int64_t wid = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
     if (wid >= (int64_t)rows * nb_max) return;
     const int r = (int)(wid / nb_max), j = (int)(wid % nb_max);
@@ -148,7 +148,9 @@ __global__ void __launch_bounds__(128) build_summaries_kernel(
     int T = seq_lens[i];
     T = T < 0 ? 0 : (T > t_cap ? t_cap : T);
     if (j >= T / b || j >= nb_cap) return;
-    const __nv_bfloat16* blk = K + i * sb + hk * sh + (int64_t)j * b * st;
+    // contiguous cache: block j of sequence i; paged cache: the page the table names for it
+    const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
+                                     : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
     summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
 }
@@ -157,7 +159,7 @@ template <int D>
 __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
     int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
-    float* __restrict__ mnorm) {
+    float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride) {
     const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
     pdl_trigger();       // nothing later in a decode step needs this kernel's output before it has waited for it
     if (r >= rows) return;
@@ -166,19 +168,25 @@ __global__ void __launch_bounds__(128) append_summary_kernel(
     if (T <= 0 || T > t_cap || T % b != 0) return;
     const int j = T / b - 1;
     if (j >= nb_cap) return;
-    const __nv_bfloat16* blk = K + i * sb + hk * sh + (int64_t)j * b * st;
+    const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
+                                     : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
     summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
 }
 
-}  // namespace eta
+int validate_pages(const eta_cache_desc* desc, const eta_page_table* pages) {
+    if (!pages || !pages->block_table || pages->n_pages <= 0) return ETA_ERR_INVALID_ARG;
+    if ((int64_t)pages->table_stride * desc->block_size < desc->t_cap) return ETA_ERR_INVALID_ARG;
+    return ETA_OK;
+}
 
-extern "C" {
-
-int eta_build_block_summaries(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens, void* musig,
-                              float* mnorm, uint32_t flags, void* stream) {
+static int build_impl(const eta_cache_desc* desc, const eta_page_table* pages, const void* K, const int32_t* seq_lens,
+                      void* musig, float* mnorm, uint32_t flags, void* stream) {
     int rc = eta::validate_desc(desc);
     if (rc != ETA_OK) return rc;
+    if (pages && (rc = validate_pages(desc, pages)) != ETA_OK) return rc;
+    const int32_t* table = pages ? pages->block_table : nullptr;
+    const int tstride = pages ? pages->table_stride : 0;
     if (!K || !seq_lens || !musig || !mnorm) return ETA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(musig)) & 15) return ETA_ERR_UNSUPPORTED;
     const int rows = desc->batch * desc->n_kv_heads;
@@ -192,17 +200,22 @@ int eta_build_block_summaries(const eta_cache_desc* desc, const void* K, const i
     auto mp = static_cast<__half*>(musig);
     if (desc->head_dim == 128)
         eta::build_summaries_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
-            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, nb_max, rows, seq_lens, env, mp, mnorm);
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, nb_max, rows, seq_lens, env, mp, mnorm,
+            table, tstride);
     else
         eta::build_summaries_kernel<64><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
-            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, nb_max, rows, seq_lens, env, mp, mnorm);
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, nb_max, rows, seq_lens, env, mp, mnorm,
+            table, tstride);
     return eta::check_launch("eta_build_block_summaries");
 }
 
-int eta_append_summary(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens_after, void* musig,
-                       float* mnorm, uint32_t flags, void* stream) {
+static int append_impl(const eta_cache_desc* desc, const eta_page_table* pages, const void* K,
+                       const int32_t* seq_lens_after, void* musig, float* mnorm, uint32_t flags, void* stream) {
     int rc = eta::validate_desc(desc);
     if (rc != ETA_OK) return rc;
+    if (pages && (rc = validate_pages(desc, pages)) != ETA_OK) return rc;
+    const int32_t* table = pages ? pages->block_table : nullptr;
+    const int tstride = pages ? pages->table_stride : 0;
     if (!K || !seq_lens_after || !musig || !mnorm) return ETA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(musig)) & 15) return ETA_ERR_UNSUPPORTED;
     const int rows = desc->batch * desc->n_kv_heads;
@@ -214,11 +227,39 @@ int eta_append_summary(const eta_cache_desc* desc, const void* K, const int32_t*
     eta::profile_mark(0, s);
     if (desc->head_dim == 128)
         eta::append_summary_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
-            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm);
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm,
+            table, tstride);
     else
         eta::append_summary_kernel<64><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
-            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm);
+            desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm,
+            table, tstride);
     return eta::check_launch("eta_append_summary");
+}
+
+}  // namespace eta
+
+extern "C" {
+
+int eta_build_block_summaries(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens, void* musig,
+                              float* mnorm, uint32_t flags, void* stream) {
+    return eta::build_impl(desc, nullptr, K, seq_lens, musig, mnorm, flags, stream);
+}
+
+int eta_build_block_summaries_paged(const eta_cache_desc* desc, const eta_page_table* pages, const void* K_pool,
+                                    const int32_t* seq_lens, void* musig, float* mnorm, uint32_t flags, void* stream) {
+    if (!pages) return ETA_ERR_INVALID_ARG;
+    return eta::build_impl(desc, pages, K_pool, seq_lens, musig, mnorm, flags, stream);
+}
+
+int eta_append_summary(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens_after, void* musig,
+                       float* mnorm, uint32_t flags, void* stream) {
+    return eta::append_impl(desc, nullptr, K, seq_lens_after, musig, mnorm, flags, stream);
+}
+
+int eta_append_summary_paged(const eta_cache_desc* desc, const eta_page_table* pages, const void* K_pool,
+                             const int32_t* seq_lens_after, void* musig, float* mnorm, uint32_t flags, void* stream) {
+    if (!pages) return ETA_ERR_INVALID_ARG;
+    return eta::append_impl(desc, pages, K_pool, seq_lens_after, musig, mnorm, flags, stream);
 }
 
 }  // extern "C"

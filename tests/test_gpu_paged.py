@@ -1,0 +1,131 @@
+"""Paged KV cache (Section 3: summaries in a held-out table beside a paged cache): the paged entry points must give,
+bit for bit, what the contiguous ones give on the gathered cache (whose parity with the oracle
+tests/test_gpu_parity.py establishes).  Pages are scattered by a seeded permutation; unused pages and the unused
+part of every tail page hold large finite garbage that must not leak into any result."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_20888_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _eb():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a GPU")
+    from paper_2609_20888_b200 import binding as eb
+    eb.load()
+    return eb
+
+
+def _scatter(K, V, lens, b, seed, layout):
+    """-> K_pool, V_pool (bf16 CUDA), block_table (int32 CUDA [B, stride]), n_pages"""
+    B, Hkv, Tcap, d = K.shape
+    per_seq = (Tcap + b - 1) // b
+    n_pages = B * per_seq + 7
+    g = torch.Generator().manual_seed(seed)
+    perm = torch.randperm(n_pages, generator=g)[:B * per_seq].view(B, per_seq)
+    shape = (n_pages, Hkv, b, d) if layout == "phbd" else (n_pages, b, Hkv, d)
+    Kp = torch.full(shape, 1.0e4, dtype=torch.bfloat16)
+    Vp = torch.full(shape, -1.0e4, dtype=torch.bfloat16)
+    if layout != "phbd":
+        Kp, Vp = Kp.permute(0, 2, 1, 3), Vp.permute(0, 2, 1, 3)      # logical [page, head, token, dim], other strides
+    for i in range(B):
+        T = int(lens[i])
+        for j in range((T + b - 1) // b):
+            n = min(b, T - j * b)
+            Kp[perm[i, j], :, :n] = K[i, :, j * b:j * b + n]
+            Vp[perm[i, j], :, :n] = V[i, :, j * b:j * b + n]
+    table = torch.full((B, per_seq + 3), -12345, dtype=torch.int32)      # entries past the sequence are never read
+    table[:, :per_seq] = perm.to(torch.int32)
+    dev = torch.device("cuda:0")
+    return Kp.to(dev), Vp.to(dev), table.to(dev), n_pages
+
+
+@pytest.mark.parametrize("name,ctx,batch,layout", [("c2_32k", 4096 + 77, 2, "phbd"), ("c5_frozen", 8192, 4, "pbhd"),
+                                                   ("c4_512k", 16384 + 5, 1, "phbd"), ("c1_tiny", 2048 + 16, 1, "pbhd")])
+def test_paged_cache_equals_contiguous_bit_for_bit(name, ctx, batch, layout):
+    eb = _eb()
+    dev = torch.device("cuda:0")
+    sp = wl.CONFIGS[name].scaled(ctx, batch=batch)
+    w = wl.make_workload(sp)
+    b = sp.block_size
+    lens = w.seq_lens.clone()
+    K, V = w.K.to(dev), w.V.to(dev)
+    lens_d = lens.to(dev)
+    q = w.queries(0).to(dev)
+    params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window)
+
+    # contiguous reference run
+    st = eb.DecodeState(K, V, sp.n_q_heads, b)
+    eb.eta_build_block_summaries(st.desc, K, lens_d, st.musig, st.mnorm)
+    # thresholds at each head's median bound: about half of the blocks are pruned
+    bound = torch.full((sp.batch, sp.n_q_heads, st.desc.nb_cap), float("nan"), dtype=torch.float32, device=dev)
+    eb.eta_score_dual(st.desc, params, q, lens_d, st.musig, st.mnorm, bound)
+    tau = torch.nanmedian(bound, dim=2).values.contiguous()
+    eb.eta_decode(st.desc, params, q, K, V, lens_d, st.musig, st.mnorm, tau, None, st.out, st.sel_mask, st.workspace,
+                  stats=st.stats, status=st.status)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    frac = float(st.stats.sum().item()) / max(1, sum(int(t) // b for t in lens) * sp.n_kv_heads)
+    assert 0.02 < frac < 0.98, "the case must prune some blocks and keep some"
+
+    # paged run on the scattered pools
+    Kp, Vp, table, n_pages = _scatter(w.K, w.V, lens, b, seed=sp.seed + 1, layout=layout)
+    pdesc = eb.paged_cache_desc(Kp, Vp, sp.batch, sp.n_q_heads, t_cap=w.K.shape[2], nb_cap=st.desc.nb_cap)
+    pages = eb.page_table(table, n_pages)
+    musig, mnorm = eb.alloc_summaries(pdesc, dev)
+    eb.eta_build_block_summaries_paged(pdesc, pages, Kp, lens_d, musig, mnorm)
+    torch.cuda.synchronize()
+    assert torch.equal(musig.view(torch.int16), st.musig.view(torch.int16))
+    assert torch.equal(mnorm.view(torch.int32), st.mnorm.view(torch.int32))
+    out = torch.full_like(st.out, float("nan"))
+    sel = torch.zeros_like(st.sel_mask)
+    stats = torch.zeros_like(st.stats)
+    status = torch.zeros_like(st.status)
+    ws = torch.zeros_like(st.workspace)
+    eb.eta_decode_paged(pdesc, pages, params, q, Kp, Vp, lens_d, musig, mnorm, tau, None, out, sel, ws,
+                        stats=stats, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(sel, st.sel_mask)
+    assert torch.equal(stats, st.stats)
+    assert torch.equal(out.view(torch.int32), st.out.view(torch.int32))
+
+
+def test_paged_append_equals_paged_rebuild():
+    """Appending tokens until a block fills up: the paged append writes the record the paged build writes."""
+    eb = _eb()
+    dev = torch.device("cuda:0")
+    sp = wl.CONFIGS["c2_32k"].scaled(2048, batch=3)
+    w = wl.make_workload(sp)
+    b = sp.block_size
+    lens = torch.tensor([2048 - b, 2048 - 2 * b, 2048 - b - 5], dtype=torch.int32)
+    Kp, Vp, table, n_pages = _scatter(w.K, w.V, torch.full((3,), 2048), b, seed=7, layout="phbd")
+    pdesc = eb.paged_cache_desc(Kp, Vp, sp.batch, sp.n_q_heads, t_cap=2048)
+    pages = eb.page_table(table, n_pages)
+    musig, mnorm = eb.alloc_summaries(pdesc, dev)
+    eb.eta_build_block_summaries_paged(pdesc, pages, Kp, lens.to(dev), musig, mnorm)
+    after = lens + torch.tensor([b, b, 5], dtype=torch.int32)          # all three now end on a block boundary
+    eb.eta_append_summary_paged(pdesc, pages, Kp, after.to(dev), musig, mnorm)
+    ref_musig, ref_mnorm = eb.alloc_summaries(pdesc, dev)
+    eb.eta_build_block_summaries_paged(pdesc, pages, Kp, after.to(dev), ref_musig, ref_mnorm)
+    torch.cuda.synchronize()
+    assert torch.equal(musig.view(torch.int16), ref_musig.view(torch.int16))
+    assert torch.equal(mnorm.view(torch.int32), ref_mnorm.view(torch.int32))
+
+
+def test_paged_arguments_are_validated():
+    eb = _eb()
+    dev = torch.device("cuda:0")
+    Kp = torch.zeros((8, 2, 32, 64), dtype=torch.bfloat16, device=dev)
+    pdesc = eb.paged_cache_desc(Kp, Kp, 1, 4, t_cap=128)
+    lens = torch.tensor([64], dtype=torch.int32, device=dev)
+    musig, mnorm = eb.alloc_summaries(pdesc, dev)
+    short = torch.zeros((1, 3), dtype=torch.int32, device=dev)           # 3 * 32 < t_cap
+    with pytest.raises(eb.EtaError):
+        eb.eta_build_block_summaries_paged(pdesc, eb.page_table(short, 8), Kp, lens, musig, mnorm)
+    ok = torch.zeros((1, 4), dtype=torch.int32, device=dev)
+    with pytest.raises(eb.EtaError):
+        eb.eta_build_block_summaries_paged(pdesc, eb.page_table(ok, 0), Kp, lens, musig, mnorm)
