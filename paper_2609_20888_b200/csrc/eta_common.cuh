@@ -202,6 +202,15 @@ __device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, f
         : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
 }
 
+// (d0, d1) += (a0, a1): the packed fp32 add of sm_100
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
+    asm("{\n\t.reg .b64 ra, rc;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rc, {%0, %1};\n\t"
+        "add.rn.f32x2 rc, rc, ra;\n\t"
+        "mov.b64 {%0, %1}, rc;\n\t}"
+        : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
+}
+
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"

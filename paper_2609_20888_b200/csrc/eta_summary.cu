@@ -6,13 +6,102 @@
 // One warp owns one block of b keys.  A row of d bf16 values is read by d/8
 // lanes as 16-byte vectors, so a warp covers 32/(d/8) rows per load
 // instruction and every 32-byte sector of the block is requested exactly once
-// from HBM; eight such loads are in flight per lane.  The second pass
-// (deviations about the mean) re-reads the block from L1/L2.  Arithmetic is
-// fp32.  Build and append share this routine, so appending a block gives the
-// same bytes as rebuilding the index.
+// from HBM; eight such loads are in flight per lane.  The plain sigma needs
+// one pass (deviations about the block's first key); the sub-block envelope
+// takes a second pass (deviations about the mean) that re-reads the block
+// from L1/L2.  Arithmetic is fp32.  Build and append share these routines, so
+// appending a block gives the same bytes as rebuilding the index.
 #include "eta_common.cuh"
 
 namespace eta {
+
+// One pass over the block for centroid, sigma and the largest norm: squared deviations are taken about the block's
+// first key k0 instead of the (not yet known) mean,
+//   mu = S / b,   sigma^2 = S2 / b - (mu - k0)^2,   S = sum k,  S2 = sum (k - k0)^2,
+// which is exact for identical keys and loses only a factor 1 + (mu - k0)^2 / sigma^2 (a few units for a key drawn
+// from the block) of fp32's 24 bits against the fp16 the result is stored in.  The centroid comes from the plain
+// sum: bf16 keys have 8 significant bits, so fp32 partial sums of a block's keys are exact or nearly so, which the
+// shifted sum (whose partial sums grow like t (mu - k0)) would not be for a centroid close to zero.  Packed fp32
+// arithmetic: two coordinates per issue.
+// INFLIGHT: rows a lane requests before it starts on the first of them (8 in the throughput-bound build, where
+// many warps per SM hide the latency; 32 in the append, where a warp is alone with one block and the whole block
+// is requested at once).  The order of the arithmetic, hence every result bit, is the same for any INFLIGHT.
+template <int D, int INFLIGHT>
+__device__ __forceinline__ void summarize_block_onepass(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
+                                                        __half* __restrict__ rec, float* __restrict__ mn) {
+    constexpr int LPR = D / 8;        // lanes per row
+    constexpr int RPP = 32 / LPR;     // rows per pass
+    const int lane = threadIdx.x & 31;
+    const int cc = lane % LPR, ro = lane / LPR;
+    const __nv_bfloat16* base = blk + cc * 8;
+
+    float nk0[8];        // minus the first key's coordinates
+    {
+        const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(base));
+        const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { nk0[2 * k] = -bf16_lo(w[k]); nk0[2 * k + 1] = -bf16_hi(w[k]); }
+    }
+    float s1[8], s2[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { s1[k] = 0.f; s2[k] = 0.f; }
+    float maxn2 = 0.f;
+    for (int t0 = ro; t0 < b; t0 += INFLIGHT * RPP) {
+        uint4 v[INFLIGHT];
+#pragma unroll
+        for (int u = 0; u < INFLIGHT; ++u)
+            if (INFLIGHT == 8 || t0 + u * RPP < b)      // b is a multiple of 8 * RPP for every supported block size
+                v[u] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)(t0 + u * RPP) * stride_t));
+#pragma unroll
+        for (int u = 0; u < INFLIGHT; ++u) {
+            if (INFLIGHT != 8 && t0 + u * RPP >= b) break;
+            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            float na = 0.f, nb = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float lo = bf16_lo(w[k]), hi = bf16_hi(w[k]);
+                fma2(na, nb, lo, hi, lo, hi);
+                add2(s1[2 * k], s1[2 * k + 1], lo, hi);
+                float dl = lo, dh = hi;
+                add2(dl, dh, nk0[2 * k], nk0[2 * k + 1]);
+                fma2(s2[2 * k], s2[2 * k + 1], dl, dh, dl, dh);
+            }
+            float n2 = na + nb;
+#pragma unroll
+            for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+            maxn2 = fmaxf(maxn2, n2);
+        }
+    }
+#pragma unroll
+    for (int s = LPR; s < 32; s <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            s1[k] += __shfl_xor_sync(0xffffffffu, s1[k], s);
+            s2[k] += __shfl_xor_sync(0xffffffffu, s2[k], s);
+        }
+        maxn2 = fmaxf(maxn2, __shfl_xor_sync(0xffffffffu, maxn2, s));
+    }
+    const float inv_b = 1.0f / (float)b;
+    if (ro < 2) {
+        float src[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float mean = s1[k] * inv_b;
+            const float m1 = mean + nk0[k];
+            src[k] = (ro == 0) ? mean : sqrtf(fmaxf(fmaf(-m1, m1, s2[k] * inv_b), 0.f));
+        }
+        __half2 h[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) h[k] = __floats2half2_rn(src[2 * k], src[2 * k + 1]);
+        uint4 o;
+        o.x = *reinterpret_cast<uint32_t*>(&h[0]);
+        o.y = *reinterpret_cast<uint32_t*>(&h[1]);
+        o.z = *reinterpret_cast<uint32_t*>(&h[2]);
+        o.w = *reinterpret_cast<uint32_t*>(&h[3]);
+        *reinterpret_cast<uint4*>(rec + ro * D + cc * 8) = o;
+    }
+    if (lane == 0) *mn = sqrtf(maxn2);
+}
 
 // b is a multiple of 8 * (rows per warp instruction) for every supported block size, so the loops need no guards.
 template <int D, bool envelope>
@@ -129,11 +218,11 @@ __device__ __forceinline__ void summarize_block_t(const __nv_bfloat16* __restric
     if (lane == 0) *mn = sqrtf(maxn2);
 }
 
-template <int D>
+template <int D, int INFLIGHT>
 __device__ __forceinline__ void summarize_block(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
                                                 bool envelope, __half* __restrict__ rec, float* __restrict__ mn) {
     if (envelope) summarize_block_t<D, true>(blk, stride_t, b, rec, mn);
-    else summarize_block_t<D, false>(blk, stride_t, b, rec, mn);
+    else summarize_block_onepass<D, INFLIGHT>(blk, stride_t, b, rec, mn);
 }
 
 template <int D>
@@ -152,7 +241,7 @@ __global__ void __launch_bounds__(128) build_summaries_kernel(
     const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
                                      : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
-    summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
+    summarize_block<D, 8>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
 }
 
 template <int D>
@@ -171,7 +260,7 @@ __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
                                      : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
-    summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
+    summarize_block<D, 32>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
 }
 
 int validate_pages(const eta_cache_desc* desc, const eta_page_table* pages) {
