@@ -199,6 +199,11 @@ int eta_calibrate_head_const(int32_t n_seq, int32_t seq_len, int32_t n_q_heads, 
  * status_dev (nullable, uint32, caller-zeroed) device-side problems.
  * bf16 operands, fp32 scores / softmax statistics / accumulators; deterministic
  * for a given device and launch hint.  workspace: eta_workspace_bytes() bytes.
+ * Launch order: the kernels are launched with programmatic dependent launch and read q, seq_lens and every
+ * summary except the newest block's before they wait for the preceding kernel of the stream.  Producers of those
+ * inputs must therefore be complete when that preceding kernel starts: true for copies, for kernels launched
+ * without early dependent release (eta_stage_query among them) and for anything ordered by an event or a
+ * synchronisation; only a kernel that releases its dependents early and then writes q would break it.
  */
 int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void* q,
                const void* K, const void* V, const int32_t* seq_lens,
