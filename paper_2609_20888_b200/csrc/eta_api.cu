@@ -62,6 +62,15 @@ static bool g_pdl = true;
 bool pdl_enabled() { return g_pdl; }
 void set_pdl(bool on) { g_pdl = on; }
 
+void prefer_max_shared(const void* kernel) {
+    static const void* seen[64];
+    static int n_seen = 0;
+    for (int k = 0; k < n_seen; ++k)
+        if (seen[k] == kernel) return;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (n_seen < 64) seen[n_seen++] = kernel;
+}
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 WsLayout ws_layout(const eta_cache_desc* d) {

@@ -103,9 +103,15 @@ int launch_screen(const ScreenArgs& a, int rows, int D, int G, int n_ctas, cudaS
 // still draining, and must call pdl_wait() before touching anything the predecessor wrote.
 unsigned long long* debug_timeline();   // device buffer for per-CTA time stamps, or nullptr (see eta_debug_timeline)
 bool pdl_enabled();          // false after eta_set_pdl(0): every launch is then fully serialised
+// Asks (once per kernel) for the largest shared-memory carve-out.  The streaming kernel needs it; when its
+// neighbours in the stream run with another split of the SM's L1/shared memory, an SM has to drain and
+// reconfigure before the first CTA of the next kernel can start on it, which showed as ~2 us between the last CTA of
+// one kernel and the first of the next.  None of the kernels of a step depends on L1 capacity.
+void prefer_max_shared(const void* kernel);
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
                               Args&&... args) {
+    prefer_max_shared(reinterpret_cast<const void*>(kernel));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -214,6 +220,13 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }

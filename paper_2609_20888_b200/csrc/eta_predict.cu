@@ -93,6 +93,7 @@ extern "C" int eta_stage_query(int32_t batch, int32_t n_q_heads, int32_t head_di
     const int n16 = (int)(bytes / 16);
     int grid = (n16 + 255) / 256;
     if (grid > 296) grid = 296;
+    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::stage_query_kernel));
     eta::stage_query_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(q_host),
                                                                                  static_cast<uint4*>(q_dev), n16);
     return eta::check_launch("eta_stage_query");
@@ -125,6 +126,7 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
     attr[1].val.programmaticStreamSerializationAllowed = eta::pdl_enabled() ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
+    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::predict_threshold_kernel));
     eta::profile_mark(1, cfg.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, eta::predict_threshold_kernel, static_cast<const __nv_bfloat16*>(q), W,
                                        bias, tau, (int)n_q_heads, rows);

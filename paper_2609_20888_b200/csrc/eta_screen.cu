@@ -57,6 +57,10 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     constexpr int RB = RPW * NI;          // records per warp per batch
     constexpr int REC_BYTES = L::REC_BYTES;
     constexpr bool USE_Q2 = (G <= 4);
+    // head_dim 128 with 4 heads per group (every benchmark configuration): the centroid term <q, mu> of a warp's
+    // eight records is one 16 x 8 x 128 tensor-core product (fp16 operands, fp32 accumulation; bf16 -> fp16 is
+    // exact from 2^-17 up), which leaves the fp32 pipe the variance term only
+    constexpr bool USE_MMA = (D == 128 && G == 4);
     static_assert(NI >= 1, "group size too large for this head_dim");
 
     extern __shared__ unsigned char scr_raw[];
@@ -135,6 +139,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     };
 
     float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G], my_qn = 0.f;
+    uint32_t qa[USE_MMA ? 8 : 1][2];       // A fragments of the centroid product: head lane / 4, one pair of registers per k-step
     int q_row = -1;
     bool waited = false;
     Geom gc = item_geom(it0);
@@ -193,8 +198,98 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                     my_qn = qn[0];
 #pragma unroll
                     for (int g = 1; g < G; ++g) my_qn = (my_g == g) ? qn[g] : my_qn;
+                    if constexpr (USE_MMA) {
+                        // A[head][k]: lane (t = lane % 4, head = lane / 4 < G) holds, for k-steps 2j and 2j + 1, the
+                        // eight dimensions 8 (4 j + t) .. + 7 of its head: the same dimensions the B fragments below
+                        // take from one 16-byte load of a record (a dot product does not care about the order of k)
+                        const int t4 = lane & 3, hd = lane >> 2;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint4 v = make_uint4(0, 0, 0, 0);
+                            if (hd < G) v = lds128(rec_base + SEG * REC_BYTES + (hd * D + 8 * (4 * j + t4)) * 2);
+                            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                            uint32_t h[4];
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) {
+                                const __half2 hh = __floats2half2_rn(bf16_lo(w[kk]), bf16_hi(w[kk]));
+                                h[kk] = *reinterpret_cast<const uint32_t*>(&hh);
+                            }
+                            qa[2 * j][0] = h[0]; qa[2 * j][1] = h[1];
+                            qa[2 * j + 1][0] = h[2]; qa[2 * j + 1][1] = h[3];
+                        }
+                    }
                 }
 
+                if constexpr (USE_MMA) {
+                    const int base = warp * RB;            // RB = 8 records per warp: one n-tile of the product
+                    if (base < n_rec) {
+                        // centroid term: D[head][record] += q[head][k] * mu[record][k] over 8 k-steps
+                        float c[4] = {0.f, 0.f, 0.f, 0.f};
+                        {
+                            const int t4 = lane & 3, n8 = lane >> 2;
+                            const uint32_t mu_addr = rec_base + (base + n8) * REC_BYTES + t4 * 16;
+                            uint4 bq[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) bq[j] = lds128(mu_addr + j * 64);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                mma_f16_16816(c, qa[2 * j][0], 0u, qa[2 * j][1], 0u, bq[j].x, bq[j].y);
+                                mma_f16_16816(c, qa[2 * j + 1][0], 0u, qa[2 * j + 1][1], 0u, bq[j].z, bq[j].w);
+                            }
+                        }
+                        // variance term on the fp32 pipe, two heads per packed fma: lane (cc, rg) takes dimensions
+                        // 8 cc .. + 7 of record base + it * RPW + rg
+                        float v[NI * G];
+#pragma unroll
+                        for (int it = 0; it < NI; ++it) {
+                            const int rec = base + it * RPW + rg;
+                            float s2[8];
+                            if (rec < n_rec) {
+                                const uint4 s4 = lds128(rec_base + rec * REC_BYTES + 2 * D + cc * 16);
+                                const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk) {
+                                    const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
+                                    s2[2 * kk] = sf.x * sf.x;
+                                    s2[2 * kk + 1] = sf.y * sf.y;
+                                }
+                            } else {
+#pragma unroll
+                                for (int kk = 0; kk < 8; ++kk) s2[kk] = 0.f;
+                            }
+                            float var[G];
+#pragma unroll
+                            for (int g = 0; g < G; ++g) var[g] = 0.f;
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk)
+#pragma unroll
+                                for (int g = 0; g < G; g += 2)
+                                    fma2(var[g], var[g + 1], q2[g][kk], q2[g + 1][kk], s2[kk], s2[kk]);
+#pragma unroll
+                            for (int g = 0; g < G; ++g) v[it * G + g] = var[g];
+                        }
+                        // transposed butterfly over the LPR lanes of a record: lane cc ends with the variance term
+                        // of pair cc = it * G + g
+#pragma unroll
+                        for (int s = LPR / 2, n = NI * G / 2; s >= 1; s >>= 1, n >>= 1) {
+                            const bool upper = (lane & s) != 0;
+#pragma unroll
+                            for (int kk = 0; kk < n; ++kk) {
+                                const float send = upper ? v[kk] : v[kk + n];
+                                const float keep = upper ? v[kk + n] : v[kk];
+                                v[kk] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+                            }
+                        }
+                        // the centroid term of (record base + 2 it + rg, head g) sits in lane 4 g + it, element rg
+                        const int it = cc / G;
+                        const float d0 = __shfl_sync(0xffffffffu, c[0], 4 * my_g + it);
+                        const float d1 = __shfl_sync(0xffffffffu, c[1], 4 * my_g + it);
+                        const float dot = rg ? d1 : d0;
+                        const int rec = base + it * RPW + rg;
+                        if (rec < n_rec)
+                            sbound[rec][my_g] = a.scale * min_keep_nan(dot + a.z * sqrtf(v[0]), my_qn * smn[rec]);
+                    }
+                } else
                 for (int base = warp * RB; base < n_rec; base += 8 * RB) {
                     float v[NV];
 #pragma unroll
@@ -458,9 +553,9 @@ static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream
     // The slowest CTA sets the kernel's end.  All CTAs are resident at once (n_ctas = two per SM), but under
     // programmatic dependent launch the kernel starts while its predecessors (summary append, threshold predictor)
     // still hold some SMs, where no CTA of this kernel fits until they exit: the CTAs dispatched last (the
-    // highest indices) start late and get two items fewer (measured at G = 4, D = 128: giving them three or four
-    // fewer evens out the mean end time but leaves some early CTAs with one item more, which ends later).
-    // With x items for an early CTA all end together when  n_early x + n_late (x - 2) = n_items.
+    // highest indices) start late, by the time `lag` items take (measured at d = 128: 7.6 us against 1.4 us per
+    // item with the tensor-core centroid term at G = 4, 1.9 us without), and get that many items fewer, down to
+    // none.  With x items for an early CTA all end together when  n_early x + n_late max(x - lag, 0) = n_items.
     const int n_items = rows * a.nseg;
     ScreenArgs b2 = a;
     int grid = 0, n_late = 0;
@@ -469,13 +564,16 @@ static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream
         n_late = 2 * ((rows + 3) / 4 + (a.tau ? 8 * batch : 0));      // two slots per CTA of the append / predictor kernel
         if (n_late > n_ctas / 3) n_late = n_ctas / 3;
     }
-    const int x = (n_items + 2 * n_late + n_ctas - 1) / n_ctas;
+    const int lag = (D == 128 && G == 4) ? 5 : 2;
+    int x = (n_items + lag * n_late + n_ctas - 1) / n_ctas;
+    if (x <= lag) x = (n_items + (n_ctas - n_late) - 1) / (n_ctas - n_late);      // the late CTAs take nothing
     if (n_late > 0 && x >= 3) {
         grid = n_ctas;
-        b2.per_late = x - 2;
+        b2.per_late = x > lag ? x - lag : 0;
         b2.n_early = grid - n_late;
         b2.per_early = n_items - n_late * b2.per_late;       // shared evenly by the early CTAs
         if (b2.per_early < b2.n_early) n_late = 0;
+        else if (b2.per_late == 0) grid = b2.n_early;        // nothing to launch the late CTAs for
     } else {
         n_late = 0;
     }

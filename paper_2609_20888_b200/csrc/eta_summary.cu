@@ -313,6 +313,8 @@ static int append_impl(const eta_cache_desc* desc, const eta_page_table* pages, 
     const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
     auto Kp = static_cast<const __nv_bfloat16*>(K);
     auto mp = static_cast<__half*>(musig);
+    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::append_summary_kernel<128>));
+    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::append_summary_kernel<64>));
     eta::profile_mark(0, s);
     if (desc->head_dim == 128)
         eta::append_summary_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
