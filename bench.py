@@ -42,7 +42,7 @@ PEAKS = os.path.join(ROOT, "MEASURED_PEAKS.json")
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per launch of the streaming kernel from the ncu capture summarised in
 # profiles/decode_kernel_c3_128k_s90.md (mean of the two captured launches), keyed by (workload, target sparsity).
-NCU_TRAFFIC_BYTES = {("c3_128k", 0.90): 218.2e6}
+NCU_TRAFFIC_BYTES = {("c3_128k", 0.90): 216.7e6}
 
 
 def load_bias(name: str, target: float) -> np.ndarray:
