@@ -49,10 +49,7 @@ struct DecodeArgs {
 
 constexpr uint32_t UF_END = 1u;
 constexpr int WARPS_PER_GROUP = 4;     // the four warps of a group each take a quarter of a tile's tokens
-#ifndef ETA_PIECE_COST
-#define ETA_PIECE_COST 3
-#endif
-constexpr int PIECE_COST = ETA_PIECE_COST;          // tiles a row boundary inside a CTA's range is worth (flush + query reload)
+constexpr int PIECE_COST = 3;          // tiles a row boundary inside a CTA's range is worth (flush + query reload)
 constexpr int RESC_ROWS = 8;           // rows (from the CTA's first) whose rescue decisions stay in shared memory
 constexpr int PW = 256;                // entries of the unit prefix the producer keeps in shared memory
 
