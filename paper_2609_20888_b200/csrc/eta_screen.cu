@@ -380,8 +380,8 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
 #pragma unroll
             for (int gq = 0; gq < G; ++gq) te_g[gq] = __shfl_sync(0xffffffffu, te_l, gq);
             // The record of a block that filled up with the newest token was possibly copied before the append kernel
-            // wrote it: its bound is computed again here, from global memory past the L1, with the arithmetic (and
-            // the order of the sums) of phase 1.
+            // wrote it: its bound is computed again here, from global memory past the L1, with the fp32 arithmetic
+            // (and the order of the sums) of phase 1's path without tensor cores.
             if (!dense && ok && n_rec > 0 && (g.T & (a.b - 1)) == 0 && j0 + n_rec == NB) {
                 const int rec = n_rec - 1;
                 const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
