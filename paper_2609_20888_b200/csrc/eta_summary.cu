@@ -225,8 +225,10 @@ __device__ __forceinline__ void summarize_block(const __nv_bfloat16* __restrict_
     else summarize_block_onepass<D, INFLIGHT>(blk, stride_t, b, rec, mn);
 }
 
+// Eight CTAs (32 warps) per SM: the kernel is bound by memory latency at the bytes it keeps in flight, and 64
+// registers per thread (a few spilled words) buy one more CTA than the 72 the routine would take.
 template <int D>
-__global__ void __launch_bounds__(128) build_summaries_kernel(
+__global__ void __launch_bounds__(128, 8) build_summaries_kernel(
     const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
     int nb_max, int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
     float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride) {
