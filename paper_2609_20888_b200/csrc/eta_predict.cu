@@ -23,8 +23,11 @@ constexpr int PRED_CLUSTER = 8;
 
 __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     const __nv_bfloat16* __restrict__ q, const float* __restrict__ W, const float* __restrict__ bias,
-    float* __restrict__ tau, int Hq, int rows) {
+    float* __restrict__ tau, int Hq, int rows, unsigned long long* timeline) {
     extern __shared__ float sm[];
+    unsigned long long* tl = timeline ? timeline + (size_t)(936 + blockIdx.y * PRED_CLUSTER + blockIdx.x) * 8 : nullptr;
+    if (tl && blockIdx.y * PRED_CLUSTER + blockIdx.x >= 88) tl = nullptr;
+    if (tl && threadIdx.x == 0) tl[0] = globaltimer_ns();
     const int NRG = PRED_THREADS / Hq;           // row groups inside a CTA
     float* part = sm;                            // [NRG][Hq] partial sums of this CTA
     float* cpart = sm + NRG * Hq;                // [PRED_CLUSTER][Hq], used in the cluster's first CTA
@@ -39,22 +42,30 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
 
     float acc = 0.f;
     if (rg < NRG) {
-        // rows r_begin + rg, + NRG, ...: sixteen independent loads in flight per pass
-        for (int r0 = r_begin + rg; r0 < r_end; r0 += 16 * NRG) {
-            float w[16], x[16];
+        // rows r_begin + rg, + NRG, ...: thirty-two independent loads in flight per pass (one pass at 32 heads of
+        // 128 dimensions: the kernel's time is its round trips to memory)
+        for (int r0 = r_begin + rg; r0 < r_end; r0 += 32 * NRG) {
+            // volatile loads keep their program order, so all of them are issued before the first is used (left to
+            // itself the compiler interleaves loads and arithmetic to save registers: four round trips instead of one)
+            float w[32];
+            unsigned short xb[32];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const int r = r0 + k * NRG;
-                const bool in = r < r_end;
-                w[k] = in ? __ldg(W + (int64_t)r * Hq + h) : 0.f;
-                x[k] = in ? __bfloat162float(qi[r]) : 0.f;
+            for (int k = 0; k < 32; ++k) {
+                const int r = min(r0 + k * NRG, r_end - 1);
+                asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(w[k]) : "l"(W + (int64_t)r * Hq + h));
+                asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(xb[k]) : "l"(qi + r));
             }
 #pragma unroll
-            for (int k = 0; k < 16; ++k) acc = fmaf(x[k], w[k], acc);
+            for (int k = 0; k < 32; ++k) {
+                const float x = __uint_as_float((unsigned)xb[k] << 16);
+                if (r0 + k * NRG < r_end) acc = fmaf(x, w[k], acc);
+            }
         }
         part[rg * Hq + h] = acc;
     }
+    if (tl && threadIdx.x == 0) tl[1] = globaltimer_ns() + (__float_as_int(acc) & 0);
     __syncthreads();
+    if (tl && threadIdx.x == 0) tl[2] = globaltimer_ns();
     if (threadIdx.x < Hq) {
         float s = 0.f;
         for (int k = 0; k < NRG; ++k) s += part[k * Hq + threadIdx.x];
@@ -62,13 +73,16 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
         dst[crank * Hq + threadIdx.x] = s;
     }
     cluster.sync();
+    if (tl && threadIdx.x == 0) tl[3] = globaltimer_ns();
     if (crank == 0 && threadIdx.x < Hq) {
         float s = 0.f;
 #pragma unroll
         for (int c = 0; c < PRED_CLUSTER; ++c) s += cpart[c * Hq + threadIdx.x];
         tau[(int64_t)i * Hq + threadIdx.x] = s + bias[threadIdx.x];
     }
+    if (tl && threadIdx.x == 0) tl[4] = globaltimer_ns();
     if (threadIdx.x == 0) pdl_wait();
+    if (tl && threadIdx.x == 0) tl[5] = globaltimer_ns();
 }
 
 // Copy of a step's queries from page-locked host memory to device memory by a kernel: for a few tens of
@@ -129,7 +143,7 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
     eta::prefer_max_shared(reinterpret_cast<const void*>(eta::predict_threshold_kernel));
     eta::profile_mark(1, cfg.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, eta::predict_threshold_kernel, static_cast<const __nv_bfloat16*>(q), W,
-                                       bias, tau, (int)n_q_heads, rows);
+                                       bias, tau, (int)n_q_heads, rows, eta::debug_timeline());
     if (e != cudaSuccess) { eta::set_cuda_error(e, "eta_predict_threshold"); return ETA_ERR_CUDA; }
     return eta::check_launch("eta_predict_threshold");
 }
