@@ -23,14 +23,14 @@ constexpr int PRED_CLUSTER = 8;
 
 __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     const __nv_bfloat16* __restrict__ q, const float* __restrict__ W, const float* __restrict__ bias,
-    float* __restrict__ tau, int Hq, int rows, unsigned long long* timeline) {
+    float* __restrict__ tau, int Hq, int rows, int vec4, unsigned long long* timeline) {
     extern __shared__ float sm[];
     unsigned long long* tl = timeline ? timeline + (size_t)(936 + blockIdx.y * PRED_CLUSTER + blockIdx.x) * 8 : nullptr;
     if (tl && blockIdx.y * PRED_CLUSTER + blockIdx.x >= 88) tl = nullptr;
     if (tl && threadIdx.x == 0) tl[0] = globaltimer_ns();
     const int NRG = PRED_THREADS / Hq;           // row groups inside a CTA
-    float* part = sm;                            // [NRG][Hq] partial sums of this CTA
-    float* cpart = sm + NRG * Hq;                // [PRED_CLUSTER][Hq], used in the cluster's first CTA
+    float* part = sm;                            // [max(NRG, warps)][Hq] partial sums of this CTA
+    float* cpart = sm + max(NRG, PRED_THREADS / 32) * Hq;      // [PRED_CLUSTER][Hq], used in the cluster's first CTA
     pdl_trigger();
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank();
@@ -40,37 +40,78 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     const __nv_bfloat16* qi = q + (int64_t)i * rows;
     const int h = threadIdx.x % Hq, rg = threadIdx.x / Hq;
 
-    float acc = 0.f;
-    if (rg < NRG) {
-        // rows r_begin + rg, + NRG, ...: thirty-two independent loads in flight per pass (one pass at 32 heads of
-        // 128 dimensions: the kernel's time is its round trips to memory)
-        for (int r0 = r_begin + rg; r0 < r_end; r0 += 32 * NRG) {
-            // volatile loads keep their program order, so all of them are issued before the first is used (left to
-            // itself the compiler interleaves loads and arithmetic to save registers: four round trips instead of one)
-            float w[32];
-            unsigned short xb[32];
+    if (vec4) {
+        // Four heads per thread: a row of W is read as 16-byte pieces, so a warp instruction covers 512 bytes and the
+        // CTA needs a quarter of the load instructions of the scalar form (the kernel's time is the number of requests
+        // its SM's load unit has to take, not bytes).  Thread (rl, cg): heads 4 cg .. 4 cg + 3 of rows rl, rl + RL, ...
+        const int CG = Hq >> 2, RL = PRED_THREADS / CG;
+        const int cg4 = threadIdx.x % CG, rl = threadIdx.x / CG;
+        float a4[4] = {0.f, 0.f, 0.f, 0.f};
+        if (rl < RL) {
+            for (int r0 = r_begin + rl; r0 < r_end; r0 += 8 * RL) {
+                float4 w[8];
+                float x[8];
 #pragma unroll
-            for (int k = 0; k < 32; ++k) {
-                const int r = min(r0 + k * NRG, r_end - 1);
-                asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(w[k]) : "l"(W + (int64_t)r * Hq + h));
-                asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(xb[k]) : "l"(qi + r));
-            }
+                for (int k = 0; k < 8; ++k) {
+                    const int r = min(r0 + k * RL, r_end - 1);
+                    w[k] = __ldg(reinterpret_cast<const float4*>(W + (int64_t)r * Hq) + cg4);
+                    x[k] = (r0 + k * RL < r_end) ? __bfloat162float(qi[r]) : 0.f;
+                }
 #pragma unroll
-            for (int k = 0; k < 32; ++k) {
-                const float x = __uint_as_float((unsigned)xb[k] << 16);
-                if (r0 + k * NRG < r_end) acc = fmaf(x, w[k], acc);
+                for (int k = 0; k < 8; ++k) {
+                    a4[0] = fmaf(x[k], w[k].x, a4[0]);
+                    a4[1] = fmaf(x[k], w[k].y, a4[1]);
+                    a4[2] = fmaf(x[k], w[k].z, a4[2]);
+                    a4[3] = fmaf(x[k], w[k].w, a4[3]);
+                }
             }
         }
-        part[rg * Hq + h] = acc;
-    }
-    if (tl && threadIdx.x == 0) tl[1] = globaltimer_ns() + (__float_as_int(acc) & 0);
-    __syncthreads();
-    if (tl && threadIdx.x == 0) tl[2] = globaltimer_ns();
-    if (threadIdx.x < Hq) {
-        float s = 0.f;
-        for (int k = 0; k < NRG; ++k) s += part[k * Hq + threadIdx.x];
-        float* dst = cluster.map_shared_rank(cpart, 0);
-        dst[crank * Hq + threadIdx.x] = s;
+        // rows of one warp first (lanes that share cg: exchanges at distance CG, 2 CG, ...), then the warps in order
+        for (int s = CG; s < 32; s <<= 1) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) a4[j] += __shfl_xor_sync(0xffffffffu, a4[j], s);
+        }
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        if (lane < CG) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) part[warp * Hq + 4 * lane + j] = a4[j];
+        }
+        if (tl && threadIdx.x == 0) tl[1] = globaltimer_ns();
+        __syncthreads();
+        if (tl && threadIdx.x == 0) tl[2] = globaltimer_ns();
+        if (threadIdx.x < Hq) {
+            float s = 0.f;
+            for (int k = 0; k < PRED_THREADS / 32; ++k) s += part[k * Hq + threadIdx.x];
+            float* dst = cluster.map_shared_rank(cpart, 0);
+            dst[crank * Hq + threadIdx.x] = s;
+        }
+    } else {
+        // any other number of heads: a head per thread, sixteen loads in flight per pass
+        float acc = 0.f;
+        if (rg < NRG) {
+            for (int r0 = r_begin + rg; r0 < r_end; r0 += 16 * NRG) {
+                float w[16], x[16];
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const int r = r0 + k * NRG;
+                    const bool in = r < r_end;
+                    w[k] = in ? __ldg(W + (int64_t)r * Hq + h) : 0.f;
+                    x[k] = in ? __bfloat162float(qi[r]) : 0.f;
+                }
+#pragma unroll
+                for (int k = 0; k < 16; ++k) acc = fmaf(x[k], w[k], acc);
+            }
+            part[rg * Hq + h] = acc;
+        }
+        if (tl && threadIdx.x == 0) tl[1] = globaltimer_ns();
+        __syncthreads();
+        if (tl && threadIdx.x == 0) tl[2] = globaltimer_ns();
+        if (threadIdx.x < Hq) {
+            float s = 0.f;
+            for (int k = 0; k < NRG; ++k) s += part[k * Hq + threadIdx.x];
+            float* dst = cluster.map_shared_rank(cpart, 0);
+            dst[crank * Hq + threadIdx.x] = s;
+        }
     }
     cluster.sync();
     if (tl && threadIdx.x == 0) tl[3] = globaltimer_ns();
@@ -120,7 +161,11 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
     if (n_q_heads > eta::PRED_THREADS || batch > 65535) return ETA_ERR_UNSUPPORTED;
     const int rows = n_q_heads * head_dim;
     const int NRG = eta::PRED_THREADS / n_q_heads;
-    const size_t smem = sizeof(float) * ((size_t)NRG * n_q_heads + (size_t)eta::PRED_CLUSTER * n_q_heads);
+    const int part_rows = NRG > eta::PRED_THREADS / 32 ? NRG : eta::PRED_THREADS / 32;
+    const size_t smem = sizeof(float) * ((size_t)part_rows * n_q_heads + (size_t)eta::PRED_CLUSTER * n_q_heads);
+    // four heads per thread need a power-of-two head count (4 .. 128) and 16-byte aligned rows of W
+    const int vec4 = (n_q_heads >= 4 && n_q_heads <= 128 && (n_q_heads & (n_q_heads - 1)) == 0 &&
+                      (reinterpret_cast<uintptr_t>(W) & 15) == 0) ? 1 : 0;
     if (smem > 48 * 1024) return ETA_ERR_UNSUPPORTED;
 
     cudaLaunchConfig_t cfg = {};
@@ -143,7 +188,7 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
     eta::prefer_max_shared(reinterpret_cast<const void*>(eta::predict_threshold_kernel));
     eta::profile_mark(1, cfg.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, eta::predict_threshold_kernel, static_cast<const __nv_bfloat16*>(q), W,
-                                       bias, tau, (int)n_q_heads, rows, eta::debug_timeline());
+                                       bias, tau, (int)n_q_heads, rows, vec4, eta::debug_timeline());
     if (e != cudaSuccess) { eta::set_cuda_error(e, "eta_predict_threshold"); return ETA_ERR_CUDA; }
     return eta::check_launch("eta_predict_threshold");
 }

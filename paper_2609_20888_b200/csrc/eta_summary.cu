@@ -250,8 +250,10 @@ template <int D>
 __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
     int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
-    float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride) {
+    float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride, unsigned long long* timeline) {
     const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
+    unsigned long long* tl = (timeline && r < 48) ? timeline + (size_t)(968 + r) * 8 : nullptr;
+    if (tl && (threadIdx.x & 31) == 0) tl[0] = globaltimer_ns();
     pdl_trigger();       // nothing later in a decode step needs this kernel's output before it has waited for it
     if (r >= rows) return;
     const int i = r / Hkv, hk = r % Hkv;
@@ -262,7 +264,9 @@ __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
                                      : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
+    if (tl && (threadIdx.x & 31) == 0) tl[1] = globaltimer_ns();
     summarize_block<D, 32>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
+    if (tl && (threadIdx.x & 31) == 0) tl[2] = globaltimer_ns();
 }
 
 int validate_pages(const eta_cache_desc* desc, const eta_page_table* pages) {
@@ -321,11 +325,11 @@ static int append_impl(const eta_cache_desc* desc, const eta_page_table* pages, 
     if (desc->head_dim == 128)
         eta::append_summary_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
             desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm,
-            table, tstride);
+            table, tstride, eta::debug_timeline());
     else
         eta::append_summary_kernel<64><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
             desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, rows, seq_lens_after, env, mp, mnorm,
-            table, tstride);
+            table, tstride, eta::debug_timeline());
     return eta::check_launch("eta_append_summary");
 }
 
