@@ -298,10 +298,11 @@ int eta_set_pdl(int on);
 
 /*
  * Development aid (the paper has no counterpart): when dev_buffer is a device array of at least
- * 8 * 1024 uint64, every CTA c of the screening kernel (c < 512) and of the streaming kernel writes up to eight
- * %globaltimer stamps (ns) at [k * 8 .. k * 8 + 7], k = c for the streaming kernel and 512 + c for the screening
- * kernel: kernel entry, set-up done, first copy issued, first tile consumed, last tile consumed, partials stored.
- * NULL switches it off (the default).
+ * 8 * 1024 uint64, the kernels of a decode step write up to eight %globaltimer stamps (ns) per CTA (per warp in the
+ * append kernel) at [k * 8 .. k * 8 + 7]: k = c for CTA c of the streaming kernel (entry, set-up done, first copy
+ * issued, first tile consumed, last tile consumed, partials stored, prefix window loaded, dependency wait
+ * returned), 512 + c for the screening kernel (c < 296), 808 + c for the merge kernel (c < 128), 936 + c for the
+ * predictor (c < 32), 968 + r for row r of the append kernel (r < 48).  NULL switches it off (the default).
  */
 int eta_debug_timeline(void* dev_buffer);
 

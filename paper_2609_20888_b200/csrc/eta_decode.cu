@@ -919,7 +919,7 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
-    unsigned long long* tl = (a.timeline && blockIdx.x < 200) ? a.timeline + (size_t)(808 + blockIdx.x) * 8 : nullptr;
+    unsigned long long* tl = (a.timeline && blockIdx.x < 128) ? a.timeline + (size_t)(808 + blockIdx.x) * 8 : nullptr;
     if (tl && tid == 0) tl[0] = globaltimer_ns();
     pdl_trigger();
     pdl_wait();          // every partial of the streaming kernel is in memory from here on

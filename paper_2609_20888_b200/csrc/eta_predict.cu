@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     float* __restrict__ tau, int Hq, int rows, int vec4, unsigned long long* timeline) {
     extern __shared__ float sm[];
     unsigned long long* tl = timeline ? timeline + (size_t)(936 + blockIdx.y * PRED_CLUSTER + blockIdx.x) * 8 : nullptr;
-    if (tl && blockIdx.y * PRED_CLUSTER + blockIdx.x >= 88) tl = nullptr;
+    if (tl && blockIdx.y * PRED_CLUSTER + blockIdx.x >= 32) tl = nullptr;
     if (tl && threadIdx.x == 0) tl[0] = globaltimer_ns();
     const int NRG = PRED_THREADS / Hq;           // row groups inside a CTA
     float* part = sm;                            // [max(NRG, warps)][Hq] partial sums of this CTA

@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool dense = (a.flags & ETA_FLAG_DENSE) != 0;
-    unsigned long long* tl = (a.timeline && blockIdx.x < 512) ? a.timeline + (size_t)(512 + blockIdx.x) * 8 : nullptr;
+    unsigned long long* tl = (a.timeline && blockIdx.x < 296) ? a.timeline + (size_t)(512 + blockIdx.x) * 8 : nullptr;
     if (tl && tid == 0) tl[0] = globaltimer_ns();
 
     const int n_items = a.rows * a.nseg;
