@@ -94,6 +94,20 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         mbar_init(&bars[0], 1);
         mbar_init(&bars[1], 1);
         fence_barrier_init();
+        // The copy of the CTA's first item starts before the sequence lengths are known: it takes every record of
+        // the segment that the summary array holds (how many of them are blocks of the sequence only matters
+        // when the bounds are computed), which saves the round trip for the lengths ahead of the first copy.
+        if (it0 < it1 && !dense) {
+            int r0, seg0, i0, hk0;
+            a.div_nseg.divmod(it0, r0, seg0);
+            a.div_hkv.divmod(r0, i0, hk0);
+            const int n_spec = min(SEG, a.nb_cap - seg0 * SEG);
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
+                                       ((int64_t)r0 * a.nb_cap + seg0 * SEG) * REC_BYTES;
+            mbar_arrive_expect_tx(&bars[0], n_spec * REC_BYTES + G * D * 2);
+            tma_load_1d(sm, src, n_spec * REC_BYTES, &bars[0]);
+            tma_load_1d(sm + SEG * REC_BYTES, a.q + ((int64_t)i0 * a.Hq + hk0 * G) * D, G * D * 2, &bars[0]);
+        }
     }
     if (tid < SCR_GROUP) s_ok[tid] = 1;
     // sequence lengths (a caller input) of every row, clamped, once: the per-item geometry then needs no global load
@@ -143,7 +157,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     int q_row = -1;
     bool waited = false;
     Geom gc = item_geom(it0);
-    if (tid == 0) issue(gc, 0);
+    if (tid == 0 && dense) mbar_arrive(&bars[0]);      // (otherwise the first item's copy is already on its way)
     {
         const float mn0 = load_mn(gc);
         if (tid < SEG) smn_all[tid] = mn0;
