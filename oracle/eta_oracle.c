@@ -528,8 +528,8 @@ double eta_oracle_calibration_density(const double* hist, int n_bins, double s_m
  *   constant         c_h = root of g(c) = dbar_h by bisection (g decreases from 1 to 0)
  * Bins: n_bins equal bins on [s_min, s_max], centre s_b = s_min + (b + 1/2) w;
  * a score outside the range goes to the first / last bin (the paper fixes
- * neither range nor edge rule).  The bin of a score is decided on the score
- * rounded to binary32, the precision the GPU path computes scores in.
+ * neither range nor edge rule).  The bin of a score is decided on the score as
+ * computed here, in double ("bin raw scores").
  * Bisection: `iters` halvings of [s_min - 40/beta, s_max + 40/beta].
  * hist [Hq, n_bins], dbar [Hq], head_const [Hq], residual [Hq] (= g(c) - dbar).
  */
@@ -560,8 +560,7 @@ void eta_oracle_calibrate(
                                eta_oracle_bf16_to_double(Kh[(int64_t)sidx * d + c]);
                     double S = s * dot;
                     rowsum += oracle_sigmoid(beta * (S - th));
-                    double Sf = (double)(float)S;
-                    int b = (int)floor((Sf - s_min) / w);
+                    int b = (int)floor((S - s_min) / w);
                     if (b < 0) b = 0;
                     if (b >= n_bins) b = n_bins - 1;
                     H[b] += inv_t;

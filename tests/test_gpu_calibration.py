@@ -1,7 +1,7 @@
 """Offline threshold calibration on the GPU against the CPU oracle (same split, same thresholds).
 
 Tolerances: the histogram is an integer count of 1/t weights on both sides; a score within a few fp32 ulp of a bin
-edge may fall on either side of it (the oracle bins the correctly rounded score, the kernel the score its tensor
+edge may fall on either side of it (the oracle bins the score it computed in double, the kernel the score its tensor
 core accumulated in fp32, off by up to ~2e-6 for these O(1) dot products), which moves that score's weight to the
 neighbouring bin: a fraction <= 2 * 2e-6 / w of the weight, w the bin width, so the normalised histograms agree to
 2 * that in L1.  The target density (fp32 sigmoid on the GPU) agrees to 1e-6; the calibrated constant reproduces

@@ -14,7 +14,7 @@ import torch
 
 from oracle import eta_oracle as orc
 from paper_2609_20888_b200 import workloads as wl
-from tests.helpers import bits, cache_of, compare_masks, fp16_ulp_distance, output_errors
+from tests.helpers import bits, cache_of, compare_masks, fp16_ulp_distance, heads_without_near_tie, output_errors
 
 pytestmark = pytest.mark.gpu
 
@@ -101,8 +101,7 @@ class Session:
         t = np.broadcast_to(head_const, (sp.batch, sp.n_q_heads)) if tau is None else tau
         near = compare_masks(sel, ref["sel"], ref["bound"], t.astype(np.float64), self.lens, sp.block_size, sp.gqa,
                              rescued=ref["rescued"])
-        skip = {(i, h) for (i, h, _, _) in near}
-        keep = np.array([[(i, h) not in skip for h in range(sp.n_q_heads)] for i in range(sp.batch)])
+        keep = heads_without_near_tie(near, sp.batch, sp.n_q_heads)
         assert keep.mean() > 0.9
         mx, mean = output_errors(out[keep], ref["out"][keep])
         assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)

@@ -1,12 +1,16 @@
-"""Paged KV cache (Section 3: summaries in a held-out table beside a paged cache): the paged entry points must give,
-bit for bit, what the contiguous ones give on the gathered cache (whose parity with the oracle
-tests/test_gpu_parity.py establishes).  Pages are scattered by a seeded permutation; unused pages and the unused
-part of every tail page hold large finite garbage that must not leak into any result."""
+"""Paged KV cache (Section 3: summaries in a held-out table beside a paged cache): the paged entry points are checked
+against the CPU oracle run on the gathered cache (summaries within 1 fp16 ulp / 4 fp32 ulp; with the oracle's summary
+bytes and the same thresholds on both sides, masks bit-exact outside the 1e-5 near-tie band, block counts exact,
+outputs within 1e-2 max / 1e-3 mean), and must also give, bit for bit, what the contiguous entry points give.  Pages
+are scattered by a seeded permutation; unused pages and the unused part of every tail page hold large finite garbage
+that must not leak into any result."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import eta_oracle as orc
 from paper_2609_20888_b200 import workloads as wl
+from tests.helpers import bits, cache_of, compare_masks, fp16_ulp_distance, heads_without_near_tie, output_errors
 
 pytestmark = pytest.mark.gpu
 
@@ -63,7 +67,9 @@ def test_paged_cache_equals_contiguous_bit_for_bit(name, ctx, batch, layout):
     # thresholds at each head's median bound: about half of the blocks are pruned
     bound = torch.full((sp.batch, sp.n_q_heads, st.desc.nb_cap), float("nan"), dtype=torch.float32, device=dev)
     eb.eta_score_dual(st.desc, params, q, lens_d, st.musig, st.mnorm, bound)
-    tau = torch.nanmedian(bound, dim=2).values.contiguous()
+    # (a little above the median element, so that the threshold does not sit on a bound: the oracle comparison below
+    # then has no built-in near tie)
+    tau = (torch.nanmedian(bound, dim=2).values + 3e-4).contiguous()
     eb.eta_decode(st.desc, params, q, K, V, lens_d, st.musig, st.mnorm, tau, None, st.out, st.sel_mask, st.workspace,
                   stats=st.stats, status=st.status)
     torch.cuda.synchronize()
@@ -92,6 +98,38 @@ def test_paged_cache_equals_contiguous_bit_for_bit(name, ctx, batch, layout):
     assert torch.equal(sel, st.sel_mask)
     assert torch.equal(stats, st.stats)
     assert torch.equal(out.view(torch.int32), st.out.view(torch.int32))
+
+    # the paged path against the oracle on the gathered cache: first the paged summary build ...
+    c = cache_of(w)
+    o_musig, o_mnorm = orc.block_summaries(c)
+    got_ms, got_mn = bits(musig.cpu()), mnorm.cpu().numpy()
+    for i in range(sp.batch):
+        NB = int(lens[i]) // b
+        assert fp16_ulp_distance(got_ms[i, :, :NB], o_musig[i, :, :NB]).max(initial=0) <= 1
+        assert np.abs(got_mn[i, :, :NB].view(np.int32) - o_mnorm[i, :, :NB].view(np.int32)).max(initial=0) <= 4
+    # ... then the paged decode on the oracle's summary bytes and the same fp32 thresholds
+    tau_np = tau.cpu().numpy()
+    ref = orc.decode_step(bits(w.queries(0)), c, o_musig, o_mnorm, tau=tau_np, z=sp.z, beta=sp.beta, lwb=sp.lwb,
+                          rescue_window=sp.rescue_window)
+    musig.copy_(torch.from_numpy(o_musig.view(np.int16)).view(torch.float16).to(dev))
+    mnorm.copy_(torch.from_numpy(o_mnorm).to(dev))
+    out.fill_(float("nan"))
+    eb.eta_decode_paged(pdesc, pages, params, q, Kp, Vp, lens_d, musig, mnorm, tau, None, out, sel, ws,
+                        stats=stats, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    sel_np, out_np = sel.cpu().numpy(), out.cpu().numpy()
+    near = compare_masks(sel_np, ref["sel"], ref["bound"], tau_np.astype(np.float64), c.seq_lens, b, sp.gqa,
+                         rescued=ref["rescued"])
+    keep = heads_without_near_tie(near, sp.batch, sp.n_q_heads)
+    assert keep.mean() > 0.9
+    mx, mean = output_errors(out_np[keep], ref["out"][keep])
+    assert mx <= 1e-2 and mean <= 1e-3, (mx, mean)
+    union = np.array([[int((sel_np[i, hk, :int(lens[i]) // b] != 0).sum()) for hk in range(sp.n_kv_heads)]
+                      for i in range(sp.batch)])
+    assert np.array_equal(stats.cpu().numpy(), union)
+    if not near:
+        assert np.array_equal(sel_np, ref["sel"])
 
 
 def test_paged_append_equals_paged_rebuild():

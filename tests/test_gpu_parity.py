@@ -4,7 +4,7 @@ Tolerances (bf16 K/V, fp32 accumulation):
   - block summaries: mu, sigma within 1 fp16 ulp, M within 4 fp32 ulp of the fp64 oracle;
   - predicted thresholds: 1e-4 absolute;
   - selected-block masks: bit-exact, except (head, block) pairs whose oracle bound lies within
-    1e-5 * max(1, |tau_eff|) of tau_eff (logged) and rescue choices among bounds tied that closely;
+    1e-5 (absolute) of tau_eff (logged) and rescue choices among bounds tied that closely;
   - outputs: max abs error <= 1e-2 and mean abs error <= 1e-3.
 Decode parity feeds the ORACLE's summary bytes and the same fp32 tau array to both sides, so rounding of the
 summaries cannot masquerade as a selection bug; the chained path (GPU summaries -> GPU decode) is checked too.
@@ -18,7 +18,7 @@ import torch
 from oracle import eta_oracle as orc
 from paper_2609_20888_b200 import workloads as wl
 from tests.helpers import (bits, cache_of, calibrate_bias, calibrate_head_const, compare_masks, fp16_ulp_distance,
-                           gpu_decode, output_errors)
+                           gpu_decode, heads_without_near_tie, output_errors)
 
 pytestmark = pytest.mark.gpu
 
@@ -175,8 +175,7 @@ def _decode_case(w, q, tau=None, head_const=None, **params):
     near = compare_masks(sel, ref["sel"], ref["bound"], tau_eff, c.seq_lens, sp.block_size, sp.gqa,
                          rescued=ref["rescued"])
     # heads with a logged near-tie attend a different block set: leave them out of the output comparison
-    skip = {(i, h) for (i, h, _, _) in near}
-    keep = np.array([[(i, h) not in skip for h in range(sp.n_q_heads)] for i in range(sp.batch)])
+    keep = heads_without_near_tie(near, sp.batch, sp.n_q_heads)
     assert keep.mean() > 0.9
     mx, mean = output_errors(out[keep], ref["out"][keep])
     assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
@@ -323,9 +322,66 @@ def test_edge_shapes_and_group_sizes(case, G):
         out, sel, stats, status = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=tau, **params)
         assert status == 0
         near = compare_masks(sel, ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G, rescued=ref["rescued"])
-        if not near:
-            mx, mean = output_errors(out, ref["out"])
-            assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+        keep = heads_without_near_tie(near, B, Hkv * G)
+        assert keep.mean() > 0.7
+        mx, mean = output_errors(out[keep], ref["out"][keep])
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+
+
+@pytest.mark.parametrize("d,b,G", [(64, 32, 4), (128, 64, 4), (128, 64, 8), (64, 64, 2)])
+def test_threshold_equal_to_a_bound_admits_the_block_on_the_device(d, b, G):
+    """Algorithm 3 admits a block when its bound is >= tau_eff: equality admits.  Here the bounds are exactly
+    representable on both sides, so thresholds can be SET EQUAL to bounds: every key of a block is the same
+    small-integer vector (sigma = 0, centroid = the key, so the moment term is the centroid logit), the queries are
+    small integers, and the scale is 1/8 (a power of two); the sphere term never binds (<q,k> <= |q||k|).  Then
+    bound = <q,k>/8 with no rounding anywhere, in fp64, in fp32 and through the fp16 tensor-core product alike.
+    The masks must agree bit for bit with no near tie to excuse anything; the next fp32 number above the threshold
+    must drop exactly the blocks that sat on it; and with tau = +inf the rescue must take the FIRST of the many
+    blocks tied at the largest bound."""
+    _eb()
+    B, Hkv, NB, tail = 2, 2, 75, 5
+    rng = np.random.default_rng(d * 7 + b + G)
+    T = NB * b + tail
+    kvec = rng.integers(-3, 4, size=(B, Hkv, NB + 1, d)).astype(np.float64)
+    K = torch.from_numpy(np.repeat(kvec, b, axis=2)[:, :, :((T + b - 1) // b) * b]).to(torch.bfloat16)
+    V = torch.from_numpy(rng.standard_normal(K.shape)).to(torch.bfloat16)
+    q = torch.from_numpy(rng.integers(-2, 3, size=(B, Hkv * G, d)).astype(np.float64)).to(torch.bfloat16)
+    lens = np.full(B, T, np.int32)
+    c = orc.Cache(bits(K), bits(V), lens, b)
+    musig, mnorm = orc.block_summaries(c)
+    assert not musig[:, :, :NB, 1].any()                      # sigma is exactly zero
+    bound = orc.score_dual(bits(q), musig, mnorm, lens, b, 1.0, scale=0.125)
+    # the bound is the integer dot product over 8, exactly
+    for i in range(B):
+        for h in range(Hkv * G):
+            dots = kvec[i, h // G, :NB] @ q[i, h].double().numpy()
+            assert np.array_equal(bound[i, h, :NB], dots / 8.0)
+    # thresholds ON a bound: the 60th-percentile block's value (shared by several blocks: integers tie often)
+    tau = np.sort(bound[:, :, :NB], axis=2)[:, :, int(0.6 * NB)].astype(np.float32)
+    assert np.array_equal(tau.astype(np.float64), np.sort(bound[:, :, :NB], axis=2)[:, :, int(0.6 * NB)])
+    on_tau = bound[:, :, :NB] == tau[:, :, None]
+    assert on_tau.any(axis=2).all() and on_tau.sum() > B * Hkv * G
+    above = np.nextafter(tau, np.float32(np.inf))
+    for t, admits_equal in ((tau, True), (above, False), (np.full_like(tau, np.inf), None)):
+        ref = orc.decode_step(bits(q), c, musig, mnorm, tau=t, scale=0.125)
+        out, sel, stats, status = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=t, scale=0.125)
+        assert status == 0
+        assert np.array_equal(sel, ref["sel"]), "masks differ although every bound is exact"
+        if admits_equal is not None:
+            for i in range(B):
+                for h in range(Hkv * G):
+                    bits_h = (sel[i, h // G, :NB] >> (h % G)) & 1
+                    assert np.all(bits_h[on_tau[i, h]] == (1 if admits_equal else 0))
+                    assert np.all(bits_h[bound[i, h, :NB] > t[i, h]] == 1)
+        else:
+            # rescue: the first block attaining the largest bound of the window, per head
+            first = np.argmax(bound[:, :, :NB], axis=2)
+            assert np.array_equal(ref["rescued"], first)
+            for i in range(B):
+                for h in range(Hkv * G):
+                    assert (sel[i, h // G, first[i, h]] >> (h % G)) & 1
+        mx, mean = output_errors(out, ref["out"])
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
 
 
 def test_sphere_term_binds_and_large_logits_stay_finite():
@@ -343,8 +399,7 @@ def test_sphere_term_binds_and_large_logits_stay_finite():
     out, sel, _, status = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=tau, z=20.0)
     assert status == 0
     near = compare_masks(sel, ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G, rescued=ref["rescued"])
-    skip = {(i, h) for (i, h, _, _) in near}
-    keep = np.array([[(i, h) not in skip for h in range(Hkv * G)] for i in range(B)])
+    keep = heads_without_near_tie(near, B, Hkv * G)
     mx, mean = output_errors(out[keep], ref["out"][keep])
     assert mx <= MAX_ABS and mean <= MEAN_ABS
 
@@ -380,9 +435,10 @@ def test_strided_cache_layout_bthd():
     assert int(st.status.item()) == 0
     near = compare_masks(st.sel_mask.cpu().numpy(), ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G,
                          rescued=ref["rescued"])
-    if not near:
-        mx, mean = output_errors(st.out.cpu().numpy(), ref["out"])
-        assert mx <= MAX_ABS and mean <= MEAN_ABS
+    keep = heads_without_near_tie(near, B, Hkv * G)
+    assert keep.mean() > 0.7
+    mx, mean = output_errors(st.out.cpu().numpy()[keep], ref["out"][keep])
+    assert mx <= MAX_ABS and mean <= MEAN_ABS
 
 
 def test_chained_gpu_path_and_multi_step_append():
@@ -431,9 +487,9 @@ def test_chained_gpu_path_and_multi_step_append():
         near = compare_masks(st.sel_mask.cpu().numpy(), ref["sel"], ref["bound"], tau_ref, lens, sp.block_size, sp.gqa,
                              band=2e-3, rescued=ref["rescued"])   # wider band: fp16 summary ulp and fp32 tau differ
         total_near += len(near)
-        if not near:
-            mx, mean = output_errors(st.out.cpu().numpy(), ref["out"])
-            assert mx <= MAX_ABS and mean <= MEAN_ABS, (step, mx, mean)
+        keep = heads_without_near_tie(near, sp.batch, sp.n_q_heads)
+        mx, mean = output_errors(st.out.cpu().numpy()[keep], ref["out"][keep])
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (step, mx, mean)
     assert lens[0] == 2048 + 32 and total_near <= 8
 
 
