@@ -40,9 +40,16 @@ DEFAULT_TARGET = 0.90
 CALIB = os.path.join(ROOT, "tests", "golden", "workload_calibration.json")
 PEAKS = os.path.join(ROOT, "MEASURED_PEAKS.json")
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) per launch of the streaming kernel from the ncu capture summarised in
-# profiles/decode_kernel_c3_128k_s90.md (mean of the two captured launches), keyed by (workload, target sparsity).
-NCU_TRAFFIC_BYTES = {("c3_128k", 0.90): 216.7e6}
+# DRAM bytes (read + write) per launch of the streaming kernel as ncu counted them, keyed by
+# "workload@target sparsity": a small data file kept beside the ncu summaries it was taken from.
+NCU_TRAFFIC = os.path.join(ROOT, "profiles", "decode_kernel_dram_traffic.json")
+
+
+def ncu_traffic(name: str, target: float):
+    try:
+        return float(json.load(open(NCU_TRAFFIC))[f"{name}@{target:.2f}"]["dram_bytes_per_launch"])
+    except Exception:
+        return None
 
 
 def load_bias(name: str, target: float) -> np.ndarray:
@@ -249,8 +256,7 @@ def run_ours(args):
         fetching the query from the page-locked buffer `q_stage` (eta_stage_query) and the merge kernel writes the
         output straight into the page-locked `out_host`."""
         bias_d = torch.from_numpy(bias_np).to(dev)
-        params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags,
-                                 ctas_per_sm=args.ctas_per_sm)
+        params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags)
 
         host_q = host_io if host_q is None else host_q
         host_out = host_io if host_out is None else host_out
@@ -449,7 +455,7 @@ def run_ours(args):
             "gpu_launches": args.steps * (2 + eb.eta_decode_kernel_count()),
             "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get((sp.name, main_target)), "traffic_unit": "bytes per launch",
+                         "traffic": ncu_traffic(sp.name, main_target), "traffic_unit": "bytes per launch",
                          "algorithmic_bytes_per_launch": ab["decode"]},
             "prefill_build": {"ms": build_ms, "gbs": k_bytes / (build_ms * 1e-3) / 1e9},
             "calibration": cal,
@@ -527,7 +533,6 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.CONFIGS))
-    ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch the kernels directly every step")
     ap.add_argument("--no-pdl", dest="pdl", action="store_false", help="fully serialise the kernel launches")
     ap.add_argument("--e2e-io", default="kernel", choices=["kernel", "copy", "stage", "hostout"],

@@ -82,7 +82,6 @@ typedef struct eta_params {
     int32_t lwb;            /* the last `lwb` full blocks are always attended */
     int32_t rescue_window;  /* top-1 rescue looks at the first min(rescue_window, NB) blocks; >= 1 */
     uint32_t flags;         /* ETA_FLAG_* */
-    int32_t ctas_per_sm;    /* launch hint for the streaming kernel: 0 = library default */
 } eta_params;
 
 /*
@@ -101,9 +100,16 @@ int eta_workspace_bytes(const eta_cache_desc* desc, size_t* out_bytes);
  *   mu = mean of the b keys, sigma_c = sqrt(mean_k (k_c - mu_c)^2) (population),
  *   M = max_k ||k||_2
  * as fp16 / fp16 / fp32.  Records of blocks that are not full are left untouched.
- * Arithmetic is fp32 on the bf16 keys, two passes (mean first, then deviations).
+ * Arithmetic is fp32 on the bf16 keys, in one pass over the block: mu from the plain
+ * coordinate sums, sigma from squared deviations about the block's first key k0,
+ *   sigma_c^2 = (1/b) sum_k (k_c - k0_c)^2 - (mu_c - k0_c)^2   (clamped at 0),
+ * which is exact for identical keys and otherwise loses a factor
+ * 1 + (mu_c - k0_c)^2 / sigma_c^2 of fp32's precision, far inside the fp16 the
+ * result is stored in (results are within 1 fp16 ulp of the two-pass definition
+ * evaluated in double).
  * flags: ETA_BUILD_SIGMA_ENVELOPE stores max over 4-token sub-blocks of the
- * sub-block RMS deviation from mu instead of sigma.
+ * sub-block RMS deviation from mu instead of sigma (Eq. subblock_envelope_appx;
+ * this variant takes a second pass over the block for the deviations about mu).
  */
 int eta_build_block_summaries(const eta_cache_desc* desc, const void* K, const int32_t* seq_lens,
                               void* musig, float* mnorm, uint32_t flags, void* stream);
@@ -138,6 +144,14 @@ int eta_stage_query(int32_t batch, int32_t n_q_heads, int32_t head_dim, const vo
  * i (length n_q_heads * head_dim).  q bf16 [batch, n_q_heads, head_dim];
  * W fp32 [n_q_heads * head_dim, n_q_heads] row-major; bias fp32 [n_q_heads];
  * tau fp32 [batch, n_q_heads].  fp32 accumulation in a fixed order.
+ * Launch order: the kernel is launched with programmatic dependent launch and reads
+ * q, W and bias without waiting for the preceding kernel of the stream (it waits for
+ * it only before it exits, so that its completion implies its predecessor's).  The
+ * producer of q must therefore be complete when that preceding kernel starts: true
+ * for copies, for kernels launched without early dependent release (eta_stage_query
+ * and eta_append_summary's inputs among them) and for anything ordered by an event
+ * or a synchronisation; a kernel that releases its dependents early and then writes
+ * q would hand this call a stale query.
  */
 int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t head_dim, const void* q,
                           const float* W, const float* bias, float* tau, void* stream);
@@ -198,7 +212,8 @@ int eta_calibrate_head_const(int32_t n_seq, int32_t seq_len, int32_t n_q_heads, 
  * int32 [batch, n_kv_heads]) the number of blocks fetched per KV head;
  * status_dev (nullable, uint32, caller-zeroed) device-side problems.
  * bf16 operands, fp32 scores / softmax statistics / accumulators; deterministic
- * for a given device and launch hint.  workspace: eta_workspace_bytes() bytes.
+ * for a given device (the split of the work depends on its SM count only).
+ * workspace: eta_workspace_bytes() bytes.
  * Launch order: the kernels are launched with programmatic dependent launch and read q, seq_lens and every
  * summary except the newest block's before they wait for the preceding kernel of the stream.  Producers of those
  * inputs must therefore be complete when that preceding kernel starts: true for copies, for kernels launched
@@ -220,12 +235,16 @@ int eta_decode(const eta_cache_desc* desc, const eta_params* params, const void*
  * device and may fail once memory is fragmented.
  *
  * Same arguments, results and status codes as eta_decode, minus workspace / workspace_bytes.  The scratch is a
- * fixed array of ETA_STATIC_SCRATCH_BYTES (8 MiB) inside the library's CUDA module: every GPU that loads the
- * library holds it from load until the process exits.  The call allocates and frees nothing.
+ * fixed array of ETA_STATIC_SCRATCH_BYTES (8 MiB) inside the library's CUDA module: every GPU on which the
+ * module gets loaded holds it from then until the process exits.  The call allocates and frees nothing.
  *   - Limit: shapes for which eta_workspace_bytes() exceeds ETA_STATIC_SCRATCH_BYTES are refused with
  *     ETA_ERR_WORKSPACE before anything is launched (the five benchmark configurations need 0.8 - 3 MiB).
  *   - Set-up: the first call on each device looks up the array's device address (with that device current).
- *     Make that first call ahead of any stream capture.
+ *     Make that first call ahead of any stream capture, and ahead of handing the rest of the device's memory
+ *     to anybody else: CUDA loads a module lazily by default, so the array is reserved when the library's first
+ *     kernel is launched or its first symbol looked up on that device, not when the library is loaded.  A first
+ *     call that finds no memory left returns ETA_ERR_CUDA (eta_last_cuda_error names cudaGetSymbolAddress).
+ *     The address is looked up once per device and kept; it does not survive a cudaDeviceReset.
  *   - Sharing: all calls on a device use the same array, and it keeps the previous call's contents.  Nothing in
  *     it has to be cleared by the caller: each call writes every word before reading it.  For the same reason
  *     two calls whose kernels can overlap on the GPU (different streams, no dependency between them) race on
@@ -295,16 +314,6 @@ const char* eta_profile_kernel_name(int k);
  * wait for the full completion of the previous one instead (for A/B timing and for debugging).  Process-wide.
  */
 int eta_set_pdl(int on);
-
-/*
- * Development aid (the paper has no counterpart): when dev_buffer is a device array of at least
- * 8 * 1024 uint64, the kernels of a decode step write up to eight %globaltimer stamps (ns) per CTA (per warp in the
- * append kernel) at [k * 8 .. k * 8 + 7]: k = c for CTA c of the streaming kernel (entry, set-up done, first copy
- * issued, first tile consumed, last tile consumed, partials stored, prefix window loaded, dependency wait
- * returned), 512 + c for the screening kernel (c < 296), 808 + c for the merge kernel (c < 128), 936 + c for the
- * predictor (c < 32), 968 + r for row r of the append kernel (r < 48).  NULL switches it off (the default).
- */
-int eta_debug_timeline(void* dev_buffer);
 
 /* Text for an eta_status. */
 const char* eta_strerror(int code);

@@ -23,7 +23,7 @@ ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_build_block_summaries_paged",
            "eta_append_summary_paged", "eta_decode_paged", "eta_stage_query", "eta_predict_threshold",
            "eta_score_dual", "eta_calibration_workspace_bytes", "eta_calibrate_head_const", "eta_decode", "eta_decode_static", "eta_static_scratch_bytes", "eta_decode_kernel_count", "eta_profile_enable", "eta_profile_read",
-           "eta_profile_kernel_name", "eta_set_pdl", "eta_debug_timeline", "eta_strerror", "eta_last_cuda_error")
+           "eta_profile_kernel_name", "eta_set_pdl", "eta_strerror", "eta_last_cuda_error")
 
 
 class CacheDesc(ctypes.Structure):
@@ -36,8 +36,7 @@ class CacheDesc(ctypes.Structure):
 
 class Params(ctypes.Structure):
     _fields_ = [("z", ctypes.c_float), ("a", ctypes.c_float), ("beta", ctypes.c_float), ("scale", ctypes.c_float),
-                ("lwb", ctypes.c_int32), ("rescue_window", ctypes.c_int32), ("flags", ctypes.c_uint32),
-                ("ctas_per_sm", ctypes.c_int32)]
+                ("lwb", ctypes.c_int32), ("rescue_window", ctypes.c_int32), ("flags", ctypes.c_uint32)]
 
 
 class PageTable(ctypes.Structure):
@@ -86,7 +85,6 @@ def load() -> ctypes.CDLL:
         lib.eta_last_cuda_error.restype = ctypes.c_char_p
         lib.eta_profile_enable.argtypes = [ctypes.c_int]
         lib.eta_set_pdl.argtypes = [ctypes.c_int]
-        lib.eta_debug_timeline.argtypes = [ctypes.c_void_p]
         lib.eta_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int]
         lib.eta_profile_kernel_name.restype = ctypes.c_char_p
         lib.eta_profile_kernel_name.argtypes = [ctypes.c_int]
@@ -136,11 +134,9 @@ class DecodeParams:
     lwb: int = 0
     rescue_window: int = 128
     flags: int = 0
-    ctas_per_sm: int = 0
 
     def c(self) -> Params:
-        return Params(self.z, self.a, self.beta, self.scale, self.lwb, self.rescue_window, self.flags,
-                      self.ctas_per_sm)
+        return Params(self.z, self.a, self.beta, self.scale, self.lwb, self.rescue_window, self.flags)
 
 
 def cache_desc(K: torch.Tensor, V: torch.Tensor, n_q_heads: int, block_size: int, nb_cap: int | None = None) -> CacheDesc:

@@ -3,7 +3,10 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "eta_common.cuh"
+#include "eta_timeline.h"
 
 namespace eta {
 
@@ -56,19 +59,60 @@ void profile_mark(int k, cudaStream_t s) {
     g_ev_seen |= 1u << k;
 }
 
+#ifdef ETA_TIMELINE
 static unsigned long long* g_timeline = nullptr;
 unsigned long long* debug_timeline() { return g_timeline; }
+#endif
 static bool g_pdl = true;
 bool pdl_enabled() { return g_pdl; }
 void set_pdl(bool on) { g_pdl = on; }
 
-void prefer_max_shared(const void* kernel) {
-    static const void* seen[64];
-    static int n_seen = 0;
-    for (int k = 0; k < n_seen; ++k)
-        if (seen[k] == kernel) return;
-    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (n_seen < 64) seen[n_seen++] = kernel;
+// ---- per-device kernel attributes
+// cudaFuncAttributeMaxDynamicSharedMemorySize and the shared-memory carve-out belong to a (device, kernel) pair: a
+// process that uses a second GPU has to set them there again.  The table below remembers, per device ordinal and
+// kernel, the dynamic shared memory already granted and whether the carve-out was asked for; look-ups and updates
+// are serialised by a mutex (two host threads may launch at once).  The setter is a parameter so that the
+// bookkeeping can be exercised without a device.
+int KernelAttrTable::configure(int dev, const void* kernel, size_t dyn_smem, Setter set, void* ctx) {
+    std::lock_guard<std::mutex> lock(mu_);
+    Entry* e = nullptr;
+    if (dev >= 0 && dev < MAX_DEVICES) {
+        for (int k = 0; k < n_[dev]; ++k)
+            if (tab_[dev][k].kernel == kernel) e = &tab_[dev][k];
+        if (!e && n_[dev] < MAX_KERNELS) {
+            e = &tab_[dev][n_[dev]++];
+            e->kernel = kernel; e->smem = 0; e->carveout = false;
+        }
+    }
+    // a device or kernel beyond the table's capacity is configured on every call: slower, never wrong
+    if (!e || !e->carveout) {
+        const int rc = set(ctx, kernel, ATTR_CARVEOUT, 0);
+        if (rc != 0) return rc;
+        if (e) e->carveout = true;
+    }
+    if (dyn_smem > DEFAULT_DYN_SMEM && (!e || dyn_smem > e->smem)) {
+        const int rc = set(ctx, kernel, ATTR_MAX_DYN_SMEM, dyn_smem);
+        if (rc != 0) return rc;
+        if (e) e->smem = dyn_smem;
+    }
+    return 0;
+}
+
+static KernelAttrTable g_attr_table;
+
+static int cuda_setter(void*, const void* kernel, int attr, size_t value) {
+    const cudaError_t e = (attr == KernelAttrTable::ATTR_CARVEOUT)
+        ? cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)
+        : cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)value);
+    if (e != cudaSuccess) { set_cuda_error(e, "kernel attribute"); return ETA_ERR_CUDA; }
+    return 0;
+}
+
+int configure_kernel(const void* kernel, size_t dyn_smem) {
+    int dev = 0;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return ETA_ERR_CUDA; }
+    return g_attr_table.configure(dev, kernel, dyn_smem, cuda_setter, nullptr);
 }
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -117,10 +161,41 @@ const char* eta_strerror(int code) {
 
 const char* eta_last_cuda_error(void) { return eta::g_cuda_error; }
 
+// Host-only check of the per-device attribute bookkeeping with a recording setter and made-up device ordinals
+// (no device is touched).  Not part of the public interface; called by the CPU test-suite.  -> 0, or the number of
+// the first expectation that failed.
+int eta_selftest_kernel_attr_table(void) {
+    using T = eta::KernelAttrTable;
+    struct Log { int carve = 0, smem = 0; size_t last = 0; } log;
+    auto rec = [](void* ctx, const void*, int attr, size_t v) {
+        Log* l = static_cast<Log*>(ctx);
+        if (attr == T::ATTR_CARVEOUT) ++l->carve; else { ++l->smem; l->last = v; }
+        return 0;
+    };
+    static T t;                        // own instance: the library's table is left alone
+    int ka = 0, kb = 0;
+    const void *A = &ka, *B = &kb;
+    if (t.configure(0, A, 200 * 1024, rec, &log) != 0 || log.carve != 1 || log.smem != 1) return 1;
+    if (t.configure(0, A, 200 * 1024, rec, &log) != 0 || log.carve != 1 || log.smem != 1) return 2;   // remembered
+    if (t.configure(1, A, 200 * 1024, rec, &log) != 0 || log.carve != 2 || log.smem != 2) return 3;   // second device: again
+    if (t.configure(1, A, 100 * 1024, rec, &log) != 0 || log.smem != 2) return 4;                      // smaller: nothing
+    if (t.configure(1, A, 220 * 1024, rec, &log) != 0 || log.smem != 3 || log.last != 220 * 1024) return 5;
+    if (t.configure(0, B, 16 * 1024, rec, &log) != 0 || log.carve != 3 || log.smem != 3) return 6;     // under 48 KB: carve-out only
+    if (t.configure(T::MAX_DEVICES + 3, A, 200 * 1024, rec, &log) != 0 || log.carve != 4 || log.smem != 4) return 7;
+    if (t.configure(T::MAX_DEVICES + 3, A, 200 * 1024, rec, &log) != 0 || log.carve != 5 || log.smem != 5) return 8;  // untracked: every call
+    auto fail = [](void*, const void*, int, size_t) { return -4; };
+    int kc = 0;
+    if (t.configure(2, &kc, 200 * 1024, fail, nullptr) != -4) return 9;
+    if (t.configure(2, &kc, 200 * 1024, rec, &log) != 0 || log.carve != 6 || log.smem != 6) return 10;  // a failure is not remembered
+    return 0;
+}
+
+#ifdef ETA_TIMELINE
 int eta_debug_timeline(void* dev_buffer) {
     eta::g_timeline = static_cast<unsigned long long*>(dev_buffer);
     return ETA_OK;
 }
+#endif
 
 int eta_set_pdl(int on) {
     eta::set_pdl(on != 0);

@@ -240,21 +240,13 @@ int eta_calibrate_head_const(int32_t n_seq, int32_t seq_len, int32_t n_q_heads, 
     auto Qp = static_cast<const __nv_bfloat16*>(Q);
     auto Kp = static_cast<const __nv_bfloat16*>(K);
     if (head_dim == 128) {
-        static bool configured = false;
-        if (!configured) {
-            e = cudaFuncSetAttribute(calib_hist_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-            if (e != cudaSuccess) { set_cuda_error(e, "calibration smem attribute"); return ETA_ERR_CUDA; }
-            configured = true;
-        }
+        rc = configure_kernel(reinterpret_cast<const void*>(calib_hist_kernel<128>), 64 * 1024);
+        if (rc != ETA_OK) return rc;
         calib_hist_kernel<128><<<grid, CAL_THREADS, smem, s>>>(Qp, Kp, tau, n_q_heads, n_kv_heads, seq_len, beta, sc,
                                                                n_bins, s_min, inv_w, hist, dpart);
     } else {
-        static bool configured = false;
-        if (!configured) {
-            e = cudaFuncSetAttribute(calib_hist_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-            if (e != cudaSuccess) { set_cuda_error(e, "calibration smem attribute"); return ETA_ERR_CUDA; }
-            configured = true;
-        }
+        rc = configure_kernel(reinterpret_cast<const void*>(calib_hist_kernel<64>), 64 * 1024);
+        if (rc != ETA_OK) return rc;
         calib_hist_kernel<64><<<grid, CAL_THREADS, smem, s>>>(Qp, Kp, tau, n_q_heads, n_kv_heads, seq_len, beta, sc,
                                                               n_bins, s_min, inv_w, hist, dpart);
     }

@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
 #include <utility>
 
 #include "../../include/eta.h"
@@ -101,17 +102,43 @@ int launch_screen(const ScreenArgs& a, int rows, int D, int G, int n_ctas, cudaS
 
 // Launch with programmatic dependent launch allowed: the grid may start while its predecessor in the stream is
 // still draining, and must call pdl_wait() before touching anything the predecessor wrote.
-unsigned long long* debug_timeline();   // device buffer for per-CTA time stamps, or nullptr (see eta_debug_timeline)
+// Per-CTA %globaltimer stamps exist in development builds only (-DETA_TIMELINE, see eta_timeline.h): in the shipped
+// build ETA_TL() is a constant null pointer, so every `if (tl && ...)` below it is compiled out.
+#ifdef ETA_TIMELINE
+#define ETA_TL(expr) (expr)
+unsigned long long* debug_timeline();   // device buffer for the stamps, or nullptr
+#else
+#define ETA_TL(expr) (static_cast<unsigned long long*>(nullptr))
+inline unsigned long long* debug_timeline() { return nullptr; }
+#endif
 bool pdl_enabled();          // false after eta_set_pdl(0): every launch is then fully serialised
-// Asks (once per kernel) for the largest shared-memory carve-out.  The streaming kernel needs it; when its
-// neighbours in the stream run with another split of the SM's L1/shared memory, an SM has to drain and
-// reconfigure before the first CTA of the next kernel can start on it, which showed as ~2 us between the last CTA of
-// one kernel and the first of the next.  None of the kernels of a step depends on L1 capacity.
-void prefer_max_shared(const void* kernel);
+// Per-(device, kernel) attribute set-up, remembered per device ordinal under a mutex (see eta_api.cu).
+// Every kernel of a step asks for the largest shared-memory carve-out: the streaming kernel needs it, and when its
+// neighbours in the stream run with another split of the SM's L1/shared memory, an SM has to drain and reconfigure
+// before the first CTA of the next kernel can start on it, which showed as ~2 us between the last CTA of one kernel
+// and the first of the next.  None of the kernels of a step depends on L1 capacity.  dyn_smem above 48 KB is granted
+// with cudaFuncAttributeMaxDynamicSharedMemorySize.  -> ETA_OK or ETA_ERR_CUDA.
+int configure_kernel(const void* kernel, size_t dyn_smem);
+
+class KernelAttrTable {
+public:
+    static constexpr int MAX_DEVICES = 64, MAX_KERNELS = 64;
+    static constexpr size_t DEFAULT_DYN_SMEM = 48 * 1024;
+    enum { ATTR_CARVEOUT = 0, ATTR_MAX_DYN_SMEM = 1 };
+    typedef int (*Setter)(void* ctx, const void* kernel, int attr, size_t value);
+    int configure(int dev, const void* kernel, size_t dyn_smem, Setter set, void* ctx);
+private:
+    struct Entry { const void* kernel; size_t smem; bool carveout; };
+    std::mutex mu_;
+    Entry tab_[MAX_DEVICES][MAX_KERNELS] = {};
+    int n_[MAX_DEVICES] = {};
+};
+
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
-                              Args&&... args) {
-    prefer_max_shared(reinterpret_cast<const void*>(kernel));
+inline int launch_pdl(const char* what, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                      Args&&... args) {
+    const int rc = configure_kernel(reinterpret_cast<const void*>(kernel), smem);
+    if (rc != ETA_OK) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -122,7 +149,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    if (e != cudaSuccess) { set_cuda_error(e, what); return ETA_ERR_CUDA; }
+    return check_launch(what);
 }
 
 // -------------------------------------------------------------- device side

@@ -22,6 +22,7 @@
 #include <cuda.h>
 
 #include "eta_common.cuh"
+#include "eta_timeline.h"
 
 namespace eta {
 
@@ -164,7 +165,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     int32_t* resc_tab = reinterpret_cast<int32_t*>(smem + L::RESC_OFF);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    unsigned long long* tl = a.timeline ? a.timeline + (size_t)blockIdx.x * 8 : nullptr;
+    unsigned long long* const tl = ETA_TL(a.timeline ? a.timeline + (size_t)(TL_DECODE + blockIdx.x) * 8 : nullptr);
     if (tl && tid == 0) tl[0] = globaltimer_ns();
     // When NSTAGE is not a multiple of NGROUPS a stage serves different groups in successive rounds, and a parity
     // wait only tells the current phase of a barrier from the one before it: a group that runs ahead could ask for
@@ -919,7 +920,7 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
-    unsigned long long* tl = (a.timeline && blockIdx.x < 128) ? a.timeline + (size_t)(808 + blockIdx.x) * 8 : nullptr;
+    unsigned long long* const tl = ETA_TL((a.timeline && blockIdx.x < TL_MERGE_N) ? a.timeline + (size_t)(TL_MERGE + blockIdx.x) * 8 : nullptr);
     if (tl && tid == 0) tl[0] = globaltimer_ns();
     pdl_trigger();
     pdl_wait();          // every partial of the streaming kernel is in memory from here on
@@ -1060,17 +1061,8 @@ template <int D, int TS, int NSTAGE, int NGROUPS>
 static int launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const DecodeArgs& a, int n_ctas,
                            cudaStream_t s) {
     const size_t smem = DecodeSmem<D, TS, NSTAGE, NGROUPS>::bytes(a.G);
-    static size_t configured = 0;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, TS, NSTAGE, NGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
-        if (e != cudaSuccess) { set_cuda_error(e, "decode smem attribute"); return ETA_ERR_CUDA; }
-        configured = smem;
-    }
-    cudaError_t e = launch_pdl(decode_kernel<D, TS, NSTAGE, NGROUPS>, dim3(n_ctas),
-                               dim3(32 * (WARPS_PER_GROUP * NGROUPS + 1)), smem, s, tmK, tmV, a);
-    if (e != cudaSuccess) { set_cuda_error(e, "decode launch"); return ETA_ERR_CUDA; }
-    return check_launch("decode");
+    return launch_pdl("decode launch", decode_kernel<D, TS, NSTAGE, NGROUPS>, dim3(n_ctas),
+                      dim3(32 * (WARPS_PER_GROUP * NGROUPS + 1)), smem, s, tmK, tmV, a);
 }
 
 // eta_decode and eta_decode_paged: `pages` null selects the contiguous cache
@@ -1173,11 +1165,10 @@ static int decode_impl(const eta_cache_desc* desc, const eta_page_table* pages, 
     ma.row_span = da.row_span; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
     ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS; ma.timeline = debug_timeline();
     const unsigned mgrid = (unsigned)(L.rows * G);
-    cudaError_t me = (D == 128) ? launch_pdl(merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
-                                : launch_pdl(merge_kernel<64>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma);
-    if (me != cudaSuccess) { set_cuda_error(me, "merge launch"); return ETA_ERR_CUDA; }
+    rc = (D == 128) ? launch_pdl("merge launch", merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
+                    : launch_pdl("merge launch", merge_kernel<64>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma);
     profile_mark(5, s);
-    return check_launch("merge");
+    return rc;
 }
 
 }  // namespace eta

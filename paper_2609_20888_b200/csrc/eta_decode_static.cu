@@ -6,8 +6,11 @@
 // enter the CUDA allocator because cudaMalloc synchronises the device and can
 // fail once memory is fragmented.  For them the scratch eta_decode needs lives
 // here, in a file-scope __device__ array that the CUDA module carries: it is
-// reserved on every GPU that loads the library, from load until the process
-// exits, and no call allocates or frees anything.
+// reserved on every GPU on which the module gets loaded (with CUDA's default
+// lazy loading: at the library's first kernel launch or symbol look-up on that
+// device, so a caller makes one warm-up call before it gives the rest of the
+// memory away), until the process exits, and no call allocates or frees
+// anything.
 #include <mutex>
 
 #include "eta_common.cuh"

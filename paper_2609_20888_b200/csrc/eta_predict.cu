@@ -13,6 +13,7 @@
 #include <stdint.h>
 
 #include "eta_common.cuh"
+#include "eta_timeline.h"
 
 namespace cg = cooperative_groups;
 
@@ -25,8 +26,8 @@ __global__ void __launch_bounds__(PRED_THREADS) predict_threshold_kernel(
     const __nv_bfloat16* __restrict__ q, const float* __restrict__ W, const float* __restrict__ bias,
     float* __restrict__ tau, int Hq, int rows, int vec4, unsigned long long* timeline) {
     extern __shared__ float sm[];
-    unsigned long long* tl = timeline ? timeline + (size_t)(936 + blockIdx.y * PRED_CLUSTER + blockIdx.x) * 8 : nullptr;
-    if (tl && blockIdx.y * PRED_CLUSTER + blockIdx.x >= 32) tl = nullptr;
+    unsigned long long* const tl = ETA_TL((timeline && blockIdx.y * PRED_CLUSTER + blockIdx.x < TL_PREDICT_N)
+                                              ? timeline + (size_t)(TL_PREDICT + blockIdx.y * PRED_CLUSTER + blockIdx.x) * 8 : nullptr);
     if (tl && threadIdx.x == 0) tl[0] = globaltimer_ns();
     const int NRG = PRED_THREADS / Hq;           // row groups inside a CTA
     float* part = sm;                            // [max(NRG, warps)][Hq] partial sums of this CTA
@@ -148,7 +149,8 @@ extern "C" int eta_stage_query(int32_t batch, int32_t n_q_heads, int32_t head_di
     const int n16 = (int)(bytes / 16);
     int grid = (n16 + 255) / 256;
     if (grid > 296) grid = 296;
-    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::stage_query_kernel));
+    const int rc = eta::configure_kernel(reinterpret_cast<const void*>(eta::stage_query_kernel), 0);
+    if (rc != ETA_OK) return rc;
     eta::stage_query_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(q_host),
                                                                                  static_cast<uint4*>(q_dev), n16);
     return eta::check_launch("eta_stage_query");
@@ -185,7 +187,8 @@ extern "C" int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t h
     attr[1].val.programmaticStreamSerializationAllowed = eta::pdl_enabled() ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::predict_threshold_kernel));
+    const int rc = eta::configure_kernel(reinterpret_cast<const void*>(eta::predict_threshold_kernel), smem);
+    if (rc != ETA_OK) return rc;
     eta::profile_mark(1, cfg.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, eta::predict_threshold_kernel, static_cast<const __nv_bfloat16*>(q), W,
                                        bias, tau, (int)n_q_heads, rows, vec4, eta::debug_timeline());

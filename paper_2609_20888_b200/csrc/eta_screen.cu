@@ -18,6 +18,7 @@
 // count, largest bound and its index per head); the streaming kernel combines
 // them when it lays out its work.
 #include "eta_common.cuh"
+#include "eta_timeline.h"
 
 namespace eta {
 
@@ -73,7 +74,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool dense = (a.flags & ETA_FLAG_DENSE) != 0;
-    unsigned long long* tl = (a.timeline && blockIdx.x < 296) ? a.timeline + (size_t)(512 + blockIdx.x) * 8 : nullptr;
+    unsigned long long* const tl = ETA_TL((a.timeline && blockIdx.x < TL_SCREEN_N) ? a.timeline + (size_t)(TL_SCREEN + blockIdx.x) * 8 : nullptr);
     if (tl && tid == 0) tl[0] = globaltimer_ns();
 
     const int n_items = a.rows * a.nseg;
@@ -558,12 +559,6 @@ __global__ void __launch_bounds__(128) score_dual_kernel(
 template <int D, int G>
 static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream_t s) {
     const size_t smem = ScreenSmem<D, G>::BYTES;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(screen_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { set_cuda_error(e, "screen smem attribute"); return ETA_ERR_CUDA; }
-        configured = true;
-    }
     // The slowest CTA sets the kernel's end.  All CTAs are resident at once (n_ctas = two per SM), but under
     // programmatic dependent launch the kernel starts while its predecessors (summary append, threshold predictor)
     // still hold some SMs, where no CTA of this kernel fits until they exit: the CTAs dispatched last (the
@@ -599,9 +594,7 @@ static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream
         b2.n_early = grid;
         b2.per_early = n_items;
     }
-    cudaError_t e = launch_pdl(screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, b2);
-    if (e != cudaSuccess) { set_cuda_error(e, "screen launch"); return ETA_ERR_CUDA; }
-    return check_launch("screen");
+    return launch_pdl("screen launch", screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, b2);
 }
 
 int launch_screen(const ScreenArgs& a, int rows, int D, int G, int n_ctas, cudaStream_t s) {

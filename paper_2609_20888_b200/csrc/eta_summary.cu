@@ -12,6 +12,7 @@
 // from L1/L2.  Arithmetic is fp32.  Build and append share these routines, so
 // appending a block gives the same bytes as rebuilding the index.
 #include "eta_common.cuh"
+#include "eta_timeline.h"
 
 namespace eta {
 
@@ -252,7 +253,7 @@ __global__ void __launch_bounds__(128) append_summary_kernel(
     int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
     float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride, unsigned long long* timeline) {
     const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
-    unsigned long long* tl = (timeline && r < 48) ? timeline + (size_t)(968 + r) * 8 : nullptr;
+    unsigned long long* const tl = ETA_TL((timeline && r < TL_APPEND_N) ? timeline + (size_t)(TL_APPEND + r) * 8 : nullptr);
     if (tl && (threadIdx.x & 31) == 0) tl[0] = globaltimer_ns();
     pdl_trigger();       // nothing later in a decode step needs this kernel's output before it has waited for it
     if (r >= rows) return;
@@ -319,8 +320,9 @@ static int append_impl(const eta_cache_desc* desc, const eta_page_table* pages, 
     const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
     auto Kp = static_cast<const __nv_bfloat16*>(K);
     auto mp = static_cast<__half*>(musig);
-    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::append_summary_kernel<128>));
-    eta::prefer_max_shared(reinterpret_cast<const void*>(eta::append_summary_kernel<64>));
+    rc = eta::configure_kernel(desc->head_dim == 128 ? reinterpret_cast<const void*>(eta::append_summary_kernel<128>)
+                                                     : reinterpret_cast<const void*>(eta::append_summary_kernel<64>), 0);
+    if (rc != ETA_OK) return rc;
     eta::profile_mark(0, s);
     if (desc->head_dim == 128)
         eta::append_summary_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,

@@ -75,6 +75,14 @@ def test_null_and_inconsistent_arguments_are_rejected_before_any_launch(lib):
     assert lib.eta_decode(*args2, one, null, *tail) == -1
 
 
+def test_kernel_attributes_are_remembered_per_device(lib):
+    """cudaFuncSetAttribute results hold per (device, kernel): the library's bookkeeping must ask again on a second
+    device, ask again for more shared memory, not ask twice for the same, and never remember a failure.  Host-only
+    self-check with made-up device ordinals and a recording setter; 0 = every expectation held."""
+    lib.eta_selftest_kernel_attr_table.restype = ctypes.c_int
+    assert lib.eta_selftest_kernel_attr_table() == 0
+
+
 def test_status_text(lib):
     assert lib.eta_strerror(0) == b"ok"
     assert b"workspace" in lib.eta_strerror(-3)
