@@ -133,7 +133,8 @@ struct DecodeSmem {
     static constexpr int WIN_OFF = DESC_OFF + 16 * NSTAGE;      // int32 pwin[PW + 1] (+3 pad): window of the unit prefix
     static constexpr int ROW_OFF = WIN_OFF + 4 * (PW + 4);      // int32 rowbase[MAX_ROWS + 1]: unit prefix over rows
     static constexpr int INFO_OFF = ROW_OFF + 4 * (MAX_ROWS + 4);   // uint8 per row: rescue units | tail flag << 7
-    static constexpr int RESC_OFF = INFO_OFF + MAX_ROWS;        // int32 [RESC_ROWS][8]: rescued block per head, first rows
+    static constexpr int NZP_OFF = INFO_OFF + MAX_ROWS;         // uint16 per row: rows with at least one unit before the row
+    static constexpr int RESC_OFF = NZP_OFF + 2 * MAX_ROWS;     // int32 [RESC_ROWS][8]: rescued block per head, first rows
     static constexpr int ML_OFF = RESC_OFF + 4 * 8 * RESC_ROWS; // float m[NGROUPS][4][8], l[NGROUPS][4][8]
     static constexpr int MO_OFF = ML_OFF + 4 * 2 * NGROUPS * WARPS_PER_GROUP * 8;
     static size_t bytes(int G) { return 1024 + MO_OFF + sizeof(float) * NGROUPS * WARPS_PER_GROUP * G * D; }
@@ -162,10 +163,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     int32_t* pwin = reinterpret_cast<int32_t*>(smem + L::WIN_OFF);
     int32_t* rowbase = reinterpret_cast<int32_t*>(smem + L::ROW_OFF);
     uint8_t* rowinfo = smem + L::INFO_OFF;
+    uint16_t* nzp = reinterpret_cast<uint16_t*>(smem + L::NZP_OFF);
     int32_t* resc_tab = reinterpret_cast<int32_t*>(smem + L::RESC_OFF);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long* const tl = ETA_TL(a.timeline ? a.timeline + (size_t)(TL_DECODE + blockIdx.x) * 8 : nullptr);
+    unsigned long long* const tl2 = ETA_TL(a.timeline ? a.timeline + (size_t)(TL_DECODE2 + blockIdx.x) * 8 : nullptr);
     if (tl && tid == 0) tl[0] = globaltimer_ns();
     // When NSTAGE is not a multiple of NGROUPS a stage serves different groups in successive rounds, and a parity
     // wait only tells the current phase of a barrier from the one before it: a group that runs ahead could ask for
@@ -185,152 +188,118 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     // scratch for the layout, in the (still unused) stage memory
     constexpr int NWARPS = WARPS_PER_GROUP * NGROUPS + 1;
     constexpr int NTHREADS = 32 * NWARPS;
-    int* cnt32 = reinterpret_cast<int*>(smem);                 // [rows] surviving blocks of the row
-    int* resc_j = cnt32 + MAX_ROWS;                            // [rows][8] rescued block per head, -1: none
+    int* resc_j = reinterpret_cast<int*>(smem);                // [rows][8] rescued block per head, -1: none
     int* s_len = resc_j + 8 * MAX_ROWS;                        // [rows] clamped sequence length
-    int* nzp = s_len + MAX_ROWS;                               // [rows] rows with at least one unit before the row
-    uint8_t* cnt8 = reinterpret_cast<uint8_t*>(nzp + MAX_ROWS);     // [rows * nseg] survivors per segment
-    const bool counts_in_smem = (size_t)a.rows * a.nseg + 11 * 4 * MAX_ROWS <= (size_t)NSTAGE * L::STAGE_BYTES;
+    int* rowcnt = s_len + MAX_ROWS;                            // [rows] surviving blocks of the row
+    // [rows][nseg + 2] units per entry of the flattened sequence: a row's segments (surviving blocks), then its rescue
+    // units, then its tail (0 or 1): what the producer's first prefix window is summed from, one byte load per entry
+    uint8_t* cnt8 = reinterpret_cast<uint8_t*>(rowcnt + MAX_ROWS);
+    const bool counts_in_smem = (size_t)a.entries + 10 * 4 * MAX_ROWS <= (size_t)NSTAGE * L::STAGE_BYTES;
     // sequence lengths are a caller input: they can be read while the previous kernel is still running
     for (int rr = tid; rr < a.rows; rr += NTHREADS) {
         const int T = __ldg(a.seq_lens + a.div_hkv.div(rr));
         s_len[rr] = T < 0 ? 0 : (T > a.t_cap ? a.t_cap : T);
-        cnt32[rr] = 0;
+        rowcnt[rr] = 0;
     }
     __syncthreads();
     pdl_wait();          // the screening kernel's lists, counts and window statistics are complete from here on
     if (tl && tid == 0) tl[7] = globaltimer_ns();
+    const unsigned long long clk0 = ETA_TL(reinterpret_cast<unsigned long long*>(1)) ? (unsigned long long)clock64() : 0ull;
 
     // ---- every CTA lays out the flattened unit sequence for itself: per row the surviving blocks of its
-    // segments, then its rescued blocks, then its tail; a scan over the rows gives each row's first unit
-    __shared__ int s_lay[4];      // rows that have at least one unit; the CTA's unit range; CTAs that share the units
+    // segments, then its rescued blocks, then its tail; a scan over the rows gives each row's first unit.
+    // The code below runs once per CTA on a cold instruction cache, where every instruction costs tens of cycles:
+    // it is written as small loops rather than unrolled, and with as few dependent round trips to L2 as the data
+    // allow (one for the counts and window statistics, later one for the first list words).
+    __shared__ int s_lay[5];      // rows with units; the CTA's unit range; CTAs that share the units; row of the first unit
     {
-        __shared__ int s_wsum[32];
-        // all loads of the layout are independent and issued together: segment counts (summed per row with
-        // shared-memory atomics) and, per (row, head), the window statistics of the rescue window's segments
-        for (int e0 = tid; e0 < a.rows * a.nseg; e0 += 8 * NTHREADS) {
-            int cv[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int e = e0 + k * NTHREADS;
-                cv[k] = (e < a.rows * a.nseg) ? __ldg(a.seg_count + e) : 0;
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int e = e0 + k * NTHREADS;
-                if (e < a.rows * a.nseg) {
-                    if (counts_in_smem) cnt8[e] = (uint8_t)cv[k];
-                    if (cv[k]) atomicAdd(&cnt32[a.div_nseg.div(e)], cv[k]);
-                }
-            }
-        }
-        for (int p = tid; p < a.rows * a.G; p += NTHREADS) {
+        // All loads of the layout are independent and issued together, before any of them is consumed: per thread
+        // eight segment counts and, for the thread's (row, head) pair, the window statistics of up to four segments
+        // of the rescue window.
+        const int n_cnt = a.rows * a.nseg, n_rh = a.rows * a.G;
+        auto resc_load = [&](int p, int s0, int4 (&raw)[4], int& Wr) {
             int rr, g;
             a.div_g.divmod(p, rr, g);
-            const int NB = min(s_len[rr] / a.b, a.nb_cap);
-            resc_j[rr * 8 + g] = rescue_of(a.seg_resc, rr, g, a.G, a.nseg, min(a.rescue_window, NB));
-        }
-        __syncthreads();
-        // units of row rr (surviving blocks, rescued blocks, tail); heads that rescue the same block share one unit
-        auto row_units = [&](int rr) {
-            const int tailf = (s_len[rr] & (a.b - 1)) ? 1 : 0;
-            int resc = 0;
-            for (int g = 0; g < a.G; ++g) {
-                const int j = resc_j[rr * 8 + g];
-                if (j < 0) continue;
-                bool dup = false;
-                for (int g2 = 0; g2 < g; ++g2) dup = dup || (resc_j[rr * 8 + g2] == j);
-                if (!dup) ++resc;
-            }
-            rowinfo[rr] = (uint8_t)(resc | (tailf << 7));
-            return cnt32[rr] + resc + tailf;
+            Wr = (p < n_rh) ? min(a.rescue_window, min(s_len[min(rr, a.rows - 1)] / a.b, a.nb_cap)) : 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                raw[k] = ((s0 + k) * SEG < Wr)
+                    ? __ldg(reinterpret_cast<const int4*>(a.seg_resc + ((int64_t)rr * a.nseg + s0 + k) * a.G + g))
+                    : make_int4(0, 0, -1, 0);
         };
-        if (a.rows <= 32) {
-            // one warp lays out up to 32 rows in registers: no block-wide barrier until the split is known
-            if (warp == 0) {
-                const int units = lane < a.rows ? row_units(lane) : 0;
-                const int nzf = units > 0 ? 1 : 0;
-                int iu = units, iz = nzf;
+        // combines window statistics in ascending segment order: the admitted counts add up, the largest bound
+        // wins, the first block among equal bounds
+        auto resc_fold = [&](const int4 (&raw)[4], int& cnt, float& best, int& arg) {
 #pragma unroll
-                for (int s = 1; s < 32; s <<= 1) {
-                    const int ou = __shfl_up_sync(0xffffffffu, iu, s);
-                    const int oz = __shfl_up_sync(0xffffffffu, iz, s);
-                    if (lane >= s) { iu += ou; iz += oz; }
-                }
-                if (lane < a.rows) { rowbase[lane] = iu - units; nzp[lane] = iz - nzf; }
-                if (lane == 31) { rowbase[a.rows] = iu; s_lay[0] = iz; }
+            for (int k = 0; k < 4; ++k) {
+                cnt += raw[k].x;
+                const float mb = __int_as_float(raw[k].y);
+                if (raw[k].z >= 0 && mb > best) { best = mb; arg = raw[k].z; }
             }
-        } else {
-            for (int rr = tid; rr < a.rows; rr += NTHREADS) rowbase[rr] = row_units(rr);
-            __syncthreads();
-            // exclusive block scan over the rows: value of row rr from get(rr), prefix handed to put(rr, prefix)
-            auto scan_rows = [&](auto get, auto put) {
-                int carry = 0;
-                for (int r0 = 0; r0 < a.rows; r0 += NTHREADS) {
-                    const int rr = r0 + tid;
-                    const int c = (rr < a.rows) ? get(rr) : 0;
-                    int incl = c;
+        };
+        auto count_consume = [&](int e, int c) {
+            if (e < n_cnt) {
+                const int rr = a.div_nseg.div(e);
+                if (counts_in_smem) cnt8[e + 2 * rr] = (uint8_t)c;       // entry rr (nseg + 2) + segment
+                if (c) atomicAdd(&rowcnt[rr], c);
+            }
+        };
+        int4 raw[4];
+        int Wr;
+        resc_load(tid, 0, raw, Wr);
+        int cv[8];
 #pragma unroll
-                    for (int s = 1; s < 32; s <<= 1) {
-                        const int o = __shfl_up_sync(0xffffffffu, incl, s);
-                        if (lane >= s) incl += o;
+        for (int k = 0; k < 8; ++k) {
+            const int e = tid + k * NTHREADS;
+            cv[k] = (e < n_cnt) ? __ldg(a.seg_count + e) : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) count_consume(tid + k * NTHREADS, cv[k]);
+        for (int e0 = tid + 8 * NTHREADS; e0 < n_cnt; e0 += NTHREADS) count_consume(e0, __ldg(a.seg_count + e0));
+        // Top-1 rescue of head g of row rr (Algorithm 3, rescue phase): if none of the first
+        // Wr = min(rescue_window, NB) blocks was admitted for the head, the first block with the largest bound among
+        // them is.  The G heads of a row sit in consecutive lanes of one warp: a head whose block an earlier head of
+        // the row rescued too shares that head's fetch unit.
+        for (int p0 = 0; p0 < n_rh; p0 += NTHREADS) {
+            const int p = p0 + tid;
+            if (p0 > 0) resc_load(p, 0, raw, Wr);
+            int cnt = 0, arg = -1;
+            float best = -INFINITY;
+            resc_fold(raw, cnt, best, arg);
+            for (int s0 = 4; s0 * SEG < Wr; s0 += 4) {      // windows of more than four segments
+                resc_load(p, s0, raw, Wr);
+                resc_fold(raw, cnt, best, arg);
+            }
+            const int rj = (p < n_rh && Wr > 0 && cnt == 0) ? (arg < 0 ? 0 : arg) : -1;
+            int rr, g;
+            a.div_g.divmod(p, rr, g);
+            bool dup = false;
+            for (int o = 1; o < a.G; ++o) {
+                const int jo = __shfl_up_sync(0xffffffffu, rj, o);
+                dup = dup || (o <= g && jo == rj);
+            }
+            const unsigned uniq = __ballot_sync(0xffffffffu, rj >= 0 && !dup);
+            if (p < n_rh) {
+                resc_j[rr * 8 + g] = rj;
+                if (g == 0) {
+                    const int n_resc = __popc((uniq >> (lane & 31)) & ((1u << a.G) - 1u));
+                    const int tailf = (s_len[rr] & (a.b - 1)) ? 1 : 0;
+                    rowinfo[rr] = (uint8_t)(n_resc | (tailf << 7));
+                    if (counts_in_smem) {
+                        cnt8[rr * (a.nseg + 2) + a.nseg] = (uint8_t)n_resc;
+                        cnt8[rr * (a.nseg + 2) + a.nseg + 1] = (uint8_t)tailf;
                     }
-                    if (lane == 31) s_wsum[warp] = incl;
-                    __syncthreads();
-                    int wbase = 0, tot = 0;
-                    for (int w = 0; w < NWARPS; ++w) {
-                        const int v = s_wsum[w];
-                        if (w < warp) wbase += v;
-                        tot += v;
-                    }
-                    if (rr < a.rows) put(rr, carry + wbase + incl - c);
-                    carry += tot;
-                    __syncthreads();
                 }
-                return carry;
-            };
-            // nzp <- rows with at least one unit before row rr; rowbase <- units before row rr
-            const int nz_total = scan_rows([&](int rr) { return rowbase[rr] > 0 ? 1 : 0; },
-                                           [&](int rr, int p) { nzp[rr] = p; });
-            const int u_total = scan_rows([&](int rr) { return rowbase[rr]; }, [&](int rr, int p) { rowbase[rr] = p; });
-            if (tid == 0) { rowbase[a.rows] = u_total; s_lay[0] = nz_total; }
-            __syncthreads();
+            }
         }
     }
-    // Equal shares of COST, not of units: a row that starts inside a CTA's range costs that CTA a flush of its
-    // partials and a query reload, worth about PIECE_COST tiles.  Row rr spans the cost interval
-    // [rowbase[rr] + PIECE_COST * nzp[rr], +PIECE_COST (if it has units) + its units).  Two lanes of the first
-    // warp find the CTA's two range ends; everybody else picks them up after the barrier.
-    if (warp == 0) {
-        __syncwarp();
-        const int nz_rows = s_lay[0], U = rowbase[a.rows];
-        auto cost_to_unit = [&](int64_t x) {
-            int lo = 0, hi = a.rows;         // last rr in [0, rows] with cost_start(rr) <= x
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                const int nzb = (mid < a.rows) ? nzp[mid] : nz_rows;
-                if ((int64_t)rowbase[mid] + (int64_t)PIECE_COST * nzb <= x) lo = mid; else hi = mid - 1;
-            }
-            if (lo >= a.rows) return U;
-            const int units = rowbase[lo + 1] - rowbase[lo];
-            int64_t off = x - ((int64_t)rowbase[lo] + (int64_t)PIECE_COST * nzp[lo]) - (units > 0 ? PIECE_COST : 0);
-            off = off < 0 ? 0 : (off > units ? units : off);
-            return rowbase[lo] + (int)off;
-        };
-        if (lane < 2) {
-            // At least four cost units per CTA (fewer CTAs take part in a tiny problem): then no CTA's range is
-            // empty, and the CTAs that meet a row are exactly those between two ends that follow from the row's
-            // cost interval in closed form (the merge kernel finds its candidates that way).
-            const int64_t C = (int64_t)U + (int64_t)PIECE_COST * nz_rows;
-            const int P = (int)min((int64_t)gridDim.x, max((int64_t)1, C / 4));
-            const int c = blockIdx.x + lane;
-            s_lay[1 + lane] = (c >= P) ? U : cost_to_unit((c * C) / P);
-            if (lane == 0) s_lay[3] = P;
-        }
-    }
-    if (blockIdx.x == 0 && warp >= 1) {
-        // the first CTA publishes the rescued heads' admission bits and the number of blocks fetched per row
-        for (int rr = tid - 32; rr < a.rows; rr += NTHREADS - 32) {
+    if (tl2 && tid == 0) tl2[0] = (unsigned long long)clock64() - clk0;
+    __syncthreads();
+    // Publishing for the merge kernel and the caller is shared out over the CTAs (all of them hold the same layout):
+    // CTA c takes the rows c, c + gridDim.x, ...  Here the rescued heads' admission bits and the number of blocks
+    // fetched per row; the rows' spans of CTAs follow once the split is known.
+    if (warp >= 1) {
+        for (int rr = blockIdx.x + (tid - 32) * gridDim.x; rr < a.rows; rr += (NTHREADS - 32) * gridDim.x) {
             int extra = 0;
             for (int g = 0; g < a.G; ++g) {
                 const int j = resc_j[rr * 8 + g];
@@ -342,20 +311,102 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 if (w == 0 && !dup) ++extra;      // a block no head had admitted: one more block fetched
                 *mp = (uint8_t)(w | (1u << g));
             }
-            if (a.stats) a.stats[rr] = cnt32[rr] + extra;
+            if (a.stats) a.stats[rr] = rowcnt[rr] + extra;
         }
     }
+    // Equal shares of COST, not of units: a row that starts inside a CTA's range costs that CTA a flush of its
+    // partials and a query reload, worth about PIECE_COST tiles.  Row rr spans the cost interval
+    // [rowbase[rr] + PIECE_COST * nzp[rr], +PIECE_COST (if it has units) + its units).  The first warp scans the
+    // rows, two of its lanes find the CTA's two range ends; everybody else picks them up after the barrier.
+    if (warp == 0) {
+        int carry_u = 0, carry_z = 0;
+        int my_units = 0, my_base = 0, my_nzp = 0;          // of row `lane` (used when there are at most 32 rows)
+        for (int r0 = 0; r0 < a.rows; r0 += 32) {
+            const int rr = r0 + lane;
+            int units = 0;
+            if (rr < a.rows) {
+                const int info = rowinfo[rr];
+                units = rowcnt[rr] + (info & 0x7f) + (info >> 7);      // surviving blocks, rescued blocks, tail
+            }
+            const int nzf = units > 0 ? 1 : 0;
+            int iu = units, iz = nzf;
+#pragma unroll
+            for (int sft = 1; sft < 32; sft <<= 1) {
+                const int ou = __shfl_up_sync(0xffffffffu, iu, sft);
+                const int oz = __shfl_up_sync(0xffffffffu, iz, sft);
+                if (lane >= sft) { iu += ou; iz += oz; }
+            }
+            my_units = units; my_base = carry_u + iu - units; my_nzp = carry_z + iz - nzf;
+            if (rr < a.rows) { rowbase[rr] = my_base; nzp[rr] = (uint16_t)my_nzp; }
+            carry_u += __shfl_sync(0xffffffffu, iu, 31);
+            carry_z += __shfl_sync(0xffffffffu, iz, 31);
+        }
+        if (lane == 0) { rowbase[a.rows] = carry_u; s_lay[0] = carry_z; }
+        __syncwarp();
+        const int nz_rows = carry_z, U = carry_u;
+        // At least four cost units per CTA (fewer CTAs take part in a tiny problem): then no CTA's range is
+        // empty, and the CTAs that meet a row are exactly those between two ends that follow from the row's
+        // cost interval in closed form (the merge kernel finds its candidates that way).
+        const uint32_t C = (uint32_t)U + (uint32_t)PIECE_COST * (uint32_t)nz_rows;
+        const uint32_t P = min((uint32_t)gridDim.x, max(1u, C / 4u));
+        const uint32_t cq = C / P, cr = C - cq * P;
+        // cost position x -> unit: the last row rr in [0, rows] whose cost interval starts at or before x holds it
+        // (rows start in ascending order of cost).  Up to 32 rows: every lane compares its own row, a ballot counts;
+        // more rows: a binary search over the prefix arrays.
+        auto cost_to_unit = [&](uint32_t c) {
+            if (c >= P) return U;
+            const uint32_t x = c * cq + (c * cr) / P;        // floor(c C / P) without a 64-bit division: c cr < 2^16
+            int lo, lo_units, lo_base, lo_nzp;
+            if (a.rows <= 32) {
+                const bool le = lane < a.rows && (uint32_t)my_base + (uint32_t)PIECE_COST * (uint32_t)my_nzp <= x;
+                lo = __popc(__ballot_sync(0xffffffffu, le)) - 1;        // x >= 0 = the first row's start: lo >= 0
+                if (C <= x) return U;                                   // (cannot happen for c < P; the sentinel row)
+                lo_units = __shfl_sync(0xffffffffu, my_units, lo);
+                lo_base = __shfl_sync(0xffffffffu, my_base, lo);
+                lo_nzp = __shfl_sync(0xffffffffu, my_nzp, lo);
+            } else {
+                int l2 = 0, h2 = a.rows;
+                while (l2 < h2) {
+                    const int mid = (l2 + h2 + 1) >> 1;
+                    const uint32_t nzb = (mid < a.rows) ? nzp[mid] : (uint32_t)nz_rows;
+                    if ((uint32_t)rowbase[mid] + (uint32_t)PIECE_COST * nzb <= x) l2 = mid; else h2 = mid - 1;
+                }
+                if (l2 >= a.rows) return U;
+                lo = l2; lo_base = rowbase[lo]; lo_units = rowbase[lo + 1] - lo_base; lo_nzp = nzp[lo];
+            }
+            int off = (int)(x - ((uint32_t)lo_base + (uint32_t)PIECE_COST * (uint32_t)lo_nzp)) - (lo_units > 0 ? PIECE_COST : 0);
+            off = off < 0 ? 0 : (off > lo_units ? lo_units : off);
+            return lo_base + off;
+        };
+        const int unit0 = cost_to_unit(blockIdx.x), unit1 = cost_to_unit(blockIdx.x + 1);
+        // row holding the CTA's first unit: the last row that starts at or before it
+        int r_first;
+        if (a.rows <= 32) {
+            r_first = max(0, __popc(__ballot_sync(0xffffffffu, lane < a.rows && my_base <= unit0)) - 1);
+        } else {
+            int l2 = 0, h2 = a.rows - 1;
+            while (l2 < h2) {
+                const int mid = (l2 + h2 + 1) >> 1;
+                if (rowbase[mid] <= unit0) l2 = mid; else h2 = mid - 1;
+            }
+            r_first = l2;
+        }
+        if (lane == 0) { s_lay[1] = unit0; s_lay[2] = unit1; s_lay[3] = (int)P; s_lay[4] = r_first; }
+        if (tl2 && tid == 0) tl2[3] = (unsigned long long)clock64() - clk0;
+    }
     __syncthreads();
+    if (tl2 && tid == 0) tl2[4] = (unsigned long long)clock64() - clk0;
     const int U = rowbase[a.rows];
     const int u0 = s_lay[1], u1 = s_lay[2];
-    if (blockIdx.x == 0) {
+    const int row0 = s_lay[4];
+    if (warp == 1) {
         // For the merge kernel: the streaming CTAs that hold units of each row.  CTA c has the cost interval
         // [floor(c C / P), floor((c + 1) C / P)), row rr the interval [cs, ce) whose first PIECE_COST units are
         // padding, and (every CTA having at least four cost units) c holds units of the row exactly when its
         // interval starts before ce and ends after the padding.
         const int64_t C = (int64_t)U + (int64_t)PIECE_COST * s_lay[0];
         const int64_t P = s_lay[3];
-        for (int rr = tid; rr < a.rows; rr += NTHREADS) {
+        for (int rr = blockIdx.x + lane * gridDim.x; rr < a.rows; rr += 32 * gridDim.x) {
             const int units = rowbase[rr + 1] - rowbase[rr];
             int c_lo = 0, n_span = 0;
             if (units > 0) {
@@ -369,22 +420,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
     if (tl && tid == 0) tl[1] = globaltimer_ns();
     if (u0 >= u1) return;
-    // row holding unit u0: last r with rowbase[r] <= u0
-    int row0;
-    {
-        int lo = 0, hi = a.rows - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (rowbase[mid] <= u0) lo = mid; else hi = mid - 1;
-        }
-        row0 = lo;
-    }
-    // the rescue decisions of the first rows of this CTA's range outlive the layout scratch
-    if (tid < 8 * RESC_ROWS) {
-        const int rr = row0 + tid / 8;
-        resc_tab[tid] = (rr < a.rows && (tid & 7) < a.G) ? resc_j[rr * 8 + (tid & 7)] : -1;
-    }
-    __syncthreads();
 
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
@@ -415,32 +450,36 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         // units of entry e: survivors of a segment, rescue units of the row, or the row's tail
         bool first_window = counts_in_smem;     // the counts of the layout phase are still in the stage memory
         auto entry_count = [&](int e) {
-            if (e >= E) return 0;
+            if (first_window) return (e < E) ? (int)cnt8[e] : 0;
             int r, sg;
-            a.div_epr.divmod(e, r, sg);
-            if (sg < a.nseg) return first_window ? (int)cnt8[r * a.nseg + sg] : (int)__ldg(a.seg_count + r * a.nseg + sg);
+            a.div_epr.divmod(min(e, E - 1), r, sg);
+            const bool is_seg = sg < a.nseg;
+            int v = 0;
+            if (e < E && is_seg) v = __ldg(a.seg_count + r * a.nseg + sg);
             const int info = rowinfo[r];
-            return sg == a.nseg ? (info & 0x7f) : (info >> 7);
+            return (e >= E) ? 0 : (is_seg ? v : (sg == a.nseg ? (info & 0x7f) : (info >> 7)));
         };
-        // pwin[k] = units before entry e_base + k, k = 0 .. PW (PW a multiple of 32): a warp scan, 32 entries a round
+        // pwin[k] = units before entry e_base + k, k = 0 .. PW: lane l counts the PW / 32 consecutive entries from
+        // e_base + l PW / 32 on, one warp scan over the lanes' totals gives each lane its first prefix
         auto load_window = [&]() {
             __syncwarp();
-            int cw[PW / 32];
+            constexpr int EPL = PW / 32;
+            int cw[EPL];
 #pragma unroll
-            for (int m = 0; m < PW / 32; ++m) cw[m] = entry_count(e_base + 32 * m + lane);   // all loads in flight
-            int run = base_units;
+            for (int m = 0; m < EPL; ++m) cw[m] = entry_count(e_base + EPL * lane + m);   // all loads in flight
+            int tot = 0;
 #pragma unroll
-            for (int m = 0; m < PW / 32; ++m) {
-                int incl = cw[m];
+            for (int m = 0; m < EPL; ++m) tot += cw[m];
+            int incl = tot;
 #pragma unroll
-                for (int s = 1; s < 32; s <<= 1) {
-                    const int o = __shfl_up_sync(0xffffffffu, incl, s);
-                    if (lane >= s) incl += o;
-                }
-                pwin[32 * m + lane] = run + incl - cw[m];
-                run += __shfl_sync(0xffffffffu, incl, 31);
+            for (int sft = 1; sft < 32; sft <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, sft);
+                if (lane >= sft) incl += o;
             }
-            if (lane == 0) pwin[PW] = run;
+            int run = base_units + incl - tot;
+#pragma unroll
+            for (int m = 0; m < EPL; ++m) { pwin[EPL * lane + m] = run; run += cw[m]; }
+            if (lane == 31) pwin[PW] = run;
             __syncwarp();
         };
         auto search = [&](int uu) {          // largest k in [0, PW) with pwin[k] <= uu
@@ -535,13 +574,20 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
         };
 
+        // the rescue decisions of the first rows of this CTA's range outlive the layout scratch
+        for (int t = lane; t < 8 * RESC_ROWS; t += 32) {
+            const int rr = row0 + t / 8;
+            resc_tab[t] = (rr < a.rows && (t & 7) < a.G) ? resc_j[rr * 8 + (t & 7)] : -1;
+        }
+        if (tl2 && lane == 0) tl2[5] = (unsigned long long)clock64() - clk0;
         load_window();
         first_window = false;       // from the first copy on, the stage memory belongs to the tiles
-        if (tl && lane == 0) tl[6] = globaltimer_ns();
         int u = u0;
         int nb = batch_size(u);
+        if (tl2 && lane == 0) tl2[6] = (unsigned long long)clock64() - clk0;
         int c_row, c_ent, c_nrows, c_page;
         fetch(u, nb, c_row, c_ent, c_nrows, c_page);
+        if (tl2 && lane == 0) tl2[7] = (unsigned long long)clock64() - clk0 + (c_ent & 0);
         while (u < u1 && ok) {
             // the next batch is fetched once the first tiles of this batch are on their way, so that its loads
             // are in flight while the rest of this batch is issued
@@ -568,7 +614,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     const int stage = fill % NSTAGE;
                     const uint32_t round = fill / NSTAGE;
                     if (lane == 0) {
-                        if (tl && fill == 0) tl[2] = globaltimer_ns();
+                        if (tl2 && fill == 0) tl2[1] = (unsigned long long)clock64() - clk0;
                         if (!mbar_wait(&empty[stage], (round & 1) ^ 1)) {
                             ok = false;
                         } else {
@@ -905,20 +951,27 @@ struct MergeArgs {
 
 constexpr int MERGE_WARPS = 8;
 
-// One CTA per (row, query head).  The candidate parts are the (streaming CTA, consumer group) pairs of the
-// streaming CTAs that hold units of the row, which the streaming kernel lists per row; a part marked absent weighs
-// nothing.  Warp w takes a contiguous share of the candidates: a lane reads the statistics of one candidate while
-// the candidates' O rows are already on their way (eight in flight), the warp takes the largest m of its share,
-// weighs and adds the rows; the eight warps' (m, l, O) are combined in a fixed order:
-//   o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
-template <int D>
+// One CTA per (row, query head, slice of head_dim); DS slices of DW = D / DS coordinates each, chosen by the host so
+// that a small batch still fills the GPU (with one sequence and four KV heads there are only 16 (row, head) pairs,
+// each with up to 3 x 148 partials to fold).  The candidate parts are the (streaming CTA, consumer group) pairs of
+// the streaming CTAs that hold units of the row, which the streaming kernel lists per row; a part marked absent
+// weighs nothing.  Warp w takes a contiguous share of the candidates, 32 a round: lane k reads the statistics of
+// candidate k while O rows are already on their way (a row slice is DW / 4 lanes wide, so a warp instruction
+// fetches 128 / DW candidates' slices, eight instructions in flight), the warp takes the largest m of its share,
+// weighs and adds the rows; lanes that hold the same coordinates, then the eight warps, are combined in a fixed
+// order:  o = sum_k O_k e^{m_k - m*} / sum_k l_k e^{m_k - m*},  m* = max_k m_k.
+template <int D, int DS>
 __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs a) {
-    constexpr int VPL = D / 32;
-    __shared__ float s_acc[MERGE_WARPS][D];
+    constexpr int DW = D / DS;             // coordinates of this CTA's slice
+    constexpr int LPC = DW / 4;            // lanes per candidate row slice (a float4 each)
+    constexpr int CPW = 32 / LPC;          // candidates per warp instruction
+    static_assert(DW >= 4 && LPC <= 32 && LPC * CPW == 32, "slice must be 4 .. 128 coordinates");
+    __shared__ float s_acc[MERGE_WARPS][DW];
     __shared__ float s_l[MERGE_WARPS];
     __shared__ float s_m[MERGE_WARPS];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int r = blockIdx.x / a.G, gq = blockIdx.x % a.G;
+    const int pair = blockIdx.x / DS, dpart = blockIdx.x % DS;
+    const int r = pair / a.G, gq = pair % a.G;
     const int i = r / a.Hkv, hk = r % a.Hkv;
     unsigned long long* const tl = ETA_TL((a.timeline && blockIdx.x < TL_MERGE_N) ? a.timeline + (size_t)(TL_MERGE + blockIdx.x) * 8 : nullptr);
     if (tl && tid == 0) tl[0] = globaltimer_ns();
@@ -929,9 +982,8 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
     const int c_lo = span.x, n_cand = span.y * a.ngroups;
     if (tl && tid == 0) tl[2] = globaltimer_ns() + (n_cand & 0);
     auto slot_of = [&](int k) { return ((int64_t)(c_lo + k / a.ngroups) + r) * a.ngroups + k % a.ngroups; };
-    float acc[VPL];
-#pragma unroll
-    for (int k = 0; k < VPL; ++k) acc[k] = 0.f;
+    const int sub = lane / LPC, dl = lane % LPC;        // candidate within a warp instruction, float4 within the slice
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
     float m_w = -INFINITY, l_w = 0.f;        // this warp's running maximum and weighted l
     const int per = (n_cand + MERGE_WARPS - 1) / MERGE_WARPS;
     const int k_begin = warp * per, k_end = min(n_cand, k_begin + per);
@@ -943,23 +995,15 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
             const float2 ml = a.part_ml[slot_of(k) * a.G + gq];
             m_k = ml.x; l_k = ml.y;
         }
-        // the first eight O rows of the round do not wait for the statistics
-        float xv[8][VPL];
+        // the first O rows of the round do not wait for the statistics
+        float4 xv[8];
         auto load_rows = [&](int j0) {
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-#pragma unroll
-                for (int v = 0; v < VPL; ++v) xv[u][v] = 0.f;
-                if (j0 + u < nk) {
-                    const float* po = a.part_o + (slot_of(k0 + j0 + u) * a.G + gq) * D + lane * VPL;
-                    if (VPL == 4) {
-                        const float4 x = __ldg(reinterpret_cast<const float4*>(po));
-                        xv[u][0] = x.x; xv[u][1] = x.y; xv[u][VPL > 2 ? 2 : 0] = x.z; xv[u][VPL > 3 ? 3 : 0] = x.w;
-                    } else {
-                        const float2 x = __ldg(reinterpret_cast<const float2*>(po));
-                        xv[u][0] = x.x; xv[u][1] = x.y;
-                    }
-                }
+                const int j = j0 + u * CPW + sub;
+                xv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (j < nk)
+                    xv[u] = __ldg(reinterpret_cast<const float4*>(a.part_o + (slot_of(k0 + j) * a.G + gq) * D + dpart * DW) + dl);
             }
         };
         load_rows(0);
@@ -971,30 +1015,39 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
         const float rescale = (m_w == -INFINITY) ? 0.f : __expf(m_w - m_new);
         const float w = (m_k == -INFINITY) ? 0.f : __expf(m_k - m_new);
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) acc[v] *= rescale;
+        for (int v = 0; v < 4; ++v) acc[v] *= rescale;
         float lw = l_k * w;
 #pragma unroll
         for (int s = 16; s >= 1; s >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, s);
         l_w = l_w * rescale + lw;
         m_w = m_new;
-        for (int j0 = 0; j0 < nk; j0 += 8) {
+        for (int j0 = 0; j0 < nk; j0 += 8 * CPW) {
             if (j0 > 0) load_rows(j0);
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const float wk = __shfl_sync(0xffffffffu, w, min(j0 + u, 31));
-                if (j0 + u < nk && wk != 0.f) {       // an absent part's row is stale memory: never touch it
-#pragma unroll
-                    for (int v = 0; v < VPL; ++v) acc[v] = fmaf(xv[u][v], wk, acc[v]);
+                const int j = j0 + u * CPW + sub;
+                const float wk = __shfl_sync(0xffffffffu, w, min(j, 31));
+                if (j < nk && wk != 0.f) {       // an absent part's row is stale memory: never touch it
+                    acc[0] = fmaf(xv[u].x, wk, acc[0]); acc[1] = fmaf(xv[u].y, wk, acc[1]);
+                    acc[2] = fmaf(xv[u].z, wk, acc[2]); acc[3] = fmaf(xv[u].w, wk, acc[3]);
                 }
             }
         }
     }
-    if (tl && tid == 0) tl[3] = globaltimer_ns() + (__float_as_int(acc[0]) & 0);
+    // lanes that hold the same coordinates of different candidates
 #pragma unroll
-    for (int v = 0; v < VPL; ++v) s_acc[warp][lane * VPL + v] = acc[v];
+    for (int o = LPC; o < 32; o <<= 1) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[v] += __shfl_xor_sync(0xffffffffu, acc[v], o);
+    }
+    if (tl && tid == 0) tl[3] = globaltimer_ns() + (__float_as_int(acc[0]) & 0);
+    if (sub == 0) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) s_acc[warp][dl * 4 + v] = acc[v];
+    }
     if (lane == 0) { s_l[warp] = l_w; s_m[warp] = m_w; }
     __syncthreads();
-    if (tid < D) {
+    if (tid < DW) {
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < MERGE_WARPS; ++w) M = fmaxf(M, s_m[w]);
@@ -1007,7 +1060,7 @@ __global__ void __launch_bounds__(32 * MERGE_WARPS) merge_kernel(const MergeArgs
                 l = fmaf(s_l[w], sc, l);
             }
         }
-        a.out[((int64_t)i * a.Hq + hk * a.G + gq) * D + tid] = l > 0.f ? o / l : 0.f;
+        a.out[((int64_t)i * a.Hq + hk * a.G + gq) * D + dpart * DW + tid] = l > 0.f ? o / l : 0.f;
     }
     if (tl && tid == 0) tl[4] = globaltimer_ns();
 }
@@ -1164,9 +1217,14 @@ static int decode_impl(const eta_cache_desc* desc, const eta_page_table* pages, 
     MergeArgs ma;
     ma.row_span = da.row_span; ma.part_ml = da.part_ml; ma.part_o = da.part_o; ma.out = out;
     ma.Hq = desc->n_q_heads; ma.Hkv = desc->n_kv_heads; ma.G = G; ma.nseg = L.nseg; ma.rows = L.rows; ma.ngroups = DECODE_GROUPS; ma.timeline = debug_timeline();
-    const unsigned mgrid = (unsigned)(L.rows * G);
-    rc = (D == 128) ? launch_pdl("merge launch", merge_kernel<128>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma)
-                    : launch_pdl("merge launch", merge_kernel<64>, dim3(mgrid), dim3(32 * MERGE_WARPS), 0, s, ma);
+    // slices of head_dim per (row, head): enough CTAs to fill the GPU when the batch is small
+    const int pairs = L.rows * G;
+    const int DS = (pairs * 4 <= n_sm) ? 8 : (pairs * 2 <= n_sm ? 4 : (pairs <= n_sm / 2 ? 2 : 1));
+    const dim3 mgrid((unsigned)(pairs * DS)), mblock(32 * MERGE_WARPS);
+#define ETA_MERGE(DD, SS) launch_pdl("merge launch", merge_kernel<DD, SS>, mgrid, mblock, 0, s, ma)
+    if (D == 128) rc = DS == 8 ? ETA_MERGE(128, 8) : (DS == 4 ? ETA_MERGE(128, 4) : (DS == 2 ? ETA_MERGE(128, 2) : ETA_MERGE(128, 1)));
+    else rc = DS == 8 ? ETA_MERGE(64, 8) : (DS == 4 ? ETA_MERGE(64, 4) : (DS == 2 ? ETA_MERGE(64, 2) : ETA_MERGE(64, 1)));
+#undef ETA_MERGE
     profile_mark(5, s);
     return rc;
 }

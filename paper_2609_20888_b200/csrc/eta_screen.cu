@@ -1,17 +1,17 @@
 // Screening stage of eta_decode (Eq. dual_bound_eq; Algorithm 3, screening and
 // rescue lines).
 //
-// screen_kernel: one CTA per (row = sequence x KV head, segment of SEG block
-// records).  The segment's records (centroid and sigma, fp16) are one
-// contiguous run of HBM, staged into shared memory with four 1-D bulk copies so
-// that arithmetic on the first quarter overlaps the arrival of the rest.  Each
-// record is evaluated once for all G query heads of the group: d/8 lanes share
-// a record (16-byte shared-memory loads), each lane forms partial sums of
-// <q,mu> and sum q^2 sigma^2 for the G heads in fp32, and a transposed
-// butterfly leaves every lane with the two complete sums of one
-// (record, head) pair.  Admission bits are gathered with a ballot; survivors
-// are compacted per segment with ballot + popc prefix sums.  Nothing returns
-// to the host.
+// screen_kernel is persistent: two CTAs per SM, each owning a contiguous range
+// of items, an item being one segment of SEG consecutive block records of one
+// (sequence, KV head) row.  A segment's records (centroid and sigma, fp16) are
+// one contiguous run of HBM; they travel into a ring of NBUF shared-memory
+// buffers by 1-D bulk copies (with the group's queries behind them), ahead of
+// the item being worked on.  Each record is evaluated once for all G
+// query heads of the group.  Phase 1 (bounds; needs neither thresholds nor the
+// newest summary) runs item by item with one CTA barrier per item; phase 2
+// (admission, pinning, mask, ballot + popc compaction, rescue-window
+// statistics) takes a warp per item after the dependency wait.  Nothing
+// returns to the host.
 //
 // Top-1 rescue needs the whole rescue window of a head, which may span several
 // segments: this kernel only leaves per-segment window statistics (admitted
@@ -33,12 +33,17 @@ template <int D, int G>
 struct ScreenSmem {
     static constexpr int REC_BYTES = 4 * D;                    // fp16 mu[d] + fp16 sigma[d]
     static constexpr int BUF_BYTES = SEG * REC_BYTES + G * D * 2;   // a segment's records, then the group's queries
-    static constexpr int BAR_OFF = 2 * BUF_BYTES;
-    static constexpr int BOUND_OFF = BAR_OFF + 16;             // float [SCR_GROUP][SEG][G]: bounds of a group's items
+    // ring of record buffers: the copies of NBUF - 1 items are in flight while one item is worked on (a third buffer
+    // was measured and gained nothing: the kernel is bound by the latency of its arithmetic, not by bytes in flight)
+    static constexpr int FIXED_BYTES = 32 + SCR_GROUP * 4 * SEG * G + 2 * 4 * SEG + 4 * SCR_GROUP + 4 * MAX_ROWS + 128;
+    static constexpr int NBUF = 2;
+    static constexpr int BAR_OFF = NBUF * BUF_BYTES;
+    static constexpr int BOUND_OFF = BAR_OFF + 32;             // float [SCR_GROUP][SEG][G]: bounds of a group's items
     static constexpr int MN_OFF = BOUND_OFF + SCR_GROUP * 4 * SEG * G;   // float [2][SEG]: largest key norms
     static constexpr int OK_OFF = MN_OFF + 2 * 4 * SEG;        // int [SCR_GROUP]: 0 where the wait for an item's records ran out
     static constexpr int LEN_OFF = OK_OFF + 4 * SCR_GROUP;     // int32 clamped sequence lengths [MAX_ROWS]
     static constexpr int BYTES = LEN_OFF + 4 * MAX_ROWS + 128; // + slack for the 128-byte alignment of the base
+    static_assert(BYTES == BAR_OFF + FIXED_BYTES, "shared-memory layout and its size formula disagree");
 };
 
 // Persistent screening kernel.  Every CTA owns a contiguous range of (row, segment) items and works through it in
@@ -51,6 +56,7 @@ struct ScreenSmem {
 template <int D, int G>
 __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     using L = ScreenSmem<D, G>;
+    constexpr int NBUF = L::NBUF;
     constexpr int LPR = D / 8;            // lanes sharing one record
     constexpr int RPW = 32 / LPR;         // records per warp instruction
     constexpr int NI = LPR / G;           // iterations whose partial sums are reduced together
@@ -91,9 +97,11 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
     const int cc = lane % LPR, rg = lane / LPR;
     const int my_g = cc % G;
 
+    __shared__ int s_abort;               // set when a bounded wait ran out: no further copies are issued
     if (tid == 0) {
-        mbar_init(&bars[0], 1);
-        mbar_init(&bars[1], 1);
+        s_abort = 0;
+#pragma unroll
+        for (int k = 0; k < NBUF; ++k) mbar_init(&bars[k], 1);
         fence_barrier_init();
         // The copy of the CTA's first item starts before the sequence lengths are known: it takes every record of
         // the segment that the summary array holds (how many of them are blocks of the sequence only matters
@@ -132,7 +140,11 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         return g;
     };
     // one thread starts the copies of an item into buffer `buf`
-    auto issue = [&](const Geom& g, int buf) {
+    int last_issued = 0;                  // (thread 0) newest item, counted from it0, whose copies were started
+    auto issue = [&](const Geom& g, int k) {
+        if (s_abort) return;              // a wait ran out earlier: nothing is issued (or waited for) any more
+        const int buf = k % NBUF;
+        last_issued = k;
         if (g.n_rec > 0 && !dense) {
             unsigned char* dst = sm + buf * L::BUF_BYTES;
             const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
@@ -155,35 +167,52 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
 
     float qf[G][8], q2[USE_Q2 ? G : 1][8], qn[G], my_qn = 0.f;
     uint32_t qa[USE_MMA ? 8 : 1][2];       // A fragments of the centroid product: head lane / 4, one pair of registers per k-step
+    float qa_inv = 1.f;                    // undoes the power-of-two scaling of the A fragments (head lane / 4)
     int q_row = -1;
     bool waited = false;
     Geom gc = item_geom(it0);
-    if (tid == 0 && dense) mbar_arrive(&bars[0]);      // (otherwise the first item's copy is already on its way)
+    if (tid == 0) {
+        if (dense) mbar_arrive(&bars[0]);              // (otherwise the first item's copy is already on its way)
+        for (int k = 1; k < NBUF - 1 && it0 + k < it1; ++k) issue(item_geom(it0 + k), k);
+    }
     {
         const float mn0 = load_mn(gc);
         if (tid < SEG) smn_all[tid] = mn0;
     }
+    int first_failed = -1;                // (thread 0) item, counted from it0, whose wait ran out
     __syncthreads();
 
     for (int gs = it0; gs < it1; gs += SCR_GROUP) {
         const int ge = min(it1, gs + SCR_GROUP);
         // ------------------------------------------------------------ phase 1: bounds of the group's items
         for (int item = gs; item < ge; ++item) {
-            const int k = item - it0, buf = k & 1, slot = item - gs;
+            const int k = item - it0, buf = k % NBUF, npar = k & 1, slot = item - gs;
             float (*sbound)[G] = sbound_all + slot * SEG;
-            const float* smn = smn_all + buf * SEG;
+            const float* smn = smn_all + npar * SEG;
             const int r = gc.r, n_rec = gc.n_rec;
             Geom gn = gc;
             float mn_next = 0.f;
+            // the copies of item k + NBUF - 1 go into the buffer item k - 1 was read from (its reads ended at the
+            // barrier that closed item k - 1)
+            if (tid == 0 && item + NBUF - 1 < it1) issue(item_geom(item + NBUF - 1), k + NBUF - 1);
             if (item + 1 < it1) {
                 gn = item_geom(item + 1);
-                if (tid == 0) issue(gn, buf ^ 1);
                 mn_next = load_mn(gn);
             }
             if (tl && tid == 0 && item == it0 + 1) tl[6] = globaltimer_ns();
-            bool ok = mbar_wait(&bars[buf], (k >> 1) & 1);
+            // A wait that runs out: the item's blocks are all admitted (the safe direction), the call reports
+            // ETA_DEV_TIMEOUT, and the CTA stops issuing copies and waiting for them; copies already on their way
+            // are given time to land before the CTA leaves (end of the kernel).
+            bool ok = !ld_volatile(&s_abort) && mbar_wait(&bars[buf], (k / NBUF) & 1);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok && lane == 0) s_ok[slot] = 0;
+            if (!ok) {
+                if (lane == 0) s_ok[slot] = 0;
+                if (tid == 0 && first_failed < 0) {
+                    first_failed = k;
+                    s_abort = 1;
+                    if (a.status) atomicOr(a.status, ETA_DEV_TIMEOUT);
+                }
+            }
             if (tl && tid == 0 && item == it0 + 1) tl[7] = globaltimer_ns();
 
             if (n_rec > 0 && !dense && ok) {
@@ -217,7 +246,22 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                         // A[head][k]: lane (t = lane % 4, head = lane / 4 < G) holds, for k-steps 2j and 2j + 1, the
                         // eight dimensions 8 (4 j + t) .. + 7 of its head: the same dimensions the B fragments below
                         // take from one 16-byte load of a record (a dot product does not care about the order of k)
+                        //
+                        // fp16 holds neither the large nor the tiny end of bf16's range, so the head's query is first
+                        // scaled by a power of two that puts its norm in [2^13, 2^14) (every component then fits,
+                        // and one that falls below fp16's normal range is below 2^-27 of the norm), and the product
+                        // is scaled back: both scalings are exact.  A norm that overflowed fp32 gives a NaN bound
+                        // (the block is admitted); one that underflowed to zero gives a zero centroid term.
                         const int t4 = lane & 3, hd = lane >> 2;
+                        float qn_h = qn[0];
+#pragma unroll
+                        for (int g = 1; g < G; ++g) qn_h = (hd == g) ? qn[g] : qn_h;
+                        const int ef = (__float_as_int(qn_h) >> 23) & 0xff;
+                        const int sh = min(max(140 - ef, -120), 120);
+                        float q_sc = __int_as_float((127 + sh) << 23);           // 2^sh
+                        qa_inv = __int_as_float((127 - sh) << 23);               // 2^-sh
+                        if (ef == 255) q_sc = __int_as_float(0x7fc00000);
+                        if (ef == 0) { q_sc = 0.f; qa_inv = 0.f; }
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             uint4 v = make_uint4(0, 0, 0, 0);
@@ -226,7 +270,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                             uint32_t h[4];
 #pragma unroll
                             for (int kk = 0; kk < 4; ++kk) {
-                                const __half2 hh = __floats2half2_rn(bf16_lo(w[kk]), bf16_hi(w[kk]));
+                                const __half2 hh = __floats2half2_rn(bf16_lo(w[kk]) * q_sc, bf16_hi(w[kk]) * q_sc);
                                 h[kk] = *reinterpret_cast<const uint32_t*>(&hh);
                             }
                             qa[2 * j][0] = h[0]; qa[2 * j][1] = h[1];
@@ -297,8 +341,8 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                         }
                         // the centroid term of (record base + 2 it + rg, head g) sits in lane 4 g + it, element rg
                         const int it = cc / G;
-                        const float d0 = __shfl_sync(0xffffffffu, c[0], 4 * my_g + it);
-                        const float d1 = __shfl_sync(0xffffffffu, c[1], 4 * my_g + it);
+                        const float d0 = __shfl_sync(0xffffffffu, c[0] * qa_inv, 4 * my_g + it);
+                        const float d1 = __shfl_sync(0xffffffffu, c[1] * qa_inv, 4 * my_g + it);
                         const float dot = rg ? d1 : d0;
                         const int rec = base + it * RPW + rg;
                         if (rec < n_rec)
@@ -365,7 +409,7 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                 }
             }
             // the next item's key norms (fetched at the top of this iteration) go to its parity before the barrier
-            if (item + 1 < it1 && tid < SEG) smn_all[(buf ^ 1) * SEG + tid] = mn_next;
+            if (item + 1 < it1 && tid < SEG) smn_all[(npar ^ 1) * SEG + tid] = mn_next;
             // the one CTA-wide barrier of an item: its bounds are complete, and every read of the record buffer the
             // next copy goes into (and of the norms two items back) is over
             __syncthreads();
@@ -515,6 +559,11 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
             __syncthreads();          // the bounds of this group have been read: the next group may overwrite them
             if (tid < SCR_GROUP) s_ok[tid] = 1;
         }
+    }
+    if (tid == 0 && first_failed >= 0) {
+        // bounded wait for the copies that were in flight when a wait gave up, so that none lands in shared memory
+        // the next CTA on this SM already owns
+        for (int k = first_failed; k <= last_issued; ++k) mbar_wait(&bars[k % NBUF], (k / NBUF) & 1);
     }
     if (tl && tid == 0) tl[5] = globaltimer_ns();
     pdl_trigger();

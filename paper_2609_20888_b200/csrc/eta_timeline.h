@@ -10,6 +10,7 @@
 
 namespace eta {
 constexpr int TL_DECODE = 0;
+constexpr int TL_DECODE2 = 256;       // second row of stamps of the streaming kernel (set-up phases)
 constexpr int TL_SCREEN = 512, TL_SCREEN_N = 296;
 constexpr int TL_MERGE = 808, TL_MERGE_N = 128;
 constexpr int TL_PREDICT = 936, TL_PREDICT_N = 32;

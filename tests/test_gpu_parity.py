@@ -384,6 +384,43 @@ def test_threshold_equal_to_a_bound_admits_the_block_on_the_device(d, b, G):
         assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
 
 
+@pytest.mark.parametrize("d,G", [(128, 4), (64, 4)])
+def test_query_magnitudes_outside_the_fp16_range_screen_like_their_scaled_twins(d, G):
+    """Score_dual is positively homogeneous: scaling a head's query and its threshold by 2^k scales every bound by
+    2^k, exactly, in any binary floating-point format.  At head_dim 128 with four heads per group the centroid term
+    runs on the tensor cores with fp16 operands, which hold neither bf16 values above 65504 nor tiny ones: the
+    kernel normalises each head's query by a power of two first, so the selection must not depend on k.  Heads are
+    scaled by 2^17 (components beyond fp16's largest number), 2^-40 (far below its smallest), 1 and 2^9; the
+    masks must equal those of the unscaled call bit for bit, and agree with the oracle run on the scaled inputs
+    (near-tie band scaled with the head, as every bound is)."""
+    _eb()
+    b, B, Hkv = 64, 2, 2
+    rng, K, V, lens = _rand_cache_t(31 + d, B, Hkv, [64 * 70 + 9, 64 * 33], d, b)
+    q = torch.from_numpy(rng.standard_normal((B, Hkv * G, d))).to(torch.bfloat16)
+    c = orc.Cache(bits(K), bits(V), lens, b)
+    musig, mnorm = orc.block_summaries(c)
+    bound = orc.score_dual(bits(q), musig, mnorm, lens, b, 1.0)
+    tau = (np.nanquantile(bound, 0.8, axis=2) + 1e-4).astype(np.float32)
+    ks = np.array([17, -40, 0, 9] * (Hkv * G // 4))
+    scale = np.ldexp(1.0, ks)
+    q_s = (q.float() * torch.from_numpy(scale).float()[None, :, None]).to(torch.bfloat16)
+    assert torch.equal(q_s.float(), q.float() * torch.from_numpy(scale).float()[None, :, None])     # exact in bf16
+    assert float(q_s.float().abs().max()) > 65504.0
+    tau_s = (tau.astype(np.float64) * scale[None, :]).astype(np.float32)
+    _, sel0, _, status0 = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=tau)
+    out1, sel1, _, status1 = gpu_decode(q_s, K, V, lens, b, musig, mnorm, tau=tau_s)
+    assert status0 == 0 and status1 == 0 and np.isfinite(out1).all()
+    assert np.array_equal(sel0, sel1), "the selection depends on the magnitude of the query"
+    ref = orc.decode_step(bits(q_s), c, musig, mnorm, tau=tau_s)
+    diff = sel1 ^ ref["sel"]
+    for i, hk, j in zip(*np.nonzero(diff)):
+        for g in range(G):
+            if (diff[i, hk, j] >> g) & 1:
+                h = hk * G + g
+                assert abs(ref["bound"][i, h, j] - float(tau_s[i, h])) <= 1e-5 * scale[h], (i, h, j)
+    assert 0.05 < float((sel1 != 0).mean()) < 0.9
+
+
 def test_sphere_term_binds_and_large_logits_stay_finite():
     _eb()
     # a z-score above sqrt(d): the moment term exceeds the Cauchy-Schwarz ceiling, so the sphere term decides
