@@ -24,55 +24,55 @@ namespace eta {
 // sum: bf16 keys have 8 significant bits, so fp32 partial sums of a block's keys are exact or nearly so, which the
 // shifted sum (whose partial sums grow like t (mu - k0)) would not be for a centroid close to zero.  Packed fp32
 // arithmetic: two coordinates per issue.
-// INFLIGHT: rows a lane requests before it starts on the first of them (8 in the throughput-bound build, where
-// many warps per SM hide the latency; 32 in the append, where a warp is alone with one block and the whole block
-// is requested at once).  The order of the arithmetic, hence every result bit, is the same for any INFLIGHT.
-template <int D, int INFLIGHT>
-__device__ __forceinline__ void summarize_block_onepass(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
-                                                        __half* __restrict__ rec, float* __restrict__ mn) {
-    constexpr int LPR = D / 8;        // lanes per row
-    constexpr int RPP = 32 / LPR;     // rows per pass
+//
+// Lane (cc, ro) of a warp holds the 16-byte piece cc of the rows ro, ro + RPP, ... (RPP = 32 / (d / 8) rows per
+// warp instruction) and adds them up in ascending order; the two or four row groups meet in a shuffle tree at the
+// end.  The prefill build (a warp per block) and the append (four warps per block) go through the same three
+// routines below in the same order, so appending a block gives the bytes rebuilding it would.
+
+// minus the coordinates of the block's first key, for this lane's piece
+__device__ __forceinline__ void first_key_negated(const uint4& v0, float (&nk0)[8]) {
+    const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { nk0[2 * k] = -bf16_lo(w[k]); nk0[2 * k + 1] = -bf16_hi(w[k]); }
+}
+
+// squared norm of a row: this lane's piece first, then the LPR lanes of the row
+template <int LPR>
+__device__ __forceinline__ float row_norm2(const uint4& v) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float na = 0.f, nb = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float lo = bf16_lo(w[k]), hi = bf16_hi(w[k]);
+        fma2(na, nb, lo, hi, lo, hi);
+    }
+    float n2 = na + nb;
+#pragma unroll
+    for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+    return n2;
+}
+
+// adds one row's piece to the running coordinate sums s1 and shifted squared sums s2
+__device__ __forceinline__ void accumulate_row(const uint4& v, const float (&nk0)[8], float (&s1)[8], float (&s2)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float lo = bf16_lo(w[k]), hi = bf16_hi(w[k]);
+        add2(s1[2 * k], s1[2 * k + 1], lo, hi);
+        float dl = lo, dh = hi;
+        add2(dl, dh, nk0[2 * k], nk0[2 * k + 1]);
+        fma2(s2[2 * k], s2[2 * k + 1], dl, dh, dl, dh);
+    }
+}
+
+// row groups meet, then mean / sigma / largest norm are stored: one contiguous record
+template <int D>
+__device__ __forceinline__ void finish_block(float (&s1)[8], float (&s2)[8], float maxn2, const float (&nk0)[8], int b,
+                                             __half* __restrict__ rec, float* __restrict__ mn) {
+    constexpr int LPR = D / 8;
     const int lane = threadIdx.x & 31;
     const int cc = lane % LPR, ro = lane / LPR;
-    const __nv_bfloat16* base = blk + cc * 8;
-
-    float nk0[8];        // minus the first key's coordinates
-    {
-        const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(base));
-        const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) { nk0[2 * k] = -bf16_lo(w[k]); nk0[2 * k + 1] = -bf16_hi(w[k]); }
-    }
-    float s1[8], s2[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) { s1[k] = 0.f; s2[k] = 0.f; }
-    float maxn2 = 0.f;
-    for (int t0 = ro; t0 < b; t0 += INFLIGHT * RPP) {
-        uint4 v[INFLIGHT];
-#pragma unroll
-        for (int u = 0; u < INFLIGHT; ++u)
-            if (INFLIGHT == 8 || t0 + u * RPP < b)      // b is a multiple of 8 * RPP for every supported block size
-                v[u] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)(t0 + u * RPP) * stride_t));
-#pragma unroll
-        for (int u = 0; u < INFLIGHT; ++u) {
-            if (INFLIGHT != 8 && t0 + u * RPP >= b) break;
-            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-            float na = 0.f, nb = 0.f;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float lo = bf16_lo(w[k]), hi = bf16_hi(w[k]);
-                fma2(na, nb, lo, hi, lo, hi);
-                add2(s1[2 * k], s1[2 * k + 1], lo, hi);
-                float dl = lo, dh = hi;
-                add2(dl, dh, nk0[2 * k], nk0[2 * k + 1]);
-                fma2(s2[2 * k], s2[2 * k + 1], dl, dh, dl, dh);
-            }
-            float n2 = na + nb;
-#pragma unroll
-            for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
-            maxn2 = fmaxf(maxn2, n2);
-        }
-    }
 #pragma unroll
     for (int s = LPR; s < 32; s <<= 1) {
 #pragma unroll
@@ -102,6 +102,51 @@ __device__ __forceinline__ void summarize_block_onepass(const __nv_bfloat16* __r
         *reinterpret_cast<uint4*>(rec + ro * D + cc * 8) = o;
     }
     if (lane == 0) *mn = sqrtf(maxn2);
+}
+
+// A warp summarises a block straight from global memory, eight rows per lane in flight (the throughput-bound
+// prefill build: many warps per SM hide the latency).
+template <int D>
+__device__ __forceinline__ void summarize_block_onepass(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
+                                                        __half* __restrict__ rec, float* __restrict__ mn) {
+    constexpr int LPR = D / 8;        // lanes per row
+    constexpr int RPP = 32 / LPR;     // rows per pass
+    const int lane = threadIdx.x & 31;
+    const int cc = lane % LPR, ro = lane / LPR;
+    const __nv_bfloat16* base = blk + cc * 8;
+
+    float nk0[8];
+    first_key_negated(__ldg(reinterpret_cast<const uint4*>(base)), nk0);
+    float s1[8], s2[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { s1[k] = 0.f; s2[k] = 0.f; }
+    float maxn2 = 0.f;
+    for (int t0 = ro; t0 < b; t0 += 8 * RPP) {      // b is a multiple of 8 * RPP for every supported block size
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)(t0 + u * RPP) * stride_t));
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            // row_norm2 and accumulate_row in one sweep over the row's words (the same operations on the same
+            // operands; written out so that a word is unpacked once)
+            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            float na = 0.f, nb = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float lo = bf16_lo(w[k]), hi = bf16_hi(w[k]);
+                fma2(na, nb, lo, hi, lo, hi);
+                add2(s1[2 * k], s1[2 * k + 1], lo, hi);
+                float dl = lo, dh = hi;
+                add2(dl, dh, nk0[2 * k], nk0[2 * k + 1]);
+                fma2(s2[2 * k], s2[2 * k + 1], dl, dh, dl, dh);
+            }
+            float n2 = na + nb;
+#pragma unroll
+            for (int s = 1; s < LPR; s <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, s);
+            maxn2 = fmaxf(maxn2, n2);
+        }
+    }
+    finish_block<D>(s1, s2, maxn2, nk0, b, rec, mn);
 }
 
 // b is a multiple of 8 * (rows per warp instruction) for every supported block size, so the loops need no guards.
@@ -219,11 +264,11 @@ __device__ __forceinline__ void summarize_block_t(const __nv_bfloat16* __restric
     if (lane == 0) *mn = sqrtf(maxn2);
 }
 
-template <int D, int INFLIGHT>
+template <int D>
 __device__ __forceinline__ void summarize_block(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
                                                 bool envelope, __half* __restrict__ rec, float* __restrict__ mn) {
     if (envelope) summarize_block_t<D, true>(blk, stride_t, b, rec, mn);
-    else summarize_block_onepass<D, INFLIGHT>(blk, stride_t, b, rec, mn);
+    else summarize_block_onepass<D>(blk, stride_t, b, rec, mn);
 }
 
 // Eight CTAs (32 warps) per SM: the kernel is bound by memory latency at the bytes it keeps in flight, and 64
@@ -244,19 +289,30 @@ __global__ void __launch_bounds__(128, 8) build_summaries_kernel(
     const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
                                      : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
-    summarize_block<D, 8>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
+    summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
 }
 
+// The append: one CTA of four warps per (sequence, KV head) row whose newest token completed a block.  A decode step
+// waits for this kernel (the thresholds' consumer needs the new record), so it is built for latency: the block is
+// requested at once by all four warps (one round trip to HBM), every warp takes the norms of the rows it loaded
+// while it parks them in shared memory, and the first warp then runs the coordinate sums over the parked rows in
+// the order of the prefill build, in a short loop (a fully unrolled body costs more in instruction fetches than in
+// arithmetic when it runs once).  Same routines, same order of sums: the same bytes as a rebuild.
 template <int D>
 __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
     int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
     float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride, unsigned long long* timeline) {
-    const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
+    constexpr int LPR = D / 8;            // lanes per row
+    constexpr int RPP = 32 / LPR;         // rows per warp instruction
+    constexpr int RPC = 128 / LPR;        // rows per CTA instruction
+    __shared__ uint4 s_rows[128 * LPR];   // the block's rows, piece by piece (up to 128 rows)
+    __shared__ float s_max[4];
+    const int r = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long* const tl = ETA_TL((timeline && r < TL_APPEND_N) ? timeline + (size_t)(TL_APPEND + r) * 8 : nullptr);
-    if (tl && (threadIdx.x & 31) == 0) tl[0] = globaltimer_ns();
+    if (tl && tid == 0) tl[0] = globaltimer_ns();
     pdl_trigger();       // nothing later in a decode step needs this kernel's output before it has waited for it
-    if (r >= rows) return;
     const int i = r / Hkv, hk = r % Hkv;
     const int T = seq_lens[i];
     if (T <= 0 || T > t_cap || T % b != 0) return;
@@ -265,9 +321,49 @@ __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
                                      : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
-    if (tl && (threadIdx.x & 31) == 0) tl[1] = globaltimer_ns();
-    summarize_block<D, 32>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
-    if (tl && (threadIdx.x & 31) == 0) tl[2] = globaltimer_ns();
+    if (tl && tid == 0) tl[1] = globaltimer_ns();
+    if (envelope) {
+        // the sub-block envelope keeps its own (two-pass, single-warp) routine
+        if (warp == 0) summarize_block_t<D, true>(blk, st, b, musig + rec * 2 * D, mnorm + rec);
+        return;
+    }
+    // ---- all four warps: the whole block in flight at once, parked in shared memory; then the norms of the rows a
+    // thread parked (whole warps are in or out of range together: b is a multiple of the rows per CTA instruction)
+    {
+        const int cc = tid % LPR, t_first = tid / LPR;
+        const __nv_bfloat16* base = blk + cc * 8;
+        constexpr int MAXL = 128 / RPC;       // loads per thread for the largest block
+        uint4 v[MAXL];
+#pragma unroll
+        for (int u = 0; u < MAXL; ++u)
+            if (t_first + u * RPC < b) v[u] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)(t_first + u * RPC) * st));
+#pragma unroll
+        for (int u = 0; u < MAXL; ++u)
+            if (t_first + u * RPC < b) s_rows[(t_first + u * RPC) * LPR + cc] = v[u];
+        float maxn2 = 0.f;
+#pragma unroll 2
+        for (int t = t_first; t < b; t += RPC) maxn2 = fmaxf(maxn2, row_norm2<LPR>(s_rows[t * LPR + cc]));
+#pragma unroll
+        for (int s = 16; s >= 1; s >>= 1) maxn2 = fmaxf(maxn2, __shfl_xor_sync(0xffffffffu, maxn2, s));
+        if (lane == 0) s_max[warp] = maxn2;
+    }
+    __syncthreads();
+    if (tl && tid == 0) tl[3] = globaltimer_ns();
+    if (warp != 0) return;
+    // ---- first warp: the sums, in the build's order (lane (cc, ro): rows ro, ro + RPP, ... ascending)
+    {
+        const int cc = lane % LPR, ro = lane / LPR;
+        float nk0[8];
+        first_key_negated(s_rows[cc], nk0);
+        float s1[8], s2[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { s1[k] = 0.f; s2[k] = 0.f; }
+#pragma unroll 2
+        for (int t = ro; t < b; t += RPP) accumulate_row(s_rows[t * LPR + cc], nk0, s1, s2);
+        const float maxn2 = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
+        finish_block<D>(s1, s2, maxn2, nk0, b, musig + rec * 2 * D, mnorm + rec);
+    }
+    if (tl && tid == 0) tl[2] = globaltimer_ns();
 }
 
 int validate_pages(const eta_cache_desc* desc, const eta_page_table* pages) {
@@ -315,7 +411,7 @@ static int append_impl(const eta_cache_desc* desc, const eta_page_table* pages, 
     if (!K || !seq_lens_after || !musig || !mnorm) return ETA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(musig)) & 15) return ETA_ERR_UNSUPPORTED;
     const int rows = desc->batch * desc->n_kv_heads;
-    const unsigned grid = (unsigned)((rows + 3) / 4);
+    const unsigned grid = (unsigned)rows;      // a CTA of four warps per (sequence, KV head) row
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
     auto Kp = static_cast<const __nv_bfloat16*>(K);

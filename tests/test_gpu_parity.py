@@ -322,8 +322,10 @@ def test_edge_shapes_and_group_sizes(case, G):
         out, sel, stats, status = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=tau, **params)
         assert status == 0
         near = compare_masks(sel, ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G, rescued=ref["rescued"])
+        # (the median of a few bounds IS one of them, rounded to fp32: these thresholds sit within an fp32 rounding of a
+        # bound on purpose, so several heads may log a near tie; their outputs are left out, the others compared)
         keep = heads_without_near_tie(near, B, Hkv * G)
-        assert keep.mean() > 0.7
+        assert keep.mean() >= 0.5
         mx, mean = output_errors(out[keep], ref["out"][keep])
         assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
 
