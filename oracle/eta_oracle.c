@@ -103,6 +103,73 @@ uint16_t eta_oracle_double_to_fp16(double x) {
     return sign | (uint16_t)((biased << 10) | (q - 1024));
 }
 
+/* e4m3 (8-bit float: 1 sign, 4 exponent bits with bias 7, 3 fraction bits; no
+ * infinities, 0x7f / 0xff are NaN, largest finite value 448) -> double. */
+double eta_oracle_e4m3_to_double(uint8_t bits) {
+    int sign = (bits >> 7) & 1;
+    int expo = (bits >> 3) & 0xf;
+    int frac = bits & 0x7;
+    double v;
+    if (expo == 15 && frac == 7) v = NAN;
+    else if (expo == 0) v = ldexp((double)frac, -9);          /* subnormal or zero: units of 2^-9 */
+    else v = ldexp(1.0 + (double)frac / 8.0, expo - 7);
+    return sign ? -v : v;
+}
+
+/* The smallest e4m3 value that is >= x, for x >= 0 (rounding toward +infinity);
+ * x above the largest finite value (448) or NaN gives the NaN code 0x7f, which
+ * the screening rule reads as "admit".  The positive codes 0x00 .. 0x7e are in
+ * ascending order of value, so the answer is found by walking them. */
+uint8_t eta_oracle_double_to_e4m3_up(double x) {
+    if (!(x <= 448.0)) return 0x7f;
+    if (x <= 0.0) return 0;
+    for (int code = 0; code <= 0x7e; ++code)
+        if (eta_oracle_e4m3_to_double((uint8_t)code) >= x) return (uint8_t)code;
+    return 0x7f;
+}
+
+/*
+ * Packed block summaries (the paper's outlook: "FP8 metadata"; the compact
+ * layout of the fused-kernel appendix is what it shrinks).  Format "sigma8",
+ * chosen by this library: per block and KV head
+ *     mu      fp16 [d]   (as in the compact layout)
+ *     sigma^  e4m3 [d]   sigma rounded UP to the next e4m3 value
+ * (3 d bytes instead of 4 d), M stays fp32.  Score_dual is non-decreasing in
+ * every sigma_c, and every e4m3 value is an fp16 value, so with sigma^ >= sigma
+ * the packed bound is never below the bound from the fp16 record: packing adds
+ * no false negative, it only admits a few more blocks.  sigma beyond 448 becomes
+ * the NaN code (bound NaN, block admitted).
+ * sigma_raw: the unrounded doubles [B,Hkv,NBcap,d] of eta_oracle_block_summaries;
+ * musig: its fp16 records (mu is copied); musig8: bytes [B,Hkv,NBcap,3 d].
+ */
+void eta_oracle_pack_sigma8(const uint16_t* musig, const double* sigma_raw, int B, int Hkv, int d, int b, int NBcap,
+                            const int32_t* seq_lens, uint8_t* musig8)
+{
+    for (int i = 0; i < B; ++i) {
+        int NB = seq_lens[i] / b;
+        if (NB > NBcap) NB = NBcap;
+        for (int h = 0; h < Hkv; ++h)
+            for (int j = 0; j < NB; ++j) {
+                int64_t rec = ((int64_t)(i * Hkv + h) * NBcap + j);
+                uint8_t* out = musig8 + rec * 3 * d;
+                memcpy(out, musig + rec * 2 * d, 2 * (size_t)d);
+                for (int c = 0; c < d; ++c) out[2 * d + c] = eta_oracle_double_to_e4m3_up(sigma_raw[rec * d + c]);
+            }
+    }
+}
+
+/* The fp16 record layout with sigma^ in place of sigma (every e4m3 value is exactly
+ * an fp16 value; the NaN code becomes an fp16 NaN): what the screening rule
+ * evaluates for a packed index.  All records of the arrays are converted. */
+void eta_oracle_unpack_sigma8(const uint8_t* musig8, int64_t n_rec, int d, uint16_t* musig)
+{
+    for (int64_t rec = 0; rec < n_rec; ++rec) {
+        memcpy(musig + rec * 2 * d, musig8 + rec * 3 * d, 2 * (size_t)d);
+        for (int c = 0; c < d; ++c)
+            musig[rec * 2 * d + d + c] = eta_oracle_double_to_fp16(eta_oracle_e4m3_to_double(musig8[rec * 3 * d + 2 * d + c]));
+    }
+}
+
 /* ------------------------------------------------------------------------ */
 /* Section 3: the dual probabilistic-geometric block index                   */
 /* ------------------------------------------------------------------------ */

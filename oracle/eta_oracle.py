@@ -131,6 +131,38 @@ def block_summaries(cache: Cache, envelope: bool = False, raw: bool = False):
     return musig, mnorm
 
 
+def e4m3_to_double(bits: int) -> float:
+    f = lib().eta_oracle_e4m3_to_double
+    f.restype, f.argtypes = ctypes.c_double, [ctypes.c_uint8]
+    return f(int(bits))
+
+
+def double_to_e4m3_up(x: float) -> int:
+    f = lib().eta_oracle_double_to_e4m3_up
+    f.restype, f.argtypes = ctypes.c_uint8, [ctypes.c_double]
+    return int(f(float(x)))
+
+
+def block_summaries_sigma8(cache: Cache, envelope: bool = False):
+    """Packed index: -> musig8 uint8 [B,Hkv,NBcap,3d] (mu fp16, then sigma rounded up to e4m3), mnorm float32."""
+    musig, mnorm, _, sg_raw, _ = block_summaries(cache, envelope=envelope, raw=True)
+    B, Hkv, NBcap, d = cache.B, cache.Hkv, cache.NBcap, cache.d
+    musig8 = np.zeros((B, Hkv, NBcap, 3 * d), np.uint8)
+    lib().eta_oracle_pack_sigma8(_p(musig, _u16), _p(sg_raw, _f64), _I(B), _I(Hkv), _I(d), _I(cache.block_size), _I(NBcap),
+                                 _p(cache.seq_lens, _i32), _p(musig8, _u8))
+    return musig8, mnorm
+
+
+def unpack_sigma8(musig8: np.ndarray) -> np.ndarray:
+    """Packed records -> the fp16 record layout [.., 2, d] with the rounded-up sigma (exact: e4m3 is a subset of fp16)."""
+    *lead, d3 = musig8.shape
+    d = d3 // 3
+    n_rec = int(np.prod(lead))
+    musig = np.zeros((*lead, 2, d), np.uint16)
+    lib().eta_oracle_unpack_sigma8(_p(np.ascontiguousarray(musig8), _u8), _L(n_rec), _I(d), _p(musig, _u16))
+    return musig
+
+
 def predict_threshold(q: np.ndarray, W: np.ndarray, bias: np.ndarray) -> np.ndarray:
     """q uint16 [B,Hq,d], W float32 [Hq*d,Hq], bias float32 [Hq] -> tau float64 [B,Hq]."""
     B, Hq, d = q.shape

@@ -275,6 +275,117 @@ def test_cantelli_count_and_diagonal_case():
 
 
 # --------------------------------------------------------------------------
+# packed summaries (format "sigma8": mu fp16, sigma rounded up to e4m3)
+# --------------------------------------------------------------------------
+
+def _e4m3_value(code: int) -> float:
+    """The e4m3 value of a code, from the format's definition: (-1)^s 2^(e-7) (1 + m/8), subnormals m/8 2^-6."""
+    sgn = -1.0 if code & 0x80 else 1.0
+    e, m = (code >> 3) & 0xf, code & 7
+    if e == 15 and m == 7:
+        return float("nan")
+    return sgn * (m / 8.0 * 2.0 ** -6 if e == 0 else (1 + m / 8.0) * 2.0 ** (e - 7))
+
+
+def test_e4m3_decode_and_round_up_over_every_code():
+    vals = [_e4m3_value(c) for c in range(256)]
+    for c in range(256):
+        got = orc.e4m3_to_double(c)
+        assert (math.isnan(got) and math.isnan(vals[c])) or got == vals[c]
+    assert vals[0x7e] == 448.0 and vals[0x01] == 2.0 ** -9 and vals[0x08] == 2.0 ** -6
+    # every e4m3 value is an fp16 value (what lets the packed record be read as an fp16 record)
+    assert all(orc.fp16_to_double(orc.double_to_fp16(v)) == v for v in vals[:0x7f])
+    # rounding toward +infinity: a representable value maps to itself, anything just above it to the next code
+    for c in range(0x7f):
+        assert orc.double_to_e4m3_up(vals[c]) == c
+        assert orc.double_to_e4m3_up(np.nextafter(vals[c], np.inf)) == c + 1        # 0x7e + 1 = the NaN code
+    assert orc.double_to_e4m3_up(1e9) == 0x7f and orc.double_to_e4m3_up(float("nan")) == 0x7f
+    rng = np.random.default_rng(3)
+    xs = np.abs(rng.standard_normal(3000)) * 10.0 ** rng.integers(-4, 3, 3000)
+    up = np.array([vals[orc.double_to_e4m3_up(x)] for x in xs])
+    ok = xs <= 448
+    assert np.all(up[ok] >= xs[ok])
+    normal = ok & (xs >= 2.0 ** -6)
+    assert np.all(up[normal] <= xs[normal] * (1 + 1 / 8.0))        # at most one part in eight above
+    assert np.all(np.isnan(up[~ok]))
+
+
+def test_packed_record_layout_size_and_exact_expansion():
+    rng = np.random.default_rng(12)
+    d, b = 64, 64
+    c = random_cache(rng, 2, 2, 5 * b + 3, d, b, scale=0.7)
+    musig, mnorm, _, sg_raw, _ = orc.block_summaries(c, raw=True)
+    ms8, mn8 = orc.block_summaries_sigma8(c)
+    assert ms8.shape[-1] == 3 * d and np.array_equal(mn8, mnorm)          # M (the sphere term's input) is untouched
+    # 3 d + 4 bytes per block and KV head against 4 b d bytes of K and V: 1.2 % at b = 64 (1.6 % unpacked)
+    assert (3 * d + 4) / (4 * b * d) == pytest.approx(0.0120, abs=2e-4)
+    NB = 5
+    # mu bytes are the fp16 centroid, byte for byte
+    assert np.array_equal(ms8[:, :, :NB, :2 * d].copy().view(np.uint16), musig[:, :, :NB, 0])
+    # sigma^ is the smallest e4m3 value that is >= sigma (numpy restatement over the table of values)
+    table = np.array([_e4m3_value(k) for k in range(0x7f)])
+    want = np.searchsorted(table, sg_raw[:, :, :NB], side="left").astype(np.uint8)
+    assert np.array_equal(ms8[:, :, :NB, 2 * d:], want)
+    # expansion to the fp16 layout is exact and never below the fp16 sigma
+    exp = orc.unpack_sigma8(ms8)
+    assert np.array_equal(exp[:, :, :NB, 0], musig[:, :, :NB, 0])
+    assert np.array_equal(fp16_values(exp[:, :, :NB, 1]), table[want])
+    assert np.all(fp16_values(exp[:, :, :NB, 1]) >= fp16_values(musig[:, :, :NB, 1]))
+
+
+def test_packed_bound_never_falls_below_the_fp16_bound_and_keeps_the_sphere_term():
+    rng = np.random.default_rng(13)
+    for scale in (0.05, 1.0, 30.0):
+        c = random_cache(rng, 2, 2, 12 * 16, 16, 16, scale=scale)
+        q = bf16_bits_from_f64(rng.standard_normal((2, 4, 16)) * 2.0)
+        musig, mnorm = orc.block_summaries(c)
+        ms8, _ = orc.block_summaries_sigma8(c)
+        exp = orc.unpack_sigma8(ms8)
+        for z in (0.0, 1.0, 2.5):
+            b16, g16, s16 = orc.score_dual(q, musig, mnorm, c.seq_lens, 16, z, parts=True)
+            b8, g8, s8 = orc.score_dual(q, exp, mnorm, c.seq_lens, 16, z, parts=True)
+            assert np.all(b8 >= b16) and np.all(g8 >= g16)              # every (query head, block): no new false negative
+            assert np.array_equal(s8, s16)                              # the Cauchy-Schwarz ceiling is bit-identical
+            if z == 0.0:
+                assert np.array_equal(g8, g16)                          # without the variance term nothing changes
+            else:
+                # and it is not much looser: the variance term grows by at most one part in eight
+                var16 = (g16 - orc.score_dual(q, musig, mnorm, c.seq_lens, 16, 0.0, parts=True)[1])
+                assert np.all(g8 - g16 <= var16 / 8.0 + 1e-12)
+    # selection on packed summaries is a superset of the selection on fp16 summaries at the same thresholds
+    # (thresholds that admit about a third of the blocks of every head, so that no rescue interferes)
+    tau = np.nanquantile(b16, 0.7, axis=2).astype(np.float32)
+    sel16, r16 = orc.select(b16, c.seq_lens, 16, 2, tau=tau, rescue_window=1 << 30)
+    sel8, r8 = orc.select(b8, c.seq_lens, 16, 2, tau=tau, rescue_window=1 << 30)
+    assert np.all(r16 < 0) and np.all(r8 < 0)
+    assert np.all((sel16 & ~sel8) == 0) and sel8.sum() >= sel16.sum() > 0
+
+
+def test_packed_identical_keys_stay_tight_and_huge_sigma_admits():
+    d, b = 16, 8
+    k = np.linspace(-1, 1, d)
+    K = bf16_bits_from_f64(np.broadcast_to(k, (1, 1, b, d)).copy())
+    cc = orc.Cache(K, K.copy(), np.array([b], np.int32), b)
+    ms8, mn = orc.block_summaries_sigma8(cc)
+    assert not ms8[0, 0, 0, 2 * d:].any()                               # sigma = 0 stays 0
+    qq = bf16_bits_from_f64(np.random.default_rng(0).standard_normal((1, 1, d)))
+    bound, g, _ = orc.score_dual(qq, orc.unpack_sigma8(ms8), mn, cc.seq_lens, b, 3.0, parts=True)
+    logit = float(bf16_values(qq)[0, 0] @ bf16_values(K)[0, 0, 0]) / 4.0
+    assert g[0, 0, 0] == pytest.approx(logit, rel=1e-12, abs=1e-14)
+    # a coordinate whose spread exceeds e4m3's range: NaN code, NaN bound, block admitted whatever the threshold
+    Kbig = bf16_values(K).copy()
+    Kbig[0, 0, ::2, 3] = 3000.0
+    Kbig[0, 0, 1::2, 3] = -3000.0
+    cb = orc.Cache(bf16_bits_from_f64(Kbig), K.copy(), np.array([b], np.int32), b)
+    ms8b, mnb = orc.block_summaries_sigma8(cb)
+    assert ms8b[0, 0, 0, 2 * d + 3] == 0x7f
+    bb = orc.score_dual(qq, orc.unpack_sigma8(ms8b), mnb, cb.seq_lens, b, 1.0)
+    assert np.isnan(bb[0, 0, 0])
+    sel, _ = orc.select(bb, cb.seq_lens, b, 1, tau=np.full((1, 1), 1e30, np.float32))
+    assert sel[0, 0, 0] == 1
+
+
+# --------------------------------------------------------------------------
 # selection (Algorithm 3: threshold, rescue; lwb pinning)
 # --------------------------------------------------------------------------
 
