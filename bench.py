@@ -65,18 +65,51 @@ def hbm_peak():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons while the timed region runs: through NVML (read-only queries, a
+    sample every few milliseconds), or, where the NVML module is missing, by calling nvidia-smi (about ten a second)."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.index, self.samples, self._halt = index, [], threading.Event()
+        self.nvml = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            # CUDA_VISIBLE_DEVICES may renumber the devices: find the NVML handle of torch's device by its UUID
+            uuid = str(torch.cuda.get_device_properties(index).uuid)
+            handle = None
+            for k in range(pynvml.nvmlDeviceGetCount()):
+                h = pynvml.nvmlDeviceGetHandleByIndex(k)
+                u = pynvml.nvmlDeviceGetUUID(h)
+                u = u.decode() if isinstance(u, bytes) else u
+                if uuid in u or u.replace("GPU-", "") == uuid:
+                    handle = h
+            if handle is not None:
+                self.nvml, self.handle = pynvml, handle
+                self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nvml = None
+
+    def _sample_nvml(self):
+        n = self.nvml
+        mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+        r = int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)) if hasattr(n, "nvmlDeviceGetCurrentClocksEventReasons") \
+            else int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+        bits = [getattr(n, "nvmlClocksEventReasonHwSlowdown", 0x8), getattr(n, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                getattr(n, "nvmlClocksEventReasonSwThermalSlowdown", 0x20), getattr(n, "nvmlClocksEventReasonSwPowerCap", 0x4)]
+        return [mhz, self.sm_max] + ["Active" if (r & b) else "Not Active" for b in bits]
 
     def run(self):
         while not self._halt.is_set():
             try:
+                if self.nvml is not None:
+                    self.samples.append(self._sample_nvml())
+                    self._halt.wait(0.002)
+                    continue
                 out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
                                       "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
                 parts = [p.strip() for p in out.strip().split(",")]
@@ -84,7 +117,7 @@ class ClockSampler(threading.Thread):
                     self.samples.append(parts)
             except Exception:
                 pass
-            self._halt.wait(0.05)
+            self._halt.wait(0.005)
 
     def stop(self) -> dict:
         self._halt.set()
@@ -92,10 +125,9 @@ class ClockSampler(threading.Thread):
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
         mhz = sorted(float(s[0]) for s in self.samples)
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for k, n in enumerate(names) if any(s[2 + k].lower().startswith("active") for s in self.samples)]
+        reasons = [n for k, n in enumerate(self.NAMES) if any(str(s[2 + k]).lower().startswith("active") for s in self.samples)]
         return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": float(self.samples[0][1]), "reasons": reasons,
-                "samples": len(self.samples)}
+                "samples": len(self.samples), "source": "nvml" if self.nvml is not None else "nvidia-smi"}
 
 
 def algorithmic_bytes(sp, lens, union_blocks: float):
@@ -204,6 +236,10 @@ def run_ours(args):
     torch.cuda.synchronize()
     build_ms = ev0.elapsed_time(ev1)
     k_bytes = sum(int(t) // sp.block_size for t in lens) * sp.n_kv_heads * sp.block_size * sp.head_dim * 2
+    # the packed index (centroid fp16, sigma rounded up to e4m3: 3 d bytes per record instead of 4 d), for the sweep
+    musig8, mnorm8 = eb.alloc_summaries(st.desc, dev, packed=True)
+    eb.eta_build_block_summaries(st.desc, Kd, lens_d, musig8, mnorm8, flags=eb.ETA_BUILD_PACKED_SIGMA)
+    torch.cuda.synchronize()
 
     # offline calibration (prefill-side tool, timed on its own): 16 sequences of 1024 tokens at this head geometry
     cal = None
@@ -249,14 +285,18 @@ def run_ours(args):
 
     q_stage = torch.empty_like(q_host[0]).pin_memory()      # fixed page-locked buffer the end-to-end step reads its query from
 
-    def make_step(bias_np, flags=0, profiled=False, host_io=False, host_q=None, host_out=None):
+    def make_step(bias_np, flags=0, profiled=False, host_io=False, host_q=None, host_out=None, packed=False):
         """One decode step on the query in `static_q`.  With --graph (default) the launches are captured once
         into a CUDA graph and replayed, so the host costs one graph launch per step instead of several kernel
         launches through ctypes; the library calls are the same either way.  With host_io the step starts by
         fetching the query from the page-locked buffer `q_stage` (eta_stage_query) and the merge kernel writes the
         output straight into the page-locked `out_host`."""
         bias_d = torch.from_numpy(bias_np).to(dev)
+        if packed:
+            flags |= eb.ETA_FLAG_PACKED_SIGMA
         params = eb.DecodeParams(z=sp.z, beta=sp.beta, lwb=sp.lwb, rescue_window=sp.rescue_window, flags=flags)
+        ms_t, mn_t = (musig8, mnorm8) if packed else (st.musig, st.mnorm)
+        bflags = eb.ETA_BUILD_PACKED_SIGMA if packed else 0
 
         host_q = host_io if host_q is None else host_q
         host_out = host_io if host_out is None else host_out
@@ -266,14 +306,14 @@ def run_ours(args):
                 eb.eta_stage_query(q_stage, static_q)
             o = out_host if host_out else st.out
             if pages is not None:
-                eb.eta_append_summary_paged(pdesc, pages, Kp, lens_d, st.musig, st.mnorm)
+                eb.eta_append_summary_paged(pdesc, pages, Kp, lens_d, ms_t, mn_t, flags=bflags)
                 eb.eta_predict_threshold(static_q, Wd, bias_d, st.tau)
-                eb.eta_decode_paged(pdesc, pages, params, static_q, Kp, Vp, lens_d, st.musig, st.mnorm, st.tau, None,
+                eb.eta_decode_paged(pdesc, pages, params, static_q, Kp, Vp, lens_d, ms_t, mn_t, st.tau, None,
                                     o, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
                 return
-            eb.eta_append_summary(st.desc, Kd, lens_d, st.musig, st.mnorm)
+            eb.eta_append_summary(st.desc, Kd, lens_d, ms_t, mn_t, flags=bflags)
             eb.eta_predict_threshold(static_q, Wd, bias_d, st.tau)
-            eb.eta_decode(st.desc, params, static_q, Kd, Vd, lens_d, st.musig, st.mnorm, st.tau, None,
+            eb.eta_decode(st.desc, params, static_q, Kd, Vd, lens_d, ms_t, mn_t, st.tau, None,
                           o, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
 
         graph = None
@@ -338,9 +378,9 @@ def run_ours(args):
             tot += int(st.stats.sum().item())
         return tot / args.steps
 
-    def kernel_times(bias_np, flags=0):
+    def kernel_times(bias_np, flags=0, packed=False):
         """Device time from each launch to the next, averaged over the steps, from events captured in the graph."""
-        stp = make_step(bias_np, flags, profiled=True)
+        stp = make_step(bias_np, flags, profiled=True, packed=packed)
         acc = {}
         for k in range(args.steps):
             l2_flush(k)
@@ -418,6 +458,15 @@ def run_ours(args):
             sweep[f"{tgt:.2f}"] = {"ms_per_step": m, "union_sparsity": 1 - ub / nb_total,
                                    "gbs_on_algorithmic_bytes": abt["total"] / (m * 1e-3) / 1e9, "kernel_ms": ktt,
                                    "decode_kernel_gbs": abt["decode"] / (ktt["decode_kernel"] * 1e-3) / 1e9}
+        # the packed index at the same thresholds: a quarter less screening traffic, a few more blocks admitted
+        for tgt in targets:
+            stp = make_step(load_bias(sp.name, tgt), packed=True)
+            ms, _ = timed(stp)
+            ub = union_blocks_of(stp)
+            m = sum(ms) / len(ms)
+            ktt = kernel_times(load_bias(sp.name, tgt), packed=True)
+            sweep[f"{tgt:.2f}_packed_sigma"] = {"ms_per_step": m, "union_sparsity": 1 - ub / nb_total, "kernel_ms": ktt,
+                                                "summary_bytes_per_record": 3 * sp.head_dim + 4}
         stp = make_step(np.zeros(sp.n_q_heads, np.float32), flags=eb.ETA_FLAG_DENSE)
         ms, _ = timed(stp)
         m = sum(ms) / len(ms)
@@ -426,6 +475,7 @@ def run_ours(args):
         sweep["dense_baseline"] = {"ms_per_step": m, "gbs_on_algorithmic_bytes": (abt["decode"]) / (m * 1e-3) / 1e9,
                                    "speedup_of_main": m / ms_step, "kernel_ms": ktt,
                                    "decode_kernel_gbs": abt["decode"] / (ktt["decode_kernel"] * 1e-3) / 1e9}
+        sweep["sdpa_outside_baseline"] = sdpa_outside(sp, Kd, Vd, q_dev, lens, args, l2_flush, dev)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -460,12 +510,44 @@ def run_ours(args):
             "prefill_build": {"ms": build_ms, "gbs": k_bytes / (build_ms * 1e-3) / 1e9},
             "calibration": cal,
             "sweep": sweep,
+            "sweep_regime": "every figure of `sweep`, `kernel_ms`, `e2e` and `value` was taken with the L2 flush named in config.l2 (" + args.flush + "), CUDA-graph replay " + ("on" if args.graph else "off") + ", a fresh query every step",
             "cpu_baseline": cpu,
             "setup_s": {"generate": round(gen_s, 1)},
         }
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def sdpa_outside(sp, Kd, Vd, q_dev, lens, args, l2_flush, dev):
+    """An outside sanity number for the dense baseline (Section 2's dense attention): torch's
+    scaled_dot_product_attention on the same shapes, bf16, the G query heads of a group as the query length of their KV
+    head (one decode query per sequence).  Library code, timed for context beside `dense_baseline`; never a product
+    path, and only meaningful when all sequences have the same length."""
+    import torch.nn.functional as F
+    if len(set(int(t) for t in lens)) != 1:
+        return {"unavailable": "sequences of different lengths"}
+    T = int(lens[0])
+    B, Hkv, G, d = sp.batch, sp.n_kv_heads, sp.gqa, sp.head_dim
+    Kt, Vt = Kd[:, :, :T], Vd[:, :, :T]
+
+    def run(q):
+        return F.scaled_dot_product_attention(q.view(B, Hkv, G, d), Kt, Vt)
+
+    for s in range(args.warmup):
+        run(q_dev[s])
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for k in range(args.steps):
+        l2_flush(k)
+        evs[k][0].record()
+        run(q_dev[args.warmup + k])
+        evs[k][1].record()
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+    kv_bytes = 2 * B * Hkv * T * d * 2
+    return {"ms_per_step": ms, "gbs_on_kv_bytes": kv_bytes / (ms * 1e-3) / 1e9,
+            "what": "torch.nn.functional.scaled_dot_product_attention, bf16, q as [batch, kv_heads, G, d] (library code; context only)"}
 
 
 def cpu_baseline(sp, w, bias, budget_s: float, steps: int | None = None):

@@ -31,6 +31,13 @@
  *       out      fp32 [batch, n_q_heads, d]
  *       sel_mask uint8 [batch, n_kv_heads, nb_cap]: bit g set iff query head hk*G+g attends
  *                full block j.  Tokens past the last full block are always attended.
+ *   - Packed summaries (the paper's outlook names "FP8 metadata"; the format is this library's): with
+ *     ETA_BUILD_PACKED_SIGMA / ETA_FLAG_PACKED_SIGMA musig is bytes [batch, n_kv_heads, nb_cap, 3 d]: the centroid
+ *     as fp16[d], then sigma as e4m3[d] (8-bit float, 4 exponent and 3 fraction bits) rounded UP to the next e4m3
+ *     value; mnorm is unchanged.  Score_dual is non-decreasing in sigma, so the packed bound is never below the
+ *     bound of the 4 d-byte record: packing adds no false negative, it admits a few more blocks (the variance
+ *     term grows by at most one part in eight) and cuts the screening traffic by a quarter.  sigma below 2^-9 is
+ *     stored as 2^-9, sigma above 448 as the NaN code (the block is then always admitted).
  *   - Supported shapes: head_dim in {64, 128}; block_size in {32, 64, 128};
  *     G in {1, 2, 4, 8}.  Anything else returns ETA_ERR_UNSUPPORTED.
  */
@@ -59,12 +66,14 @@ typedef enum eta_status {
 
 /* flags of eta_params.flags */
 #define ETA_FLAG_DENSE           1u  /* baseline: admit every block and switch the gate off (softmax attention) */
+#define ETA_FLAG_PACKED_SIGMA     4u  /* musig holds packed records (see "Packed summaries" below) */
 #define ETA_FLAG_UNGATE_LAST     2u  /* Eq. mult_attn leaves the diagonal s = t ungated; at decode time the query's own
                                         token is the newest one: it keeps its raw logit (S~ = S), and when it closes a
                                         full block that block is admitted for every head.  Off: Algorithm 3 as
                                         printed, every token gated */
 /* flags of the summary builders */
 #define ETA_BUILD_SIGMA_ENVELOPE 1u  /* store the sub-block envelope (Eq. subblock_envelope_appx) instead of sigma */
+#define ETA_BUILD_PACKED_SIGMA   2u  /* write packed records (see "Packed summaries" below) */
 
 typedef struct eta_cache_desc {
     int32_t batch, n_q_heads, n_kv_heads, head_dim, block_size;
@@ -160,8 +169,9 @@ int eta_predict_threshold(int32_t batch, int32_t n_q_heads, int32_t head_dim, co
  * Eq. dual_bound_eq, evaluated for every (sequence, query head, full block):
  *   bound = s * min( <q, mu> + z * sqrt(sum_c q_c^2 sigma_c^2), ||q|| * M ).
  * bound fp32 [batch, n_q_heads, nb_cap]; entries of blocks that are not full are
- * left untouched.  Same arithmetic as the screening stage of eta_decode; meant
- * for diagnostics and for calibrating frozen constants, not for the hot loop.
+ * left untouched.  Same arithmetic as the screening stage of eta_decode (packed
+ * records with ETA_FLAG_PACKED_SIGMA in params->flags); meant for diagnostics
+ * and for calibrating frozen constants, not for the hot loop.
  */
 int eta_score_dual(const eta_cache_desc* desc, const eta_params* params, const void* q,
                    const int32_t* seq_lens, const void* musig, const float* mnorm,

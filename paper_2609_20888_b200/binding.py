@@ -17,7 +17,9 @@ LIB_PATH = os.path.join(_HERE, "libeta_b200.so")
 
 ETA_FLAG_DENSE = 1
 ETA_FLAG_UNGATE_LAST = 2
+ETA_FLAG_PACKED_SIGMA = 4
 ETA_BUILD_SIGMA_ENVELOPE = 1
+ETA_BUILD_PACKED_SIGMA = 2
 ETA_DEV_TIMEOUT, ETA_DEV_LEN_CLAMPED, ETA_DEV_EMPTY_ROW = 1, 2, 4
 
 EXPORTS = ("eta_workspace_bytes", "eta_build_block_summaries", "eta_append_summary", "eta_build_block_summaries_paged",
@@ -121,6 +123,13 @@ def _dev_or_pinned(t: torch.Tensor, dtype=None, name="tensor"):
     return _dev(t, dtype, name)
 
 
+def _dev_musig(t: torch.Tensor):
+    """Summary records: fp16 (compact layout) or uint8 (packed layout)."""
+    if t is not None and t.dtype not in (torch.float16, torch.uint8):
+        raise EtaError(f"musig must be float16 (compact records) or uint8 (packed records), got {t.dtype}")
+    return _dev(t, None, "musig")
+
+
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
@@ -175,7 +184,13 @@ def eta_workspace_bytes(desc: CacheDesc) -> int:
     return n.value
 
 
-def alloc_summaries(desc: CacheDesc, device):
+def alloc_summaries(desc: CacheDesc, device, packed: bool = False):
+    """musig, mnorm for the compact layout (fp16 [.., 2, d]) or, with `packed`, the packed one (bytes [.., 3 d]: the
+    centroid as fp16, then sigma rounded up to e4m3)."""
+    if packed:
+        musig = torch.zeros((desc.batch, desc.n_kv_heads, desc.nb_cap, 3 * desc.head_dim), dtype=torch.uint8, device=device)
+        mnorm = torch.zeros((desc.batch, desc.n_kv_heads, desc.nb_cap), dtype=torch.float32, device=device)
+        return musig, mnorm
     musig = torch.zeros((desc.batch, desc.n_kv_heads, desc.nb_cap, 2, desc.head_dim), dtype=torch.float16, device=device)
     mnorm = torch.zeros((desc.batch, desc.n_kv_heads, desc.nb_cap), dtype=torch.float32, device=device)
     return musig, mnorm
@@ -183,14 +198,14 @@ def alloc_summaries(desc: CacheDesc, device):
 
 def eta_build_block_summaries(desc, K, seq_lens, musig, mnorm, flags: int = 0) -> None:
     _check(load().eta_build_block_summaries(ctypes.byref(desc), _dev(K, torch.bfloat16, "K"),
-                                            _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                            _dev(seq_lens, torch.int32, "seq_lens"), _dev_musig(musig),
                                             _dev(mnorm, torch.float32, "mnorm"), flags, _stream()),
            "eta_build_block_summaries")
 
 
 def eta_append_summary(desc, K, seq_lens_after, musig, mnorm, flags: int = 0) -> None:
     _check(load().eta_append_summary(ctypes.byref(desc), _dev(K, torch.bfloat16, "K"),
-                                     _dev(seq_lens_after, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                     _dev(seq_lens_after, torch.int32, "seq_lens"), _dev_musig(musig),
                                      _dev(mnorm, torch.float32, "mnorm"), flags, _stream()),
            "eta_append_summary")
 
@@ -198,7 +213,7 @@ def eta_append_summary(desc, K, seq_lens_after, musig, mnorm, flags: int = 0) ->
 def eta_build_block_summaries_paged(desc, pages: PageTable, K_pool, seq_lens, musig, mnorm, flags: int = 0) -> None:
     _check(load().eta_build_block_summaries_paged(ctypes.byref(desc), ctypes.byref(pages), _dev(K_pool, torch.bfloat16, "K_pool"),
                                                   _dev(seq_lens, torch.int32, "seq_lens"),
-                                                  _dev(musig, torch.float16, "musig"), _dev(mnorm, torch.float32, "mnorm"),
+                                                  _dev_musig(musig), _dev(mnorm, torch.float32, "mnorm"),
                                                   flags, _stream()),
            "eta_build_block_summaries_paged")
 
@@ -206,7 +221,7 @@ def eta_build_block_summaries_paged(desc, pages: PageTable, K_pool, seq_lens, mu
 def eta_append_summary_paged(desc, pages: PageTable, K_pool, seq_lens_after, musig, mnorm, flags: int = 0) -> None:
     _check(load().eta_append_summary_paged(ctypes.byref(desc), ctypes.byref(pages), _dev(K_pool, torch.bfloat16, "K_pool"),
                                            _dev(seq_lens_after, torch.int32, "seq_lens"),
-                                           _dev(musig, torch.float16, "musig"), _dev(mnorm, torch.float32, "mnorm"),
+                                           _dev_musig(musig), _dev(mnorm, torch.float32, "mnorm"),
                                            flags, _stream()),
            "eta_append_summary_paged")
 
@@ -232,7 +247,7 @@ def eta_predict_threshold(q, W, bias, tau) -> None:
 def eta_score_dual(desc, params: DecodeParams, q, seq_lens, musig, mnorm, bound) -> None:
     p = params.c()
     _check(load().eta_score_dual(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
-                                 _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                 _dev(seq_lens, torch.int32, "seq_lens"), _dev_musig(musig),
                                  _dev(mnorm, torch.float32, "mnorm"), _dev(bound, torch.float32, "bound"), _stream()),
            "eta_score_dual")
 
@@ -264,7 +279,7 @@ def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau,
     p = params.c()
     _check(load().eta_decode(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
                              _dev(K, torch.bfloat16, "K"), _dev(V, torch.bfloat16, "V"),
-                             _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                             _dev(seq_lens, torch.int32, "seq_lens"), _dev_musig(musig),
                              _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
                              _dev(head_const, torch.float32, "head_const"), _dev_or_pinned(out, torch.float32, "out"),
                              _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),
@@ -278,7 +293,7 @@ def eta_decode_paged(desc, pages: PageTable, params: DecodeParams, q, K_pool, V_
     p = params.c()
     _check(load().eta_decode_paged(ctypes.byref(desc), ctypes.byref(pages), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
                                    _dev(K_pool, torch.bfloat16, "K_pool"), _dev(V_pool, torch.bfloat16, "V_pool"),
-                                   _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                   _dev(seq_lens, torch.int32, "seq_lens"), _dev_musig(musig),
                                    _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
                                    _dev(head_const, torch.float32, "head_const"), _dev_or_pinned(out, torch.float32, "out"),
                                    _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),
@@ -294,7 +309,7 @@ def eta_decode_static(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnor
     p = params.c()
     _check(load().eta_decode_static(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
                                     _dev(K, torch.bfloat16, "K"), _dev(V, torch.bfloat16, "V"),
-                                    _dev(seq_lens, torch.int32, "seq_lens"), _dev(musig, torch.float16, "musig"),
+                                    _dev(seq_lens, torch.int32, "seq_lens"), _dev_musig(musig),
                                     _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),
                                     _dev(head_const, torch.float32, "head_const"), _dev_or_pinned(out, torch.float32, "out"),
                                     _dev(sel_mask, torch.uint8, "sel_mask"), _dev(stats, torch.int32, "stats"),

@@ -275,6 +275,35 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 __device__ __forceinline__ int ld_volatile(const int* p) { return *reinterpret_cast<const volatile int*>(p); }
 __device__ __forceinline__ void st_volatile(int* p, int v) { *reinterpret_cast<volatile int*>(p) = v; }
 
+// e4m3 (8-bit float: 4 exponent bits, 3 fraction bits, largest finite value 448, 0x7f = NaN), the storage type of sigma in
+// packed summaries.  Two values at a time -> fp16 (exact: every e4m3 value is an fp16 value).
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_bytes) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"((unsigned short)two_bytes));
+    return r;
+}
+// eight e4m3 values (bytes 0 .. 7 of v) -> fp32, in order
+__device__ __forceinline__ void e4m3x8_to_f32(uint2 v, float (&out)[8]) {
+    const uint32_t h[4] = {e4m3x2_to_f16x2(v.x & 0xffffu), e4m3x2_to_f16x2(v.x >> 16), e4m3x2_to_f16x2(v.y & 0xffffu),
+                           e4m3x2_to_f16x2(v.y >> 16)};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h[k]));
+        out[2 * k] = f.x; out[2 * k + 1] = f.y;
+    }
+}
+// The smallest e4m3 value that is >= x, for x >= 0 (rounding toward +infinity: a packed sigma must not fall below
+// the sigma it stands for); x above 448 or NaN gives the NaN code, which the screening rule reads as "admit".
+__device__ __forceinline__ uint32_t f32_to_e4m3_up(float x) {
+    if (!(x <= 448.f)) return 0x7fu;
+    unsigned short pair;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair) : "f"(0.f), "f"(x));        // low byte: nearest to x
+    uint32_t code = pair & 0xffu;
+    const uint32_t back = e4m3x2_to_f16x2(code);
+    const float nearest = __half2float(*reinterpret_cast<const __half*>(&back));
+    return nearest < x ? code + 1u : code;      // positive codes ascend with their values
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
 

@@ -27,11 +27,43 @@ __device__ __forceinline__ float min_keep_nan(float g, float s) {
     return (g < s) ? g : ((s < g) ? s : ((g != g) ? g : s));
 }
 
+// sigma's piece cc (eight coordinates) of a record, as fp32: from the compact record (fp16) or the packed one (e4m3)
+template <int D, bool PACKED>
+__device__ __forceinline__ void sigma_piece_shared(uint32_t rec_addr, int cc, float (&sg)[8]) {
+    if constexpr (PACKED) {
+        uint2 v;
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(rec_addr + 2 * D + cc * 8));
+        e4m3x8_to_f32(v, sg);
+    } else {
+        const uint4 s4 = lds128(rec_addr + 2 * D + cc * 16);
+        const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
+            sg[2 * kk] = sf.x; sg[2 * kk + 1] = sf.y;
+        }
+    }
+}
+template <int D, bool PACKED>
+__device__ __forceinline__ void sigma_piece_global(const unsigned char* rec, int cc, float (&sg)[8]) {
+    if constexpr (PACKED) {
+        e4m3x8_to_f32(__ldcg(reinterpret_cast<const uint2*>(rec + 2 * D + cc * 8)), sg);
+    } else {
+        const uint4 s4 = __ldcg(reinterpret_cast<const uint4*>(rec + 2 * D + cc * 16));
+        const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
+            sg[2 * kk] = sf.x; sg[2 * kk + 1] = sf.y;
+        }
+    }
+}
+
 constexpr int SCR_GROUP = 8;       // items whose bounds are kept before their admission is decided: one per warp
 
-template <int D, int G>
+template <int D, int G, bool PACKED>
 struct ScreenSmem {
-    static constexpr int REC_BYTES = 4 * D;                    // fp16 mu[d] + fp16 sigma[d]
+    static constexpr int REC_BYTES = PACKED ? 3 * D : 4 * D;   // fp16 mu[d] + fp16 (packed: e4m3) sigma[d]
     static constexpr int BUF_BYTES = SEG * REC_BYTES + G * D * 2;   // a segment's records, then the group's queries
     // ring of record buffers: the copies of NBUF - 1 items are in flight while one item is worked on (a third buffer
     // was measured and gained nothing: the kernel is bound by the latency of its arithmetic, not by bytes in flight)
@@ -53,9 +85,9 @@ struct ScreenSmem {
 //   thresholds, so under programmatic dependent launch this phase runs while the predictor is still at work.
 //   Phase 2, a warp per item: admission against the thresholds, pinning, the user-visible mask, compaction of the
 //   union in ascending block order, and the rescue-window statistics.
-template <int D, int G>
+template <int D, int G, bool PACKED>
 __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
-    using L = ScreenSmem<D, G>;
+    using L = ScreenSmem<D, G, PACKED>;
     constexpr int NBUF = L::NBUF;
     constexpr int LPR = D / 8;            // lanes sharing one record
     constexpr int RPW = 32 / LPR;         // records per warp instruction
@@ -304,14 +336,10 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                             const int rec = base + it * RPW + rg;
                             float s2[8];
                             if (rec < n_rec) {
-                                const uint4 s4 = lds128(rec_base + rec * REC_BYTES + 2 * D + cc * 16);
-                                const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
+                                float sg[8];
+                                sigma_piece_shared<D, PACKED>(rec_base + rec * REC_BYTES, cc, sg);
 #pragma unroll
-                                for (int kk = 0; kk < 4; ++kk) {
-                                    const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
-                                    s2[2 * kk] = sf.x * sf.x;
-                                    s2[2 * kk + 1] = sf.y * sf.y;
-                                }
+                                for (int kk = 0; kk < 8; ++kk) s2[kk] = sg[kk] * sg[kk];
                             } else {
 #pragma unroll
                                 for (int kk = 0; kk < 8; ++kk) s2[kk] = 0.f;
@@ -357,16 +385,17 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                         float mu[8], s2[8];
                         if (rec < n_rec) {
                             const uint32_t addr = rec_base + rec * REC_BYTES + cc * 16;
-                            const uint4 m4 = lds128(addr), s4 = lds128(addr + 2 * D);
-                            const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw[4] = {s4.x, s4.y, s4.z, s4.w};
+                            const uint4 m4 = lds128(addr);
+                            const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w};
+                            float sg[8];
+                            sigma_piece_shared<D, PACKED>(rec_base + rec * REC_BYTES, cc, sg);
 #pragma unroll
                             for (int kk = 0; kk < 4; ++kk) {
                                 float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw[kk]));
-                                float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
                                 mu[2 * kk] = mf.x; mu[2 * kk + 1] = mf.y;
-                                s2[2 * kk] = USE_Q2 ? sf.x * sf.x : sf.x;
-                                s2[2 * kk + 1] = USE_Q2 ? sf.y * sf.y : sf.y;
                             }
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) s2[kk] = USE_Q2 ? sg[kk] * sg[kk] : sg[kk];
                         } else {
 #pragma unroll
                             for (int kk = 0; kk < 8; ++kk) { mu[kk] = 0.f; s2[kk] = 0.f; }
@@ -447,18 +476,17 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                                            ((int64_t)r * a.nb_cap + j0 + rec) * REC_BYTES;
                 const int cl = lane % LPR;
                 const uint4 m4 = __ldcg(reinterpret_cast<const uint4*>(src + cl * 16));
-                const uint4 s4 = __ldcg(reinterpret_cast<const uint4*>(src + 2 * D + cl * 16));
                 const float mn = __ldcg(a.mnorm + (int64_t)r * a.nb_cap + j0 + rec);
-                const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w}, sw[4] = {s4.x, s4.y, s4.z, s4.w};
-                float mu[8], s2[8];
+                const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w};
+                float mu[8], s2[8], sg[8];
+                sigma_piece_global<D, PACKED>(src, cl, sg);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
                     float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw[kk]));
-                    float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&sw[kk]));
                     mu[2 * kk] = mf.x; mu[2 * kk + 1] = mf.y;
-                    s2[2 * kk] = USE_Q2 ? sf.x * sf.x : sf.x;
-                    s2[2 * kk + 1] = USE_Q2 ? sf.y * sf.y : sf.y;
                 }
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) s2[kk] = USE_Q2 ? sg[kk] * sg[kk] : sg[kk];
 #pragma unroll
                 for (int gq = 0; gq < G; ++gq) {
                     const uint4 qv = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)g.i * a.Hq + g.hk * G + gq) * D) + cl);
@@ -571,9 +599,9 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
 
 // Diagnostic evaluation of Eq. dual_bound_eq: one warp per (sequence, query head, block).
 __global__ void __launch_bounds__(128) score_dual_kernel(
-    const __nv_bfloat16* __restrict__ q, const __half* __restrict__ musig, const float* __restrict__ mnorm,
+    const __nv_bfloat16* __restrict__ q, const unsigned char* __restrict__ musig, const float* __restrict__ mnorm,
     const int32_t* __restrict__ seq_lens, int B, int Hq, int Hkv, int d, int b, int t_cap, int nb_cap, float z,
-    float scale, float* __restrict__ bound) {
+    float scale, int packed, float* __restrict__ bound) {
     const int64_t wid = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (wid >= (int64_t)B * Hq * nb_cap) return;
@@ -589,8 +617,15 @@ __global__ void __launch_bounds__(128) score_dual_kernel(
     float dot = 0.f, var = 0.f, n2 = 0.f;
     for (int c = lane; c < d; c += 32) {
         const float x = __bfloat162float(qv[c]);
-        const float m = __half2float(musig[rec * 2 * d + c]);
-        const float s = __half2float(musig[rec * 2 * d + d + c]);
+        const unsigned char* rp = musig + rec * (packed ? 3 * d : 4 * d);
+        const float m = __half2float(reinterpret_cast<const __half*>(rp)[c]);
+        float s;
+        if (packed) {
+            const uint32_t h2 = e4m3x2_to_f16x2(rp[2 * d + c]);
+            s = __half2float(*reinterpret_cast<const __half*>(&h2));
+        } else {
+            s = __half2float(reinterpret_cast<const __half*>(rp)[d + c]);
+        }
         dot = fmaf(x, m, dot);
         var = fmaf(x * x, s * s, var);
         n2 = fmaf(x, x, n2);
@@ -605,9 +640,9 @@ __global__ void __launch_bounds__(128) score_dual_kernel(
 
 // ------------------------------------------------------------------ launchers (host)
 
-template <int D, int G>
+template <int D, int G, bool PACKED>
 static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream_t s) {
-    const size_t smem = ScreenSmem<D, G>::BYTES;
+    const size_t smem = ScreenSmem<D, G, PACKED>::BYTES;
     // The slowest CTA sets the kernel's end.  All CTAs are resident at once (n_ctas = two per SM), but under
     // programmatic dependent launch the kernel starts while its predecessors (summary append, threshold predictor)
     // still hold some SMs, where no CTA of this kernel fits until they exit: the CTAs dispatched last (the
@@ -643,11 +678,13 @@ static int launch_screen_t(const ScreenArgs& a, int rows, int n_ctas, cudaStream
         b2.n_early = grid;
         b2.per_early = n_items;
     }
-    return launch_pdl("screen launch", screen_kernel<D, G>, dim3(grid), dim3(256), smem, s, b2);
+    return launch_pdl("screen launch", screen_kernel<D, G, PACKED>, dim3(grid), dim3(256), smem, s, b2);
 }
 
 int launch_screen(const ScreenArgs& a, int rows, int D, int G, int n_ctas, cudaStream_t s) {
-#define ETA_CASE(DD, GG) if (D == DD && G == GG) return launch_screen_t<DD, GG>(a, rows, n_ctas, s);
+    const bool packed = (a.flags & ETA_FLAG_PACKED_SIGMA) != 0;
+#define ETA_CASE(DD, GG) if (D == DD && G == GG) return packed ? launch_screen_t<DD, GG, true>(a, rows, n_ctas, s) \
+                                                                : launch_screen_t<DD, GG, false>(a, rows, n_ctas, s);
     ETA_CASE(128, 1) ETA_CASE(128, 2) ETA_CASE(128, 4) ETA_CASE(128, 8)
     ETA_CASE(64, 1) ETA_CASE(64, 2) ETA_CASE(64, 4) ETA_CASE(64, 8)
 #undef ETA_CASE
@@ -665,8 +702,8 @@ extern "C" int eta_score_dual(const eta_cache_desc* desc, const eta_params* para
     const float scale = params->scale > 0.f ? params->scale : 1.0f / sqrtf((float)desc->head_dim);
     const int64_t warps = (int64_t)desc->batch * desc->n_q_heads * desc->nb_cap;
     eta::score_dual_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __nv_bfloat16*>(q), static_cast<const __half*>(musig), mnorm, seq_lens, desc->batch,
+        static_cast<const __nv_bfloat16*>(q), static_cast<const unsigned char*>(musig), mnorm, seq_lens, desc->batch,
         desc->n_q_heads, desc->n_kv_heads, desc->head_dim, desc->block_size, desc->t_cap, desc->nb_cap, params->z,
-        scale, bound);
+        scale, (params->flags & ETA_FLAG_PACKED_SIGMA) ? 1 : 0, bound);
     return eta::check_launch("eta_score_dual");
 }

@@ -66,10 +66,36 @@ __device__ __forceinline__ void accumulate_row(const uint4& v, const float (&nk0
     }
 }
 
+// Lane (cc, ro < 2) stores its piece of a record: row group 0 the centroid's piece cc (fp16), row group 1 sigma's.
+// Compact layout: mu fp16[d] | sigma fp16[d]; packed layout: mu fp16[d] | sigma e4m3[d], sigma rounded up.
+template <int D>
+__device__ __forceinline__ void store_record_piece(unsigned char* __restrict__ rec, bool packed, int ro, int cc,
+                                                   const float (&src)[8]) {
+    if (ro == 1 && packed) {
+        uint32_t c[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) c[k] = f32_to_e4m3_up(src[k]);
+        uint2 o;
+        o.x = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
+        o.y = c[4] | (c[5] << 8) | (c[6] << 16) | (c[7] << 24);
+        *reinterpret_cast<uint2*>(rec + 2 * D + cc * 8) = o;
+        return;
+    }
+    __half2 h[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) h[k] = __floats2half2_rn(src[2 * k], src[2 * k + 1]);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&h[0]);
+    o.y = *reinterpret_cast<uint32_t*>(&h[1]);
+    o.z = *reinterpret_cast<uint32_t*>(&h[2]);
+    o.w = *reinterpret_cast<uint32_t*>(&h[3]);
+    *reinterpret_cast<uint4*>(rec + ro * 2 * D + cc * 16) = o;
+}
+
 // row groups meet, then mean / sigma / largest norm are stored: one contiguous record
 template <int D>
 __device__ __forceinline__ void finish_block(float (&s1)[8], float (&s2)[8], float maxn2, const float (&nk0)[8], int b,
-                                             __half* __restrict__ rec, float* __restrict__ mn) {
+                                             unsigned char* __restrict__ rec, bool packed, float* __restrict__ mn) {
     constexpr int LPR = D / 8;
     const int lane = threadIdx.x & 31;
     const int cc = lane % LPR, ro = lane / LPR;
@@ -91,15 +117,7 @@ __device__ __forceinline__ void finish_block(float (&s1)[8], float (&s2)[8], flo
             const float m1 = mean + nk0[k];
             src[k] = (ro == 0) ? mean : sqrtf(fmaxf(fmaf(-m1, m1, s2[k] * inv_b), 0.f));
         }
-        __half2 h[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) h[k] = __floats2half2_rn(src[2 * k], src[2 * k + 1]);
-        uint4 o;
-        o.x = *reinterpret_cast<uint32_t*>(&h[0]);
-        o.y = *reinterpret_cast<uint32_t*>(&h[1]);
-        o.z = *reinterpret_cast<uint32_t*>(&h[2]);
-        o.w = *reinterpret_cast<uint32_t*>(&h[3]);
-        *reinterpret_cast<uint4*>(rec + ro * D + cc * 8) = o;
+        store_record_piece<D>(rec, packed, ro, cc, src);
     }
     if (lane == 0) *mn = sqrtf(maxn2);
 }
@@ -108,7 +126,7 @@ __device__ __forceinline__ void finish_block(float (&s1)[8], float (&s2)[8], flo
 // prefill build: many warps per SM hide the latency).
 template <int D>
 __device__ __forceinline__ void summarize_block_onepass(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
-                                                        __half* __restrict__ rec, float* __restrict__ mn) {
+                                                        unsigned char* __restrict__ rec, bool packed, float* __restrict__ mn) {
     constexpr int LPR = D / 8;        // lanes per row
     constexpr int RPP = 32 / LPR;     // rows per pass
     const int lane = threadIdx.x & 31;
@@ -146,13 +164,13 @@ __device__ __forceinline__ void summarize_block_onepass(const __nv_bfloat16* __r
             maxn2 = fmaxf(maxn2, n2);
         }
     }
-    finish_block<D>(s1, s2, maxn2, nk0, b, rec, mn);
+    finish_block<D>(s1, s2, maxn2, nk0, b, rec, packed, mn);
 }
 
 // b is a multiple of 8 * (rows per warp instruction) for every supported block size, so the loops need no guards.
 template <int D, bool envelope>
 __device__ __forceinline__ void summarize_block_t(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
-                                                  __half* __restrict__ rec, float* __restrict__ mn) {
+                                                  unsigned char* __restrict__ rec, bool packed, float* __restrict__ mn) {
     constexpr int LPR = D / 8;        // lanes per row
     constexpr int RPP = 32 / LPR;     // rows per pass
     const int lane = threadIdx.x & 31;
@@ -250,25 +268,20 @@ __device__ __forceinline__ void summarize_block_t(const __nv_bfloat16* __restric
 
     // row group 0 stores the centroid chunk, row group 1 the sigma chunk: one contiguous record
     if (ro < 2) {
-        const float* src = (ro == 0) ? mean : sg;
-        __half2 h[4];
+        float src[8];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) h[k] = __floats2half2_rn(src[2 * k], src[2 * k + 1]);
-        uint4 o;
-        o.x = *reinterpret_cast<uint32_t*>(&h[0]);
-        o.y = *reinterpret_cast<uint32_t*>(&h[1]);
-        o.z = *reinterpret_cast<uint32_t*>(&h[2]);
-        o.w = *reinterpret_cast<uint32_t*>(&h[3]);
-        *reinterpret_cast<uint4*>(rec + ro * D + cc * 8) = o;
+        for (int k = 0; k < 8; ++k) src[k] = (ro == 0) ? mean[k] : sg[k];
+        store_record_piece<D>(rec, packed, ro, cc, src);
     }
     if (lane == 0) *mn = sqrtf(maxn2);
 }
 
 template <int D>
 __device__ __forceinline__ void summarize_block(const __nv_bfloat16* __restrict__ blk, int64_t stride_t, int b,
-                                                bool envelope, __half* __restrict__ rec, float* __restrict__ mn) {
-    if (envelope) summarize_block_t<D, true>(blk, stride_t, b, rec, mn);
-    else summarize_block_onepass<D>(blk, stride_t, b, rec, mn);
+                                                bool envelope, unsigned char* __restrict__ rec, bool packed,
+                                                float* __restrict__ mn) {
+    if (envelope) summarize_block_t<D, true>(blk, stride_t, b, rec, packed, mn);
+    else summarize_block_onepass<D>(blk, stride_t, b, rec, packed, mn);
 }
 
 // Eight CTAs (32 warps) per SM: the kernel is bound by memory latency at the bytes it keeps in flight, and 64
@@ -276,7 +289,7 @@ __device__ __forceinline__ void summarize_block(const __nv_bfloat16* __restrict_
 template <int D>
 __global__ void __launch_bounds__(128, 8) build_summaries_kernel(
     const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
-    int nb_max, int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
+    int nb_max, int rows, const int32_t* __restrict__ seq_lens, int mode, unsigned char* __restrict__ musig,
     float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride) {
     const int64_t wid = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
     if (wid >= (int64_t)rows * nb_max) return;
@@ -289,7 +302,8 @@ __global__ void __launch_bounds__(128, 8) build_summaries_kernel(
     const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
                                      : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
-    summarize_block<D>(blk, st, b, envelope != 0, musig + rec * 2 * D, mnorm + rec);
+    const bool packed = (mode & 2) != 0;      // mode: bit 0 sub-block envelope, bit 1 packed records
+    summarize_block<D>(blk, st, b, (mode & 1) != 0, musig + rec * (packed ? 3 * D : 4 * D), packed, mnorm + rec);
 }
 
 // The append: one CTA of four warps per (sequence, KV head) row whose newest token completed a block.  A decode step
@@ -301,7 +315,7 @@ __global__ void __launch_bounds__(128, 8) build_summaries_kernel(
 template <int D>
 __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t sh, int64_t st, int Hkv, int b, int t_cap, int nb_cap,
-    int rows, const int32_t* __restrict__ seq_lens, int envelope, __half* __restrict__ musig,
+    int rows, const int32_t* __restrict__ seq_lens, int mode, unsigned char* __restrict__ musig,
     float* __restrict__ mnorm, const int32_t* __restrict__ table, int table_stride, unsigned long long* timeline) {
     constexpr int LPR = D / 8;            // lanes per row
     constexpr int RPP = 32 / LPR;         // rows per warp instruction
@@ -321,10 +335,12 @@ __global__ void __launch_bounds__(128) append_summary_kernel(
     const __nv_bfloat16* blk = table ? K + (int64_t)table[(int64_t)i * table_stride + j] * sb + hk * sh
                                      : K + i * sb + hk * sh + (int64_t)j * b * st;
     const int64_t rec = (int64_t)r * nb_cap + j;
+    const bool packed = (mode & 2) != 0;      // mode: bit 0 sub-block envelope, bit 1 packed records
+    unsigned char* const recp = musig + rec * (packed ? 3 * D : 4 * D);
     if (tl && tid == 0) tl[1] = globaltimer_ns();
-    if (envelope) {
+    if (mode & 1) {
         // the sub-block envelope keeps its own (two-pass, single-warp) routine
-        if (warp == 0) summarize_block_t<D, true>(blk, st, b, musig + rec * 2 * D, mnorm + rec);
+        if (warp == 0) summarize_block_t<D, true>(blk, st, b, recp, packed, mnorm + rec);
         return;
     }
     // ---- all four warps: the whole block in flight at once, parked in shared memory; then the norms of the rows a
@@ -361,7 +377,7 @@ __global__ void __launch_bounds__(128) append_summary_kernel(
 #pragma unroll 2
         for (int t = ro; t < b; t += RPP) accumulate_row(s_rows[t * LPR + cc], nk0, s1, s2);
         const float maxn2 = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
-        finish_block<D>(s1, s2, maxn2, nk0, b, musig + rec * 2 * D, mnorm + rec);
+        finish_block<D>(s1, s2, maxn2, nk0, b, recp, packed, mnorm + rec);
     }
     if (tl && tid == 0) tl[2] = globaltimer_ns();
 }
@@ -387,9 +403,9 @@ static int build_impl(const eta_cache_desc* desc, const eta_page_table* pages, c
     const int64_t warps = (int64_t)rows * nb_max;
     const unsigned grid = (unsigned)((warps + 3) / 4);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
+    const int env = ((flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0) | ((flags & ETA_BUILD_PACKED_SIGMA) ? 2 : 0);
     auto Kp = static_cast<const __nv_bfloat16*>(K);
-    auto mp = static_cast<__half*>(musig);
+    auto mp = static_cast<unsigned char*>(musig);
     if (desc->head_dim == 128)
         eta::build_summaries_kernel<128><<<grid, 128, 0, s>>>(Kp, desc->k_stride_b, desc->k_stride_h, desc->k_stride_t,
             desc->n_kv_heads, desc->block_size, desc->t_cap, desc->nb_cap, nb_max, rows, seq_lens, env, mp, mnorm,
@@ -413,9 +429,9 @@ static int append_impl(const eta_cache_desc* desc, const eta_page_table* pages, 
     const int rows = desc->batch * desc->n_kv_heads;
     const unsigned grid = (unsigned)rows;      // a CTA of four warps per (sequence, KV head) row
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int env = (flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0;
+    const int env = ((flags & ETA_BUILD_SIGMA_ENVELOPE) ? 1 : 0) | ((flags & ETA_BUILD_PACKED_SIGMA) ? 2 : 0);
     auto Kp = static_cast<const __nv_bfloat16*>(K);
-    auto mp = static_cast<__half*>(musig);
+    auto mp = static_cast<unsigned char*>(musig);
     rc = eta::configure_kernel(desc->head_dim == 128 ? reinterpret_cast<const void*>(eta::append_summary_kernel<128>)
                                                      : reinterpret_cast<const void*>(eta::append_summary_kernel<64>), 0);
     if (rc != ETA_OK) return rc;
