@@ -52,14 +52,16 @@ class EtaError(RuntimeError):
 _lib = None
 
 
-def load() -> ctypes.CDLL:
-    """Load the in-tree library; fails loudly when it has not been built."""
+def load(path: str | None = None) -> ctypes.CDLL:
+    """Load the in-tree library; fails loudly when it has not been built.  With a path: another build of the same
+    sources (a test variant), loaded beside the product library and not remembered."""
     global _lib
-    if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise EtaError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_20888_b200.build` "
+    if _lib is None or path is not None:
+        lib_path = path or LIB_PATH
+        if not os.path.exists(lib_path):
+            raise EtaError(f"{lib_path} is missing: build it with `python -m paper_2609_20888_b200.build` "
                            "(there is no fallback path)")
-        lib = ctypes.CDLL(LIB_PATH)
+        lib = ctypes.CDLL(lib_path)
         vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
         D, P = ctypes.POINTER(CacheDesc), ctypes.POINTER(Params)
         lib.eta_workspace_bytes.argtypes = [D, ctypes.POINTER(ctypes.c_size_t)]
@@ -94,6 +96,8 @@ def load() -> ctypes.CDLL:
             if name not in ("eta_strerror", "eta_last_cuda_error", "eta_decode_kernel_count",
                             "eta_profile_kernel_name", "eta_static_scratch_bytes"):
                 getattr(lib, name).restype = ctypes.c_int
+        if path is not None:
+            return lib
         _lib = lib
     return _lib
 
@@ -275,9 +279,9 @@ def eta_calibrate_head_const(Q, K, tau, head_const, dbar=None, beta=5.0, scale=0
 
 
 def eta_decode(desc, params: DecodeParams, q, K, V, seq_lens, musig, mnorm, tau, head_const, out, sel_mask,
-               workspace, stats=None, status=None) -> None:
+               workspace, stats=None, status=None, lib=None) -> None:
     p = params.c()
-    _check(load().eta_decode(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
+    _check((lib or load()).eta_decode(ctypes.byref(desc), ctypes.byref(p), _dev(q, torch.bfloat16, "q"),
                              _dev(K, torch.bfloat16, "K"), _dev(V, torch.bfloat16, "V"),
                              _dev(seq_lens, torch.int32, "seq_lens"), _dev_musig(musig),
                              _dev(mnorm, torch.float32, "mnorm"), _dev(tau, torch.float32, "tau"),

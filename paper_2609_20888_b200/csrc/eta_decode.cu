@@ -762,6 +762,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                     if (2 * t + 1 < a.G)
                         *reinterpret_cast<float2*>(sm_o + ((wq * a.G + 2 * t + 1) * D + dcol)) = make_float2(o[hf][mt][1], o[hf][mt][3]);
                 }
+#ifdef ETA_TEST_SKIP_FLUSH_ARRIVE
+            // test build only: one warp of the first CTA never arrives, so that the group's bounded wait runs out and
+            // the give-up path (status flag, orderly exit of the whole CTA) executes
+            if (!(blockIdx.x == 0 && group == 0 && wq == 1))
+#endif
             mbar_arrive(&flushbar[group]);
             if (!mbar_wait(&flushbar[group], flush_phase)) { ok = false; break; }
             flush_phase ^= 1;
