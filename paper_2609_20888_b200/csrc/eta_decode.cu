@@ -50,7 +50,10 @@ struct DecodeArgs {
 
 constexpr uint32_t UF_END = 1u;
 constexpr int WARPS_PER_GROUP = 4;     // the four warps of a group each take a quarter of a tile's tokens
-constexpr int PIECE_COST = 3;          // tiles a row boundary inside a CTA's range is worth (flush + query reload)
+// Tiles a row boundary inside a CTA's range is worth (flush of the partials, query reload, a pipeline that runs dry
+// while a group flushes).  Measured: 3 left the CTAs with several pieces last by 8 us on the mixed-length
+// configuration (128 rows); 6, 8, 10 and 14 are within noise of each other on every configuration.
+constexpr int PIECE_COST = 8;
 constexpr int RESC_ROWS = 8;           // rows (from the CTA's first) whose rescue decisions stay in shared memory
 constexpr int PW = 256;                // entries of the unit prefix the producer keeps in shared memory
 
@@ -344,11 +347,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         if (lane == 0) { rowbase[a.rows] = carry_u; s_lay[0] = carry_z; }
         __syncwarp();
         const int nz_rows = carry_z, U = carry_u;
-        // At least four cost units per CTA (fewer CTAs take part in a tiny problem): then no CTA's range is
-        // empty, and the CTAs that meet a row are exactly those between two ends that follow from the row's
-        // cost interval in closed form (the merge kernel finds its candidates that way).
+        // More cost units per CTA than a row's padding (fewer CTAs take part in a tiny problem): then no CTA's
+        // range lies inside a padding; the CTAs that meet a row are exactly those between two ends that follow
+        // from the row's cost interval in closed form (the merge kernel finds its candidates that way).
         const uint32_t C = (uint32_t)U + (uint32_t)PIECE_COST * (uint32_t)nz_rows;
-        const uint32_t P = min((uint32_t)gridDim.x, max(1u, C / 4u));
+        const uint32_t P = min((uint32_t)gridDim.x, max(1u, C / (uint32_t)(PIECE_COST + 1)));
         const uint32_t cq = C / P, cr = C - cq * P;
         // cost position x -> unit: the last row rr in [0, rows] whose cost interval starts at or before x holds it
         // (rows start in ascending order of cost).  Up to 32 rows: every lane compares its own row, a ballot counts;
@@ -402,8 +405,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     if (warp == 1) {
         // For the merge kernel: the streaming CTAs that hold units of each row.  CTA c has the cost interval
         // [floor(c C / P), floor((c + 1) C / P)), row rr the interval [cs, ce) whose first PIECE_COST units are
-        // padding, and (every CTA having at least four cost units) c holds units of the row exactly when its
-        // interval starts before ce and ends after the padding.
+        // padding, and c holds units of the row exactly when its interval starts before ce and ends after the
+        // padding.
         const int64_t C = (int64_t)U + (int64_t)PIECE_COST * s_lay[0];
         const int64_t P = s_lay[3];
         for (int rr = blockIdx.x + lane * gridDim.x; rr < a.rows; rr += 32 * gridDim.x) {
