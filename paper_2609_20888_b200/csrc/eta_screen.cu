@@ -67,14 +67,15 @@ struct ScreenSmem {
     static constexpr int BUF_BYTES = SEG * REC_BYTES + G * D * 2;   // a segment's records, then the group's queries
     // ring of record buffers: the copies of NBUF - 1 items are in flight while one item is worked on (a third buffer
     // was measured and gained nothing: the kernel is bound by the latency of its arithmetic, not by bytes in flight)
-    static constexpr int FIXED_BYTES = 32 + SCR_GROUP * 4 * SEG * G + 2 * 4 * SEG + 4 * SCR_GROUP + 4 * MAX_ROWS + 128;
+    static constexpr int FIXED_BYTES = 32 + SCR_GROUP * 4 * SEG * G + 2 * 4 * SEG + 4 * SCR_GROUP + 4 * MAX_ROWS + 8 * G * D * 2 + 128;
     static constexpr int NBUF = 2;
     static constexpr int BAR_OFF = NBUF * BUF_BYTES;
     static constexpr int BOUND_OFF = BAR_OFF + 32;             // float [SCR_GROUP][SEG][G]: bounds of a group's items
     static constexpr int MN_OFF = BOUND_OFF + SCR_GROUP * 4 * SEG * G;   // float [2][SEG]: largest key norms
     static constexpr int OK_OFF = MN_OFF + 2 * 4 * SEG;        // int [SCR_GROUP]: 0 where the wait for an item's records ran out
     static constexpr int LEN_OFF = OK_OFF + 4 * SCR_GROUP;     // int32 clamped sequence lengths [MAX_ROWS]
-    static constexpr int BYTES = LEN_OFF + 4 * MAX_ROWS + 128; // + slack for the 128-byte alignment of the base
+    static constexpr int QW_OFF = LEN_OFF + 4 * MAX_ROWS;      // bf16 [8 warps][G][D]: a warp's queries for phase 2's recomputation
+    static constexpr int BYTES = QW_OFF + 8 * G * D * 2 + 128; // + slack for the 128-byte alignment of the base
     static_assert(BYTES == BAR_OFF + FIXED_BYTES, "shared-memory layout and its size formula disagree");
 };
 
@@ -447,34 +448,42 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
         }
 
         // ------------------------------------------------------------ phase 2: a warp per item of the group
+        // What does not depend on the predecessor kernels is done ahead of the wait: the item's geometry and, for the
+        // one record per row that may have been copied stale, the group's queries (a caller input) into shared memory.
+        const bool p2 = gs + warp < ge;
+        const int slot = warp;
+        const Geom g = item_geom(min(gs + slot, n_items - 1));
+        const int r = g.r, seg = g.seg, NB = g.NB, j0 = g.j0, n_rec = g.n_rec;
+        const bool recompute = p2 && !dense && n_rec > 0 && (g.T & (a.b - 1)) == 0 && j0 + n_rec == NB;
+        uint4* qw = reinterpret_cast<uint4*>(sm + L::QW_OFF) + warp * (G * D / 8);
+        if (recompute) {
+            const uint4* qsrc = reinterpret_cast<const uint4*>(a.q + ((int64_t)g.i * a.Hq + g.hk * G) * D);
+            for (int k = lane; k < G * D / 8; k += 32) qw[k] = __ldg(qsrc + k);
+            __syncwarp();
+        }
         if (tl && tid == 0 && !waited) tl[2] = globaltimer_ns();
         if (!waited) { pdl_wait(); waited = true; }       // the thresholds (and the newest summaries) are final now
         if (tl && tid == 0 && gs == it0) tl[3] = globaltimer_ns();
-        if (gs + warp < ge) {
-            const int slot = warp;
-            const Geom g = item_geom(gs + slot);
+        if (p2) {
             const float (*sbound)[G] = sbound_all + slot * SEG;
-            const int r = g.r, seg = g.seg, NB = g.NB, j0 = g.j0, n_rec = g.n_rec;
             const bool ok = s_ok[slot] != 0;
             // an ungated newest token must be attended: when it closes a full block, that block counts as pinned
             const int lwb_item = ((a.flags & ETA_FLAG_UNGATE_LAST) && g.T > 0 && (g.T & (a.b - 1)) == 0 && a.lwb < 1) ? 1 : a.lwb;
-            // lane gq < G fetches the effective threshold of head gq of the item's group
+            // All loads that had to wait are issued together: lane gq < G fetches the effective threshold of head gq of
+            // the item's group, and, where the newest record has to be bounded again, every lane its pieces of it.
+            // (That record was possibly copied before the append kernel wrote it: its bound is computed again here,
+            // from global memory past the L1, in fp32 throughout; a difference of a rounding from the tensor-core value
+            // is far inside the near-tie band.)
             float te_l = -INFINITY;
             if (!dense && lane < G) {
                 const int h = g.hk * G + lane;
                 te_l = (a.tau ? __ldcg(a.tau + (int64_t)g.i * a.Hq + h) : __ldg(a.head_const + h)) - a.a;
             }
-            float te_g[G];
-#pragma unroll
-            for (int gq = 0; gq < G; ++gq) te_g[gq] = __shfl_sync(0xffffffffu, te_l, gq);
-            // The record of a block that filled up with the newest token was possibly copied before the append kernel
-            // wrote it: its bound is computed again here, from global memory past the L1, with the fp32 arithmetic
-            // (and the order of the sums) of phase 1's path without tensor cores.
-            if (!dense && ok && n_rec > 0 && (g.T & (a.b - 1)) == 0 && j0 + n_rec == NB) {
+            const int cl = lane % LPR;
+            if (recompute && ok) {
                 const int rec = n_rec - 1;
                 const unsigned char* src = reinterpret_cast<const unsigned char*>(a.musig) +
                                            ((int64_t)r * a.nb_cap + j0 + rec) * REC_BYTES;
-                const int cl = lane % LPR;
                 const uint4 m4 = __ldcg(reinterpret_cast<const uint4*>(src + cl * 16));
                 const float mn = __ldcg(a.mnorm + (int64_t)r * a.nb_cap + j0 + rec);
                 const uint32_t mw[4] = {m4.x, m4.y, m4.z, m4.w};
@@ -486,28 +495,22 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                     mu[2 * kk] = mf.x; mu[2 * kk + 1] = mf.y;
                 }
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) s2[kk] = USE_Q2 ? sg[kk] * sg[kk] : sg[kk];
-#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) s2[kk] = sg[kk] * sg[kk];
+#pragma unroll 1
                 for (int gq = 0; gq < G; ++gq) {
-                    const uint4 qv = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)g.i * a.Hq + g.hk * G + gq) * D) + cl);
-                    const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
+                    const uint4 qv = qw[gq * LPR + cl];
+                    const uint32_t qq[4] = {qv.x, qv.y, qv.z, qv.w};
                     float dot = 0.f, var = 0.f, n2 = 0.f;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
-                        const float x = (kk & 1) ? bf16_hi(qw[kk >> 1]) : bf16_lo(qw[kk >> 1]);
+                        const float x = (kk & 1) ? bf16_hi(qq[kk >> 1]) : bf16_lo(qq[kk >> 1]);
                         n2 = fmaf(x, x, n2);
                         dot = fmaf(x, mu[kk], dot);
-                        if (USE_Q2) {
-                            var = fmaf(x * x, s2[kk], var);
-                        } else {
-                            const float t = x * s2[kk];
-                            var = fmaf(t, t, var);
-                        }
+                        var = fmaf(x * x, s2[kk], var);
                     }
 #pragma unroll
-                    for (int sh = 1; sh < LPR; sh <<= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, sh);
-#pragma unroll
-                    for (int sh = LPR / 2; sh >= 1; sh >>= 1) {
+                    for (int sh = 1; sh < LPR; sh <<= 1) {
+                        n2 += __shfl_xor_sync(0xffffffffu, n2, sh);
                         dot += __shfl_xor_sync(0xffffffffu, dot, sh);
                         var += __shfl_xor_sync(0xffffffffu, var, sh);
                     }
@@ -516,6 +519,9 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                 }
                 __syncwarp();
             }
+            float te_g[G];
+#pragma unroll
+            for (int gq = 0; gq < G; ++gq) te_g[gq] = __shfl_sync(0xffffffffu, te_l, gq);
             if (seg == 0) {
                 if (lane < G) a.tau_eff[(int64_t)g.i * a.Hq + g.hk * G + lane] = te_l;
                 if (lane == 0 && a.status) {
@@ -551,33 +557,43 @@ __global__ void __launch_bounds__(256, 2) screen_kernel(const ScreenArgs a) {
                 }
                 if (lane == 0) a.seg_count[r * a.nseg + seg] = carry;
             }
-            // rescue statistics of the part of the rescue window inside this segment, per query head
+            // rescue statistics of the part of the rescue window inside this segment, per query head: how many of its
+            // blocks the head admits, the largest bound and the first block that attains it.  Bounds are compared as
+            // order-preserving integers (one hardware max-reduction and one ballot per head instead of a shuffle tree).
             const int Wr = min(a.rescue_window, NB);
             if (j0 < Wr && n_rec > 0) {
                 const int nwin = min(n_rec, Wr - j0);
-#pragma unroll
+#pragma unroll 1
                 for (int gq = 0; gq < G; ++gq) {
-                    int cnt = 0, arg = 0x7fffffff;
-                    float best = -INFINITY;
+                    uint32_t key = 0;                 // 0: no record of the window in this lane
+                    int arg = 0x7fffffff;
 #pragma unroll
                     for (int half = 0; half < SEG / 32; ++half) {
                         const int rec = half * 32 + lane;
                         if (rec < nwin) {
-                            cnt += (m[half] >> gq) & 1;
-                            const float bd = (dense || !ok) ? 0.f : sbound[rec][gq];
-                            if (bd > best) { best = bd; arg = rec; }
+                            const float bd = ((dense || !ok) ? 0.f : sbound[rec][gq]) + 0.f;        // (-0 counts as +0)
+                            const uint32_t u = __float_as_uint(bd);
+                            uint32_t k2 = (u & 0x80000000u) ? ~u : (u | 0x80000000u);           // ascending with the value
+                            if (bd != bd) k2 = 1;                                               // a NaN bound never wins
+                            if (k2 > key) { key = k2; arg = rec; }                              // ties keep the lower index
                         }
                     }
-#pragma unroll
-                    for (int s = 16; s >= 1; s >>= 1) {
-                        cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
-                        const float ob = __shfl_xor_sync(0xffffffffu, best, s);
-                        const int oa = __shfl_xor_sync(0xffffffffu, arg, s);
-                        if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
-                    }
+                    const int cnt = __popc(__ballot_sync(0xffffffffu, (m[0] >> gq) & 1 && lane < nwin)) +
+                                    __popc(__ballot_sync(0xffffffffu, (m[1] >> gq) & 1 && lane + 32 < nwin));
+                    const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+                    // among the lanes that hold the maximum the lowest record index wins: a lane's own candidate is its
+                    // lower record unless the higher one is strictly larger, so compare the candidates' indices
+                    const int amin = __reduce_min_sync(0xffffffffu, key == kmax ? arg : 0x7fffffff);
                     if (lane == 0) {
                         RescueRec rr;
-                        rr.cnt = cnt; rr.maxb = best; rr.arg = (arg == 0x7fffffff) ? -1 : (j0 + arg); rr.pad = 0;
+                        float best = -INFINITY;
+                        if (kmax > 1) {
+                            const uint32_t u = (kmax & 0x80000000u) ? (kmax & 0x7fffffffu) : ~kmax;
+                            best = __uint_as_float(u);
+                        }
+                        rr.cnt = cnt; rr.maxb = best;
+                        rr.arg = (kmax <= 1 || amin == 0x7fffffff) ? -1 : (j0 + amin);
+                        rr.pad = 0;
                         a.seg_resc[((int64_t)r * a.nseg + seg) * G + gq] = rr;
                     }
                 }
