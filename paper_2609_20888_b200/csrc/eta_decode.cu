@@ -3,22 +3,30 @@
 // GQA-grouped execution of the fused-kernel appendix, and the associative
 // (m, l, O) merge of its "two-stage reduction".
 //
-// Work is the flattened sequence of "units" the plan step laid out: for each
-// (sequence, KV head) row its surviving blocks, then its tail.  Every CTA owns an
-// equal, contiguous share of that sequence, so the load is balanced whatever the
-// per-head survivor counts are; a share may cross rows, and a row may be split
-// over CTAs; each (CTA, row) piece produces one partial (m, l, O) per query head.
+// decode_kernel is persistent, one CTA per SM.  Work is the flattened sequence
+// of "units": for each (sequence, KV head) row its surviving blocks (the
+// screening kernel's per-segment lists), then its rescued blocks, then its tail.
+// Every CTA lays that sequence out for itself from the per-segment counts and
+// takes an equal, contiguous share of its COST (units, plus a fixed charge for
+// every row boundary inside the share: stream-K), so the load is balanced
+// whatever the per-head survivor counts are; a share may cross rows, and a row
+// may be split over CTAs; each (CTA, row) piece produces one partial (m, l, O)
+// per query head and consumer group.
 //
 // Inside a CTA one producer warp walks the survivor lists and issues tiled TMA
-// copies (128-byte swizzle) of K and V tiles into a ring of shared-memory stages;
-// four consumer warps each take a quarter of the tokens of every tile.  The G
-// query heads of the group are packed on the M side of mma.m16n8k16 (bf16 in,
-// fp32 out), tokens on N, so each K/V byte is read once from HBM and once from
-// shared memory for all heads.  The head_dim and token orders fed to the MMAs are
-// permuted (a dot product does not care) so that every shared-memory read is a
-// conflict-free 16-byte load of the swizzled tile.  Softmax statistics and
-// accumulators are fp32; P is fed to the second MMA as a bf16 high part plus a
-// bf16 residual, so the product keeps fp32-level accuracy.
+// copies (5-D tensor maps, 128-byte swizzle) of K and V tiles into a ring of
+// shared-memory stages; three consumer groups of four warps take the fills in
+// rotation, each warp a quarter of a tile's tokens.  The G query heads of the
+// group are packed on the M side of mma.m16n8k16 (bf16 in, fp32 out), tokens on
+// N, so each K/V byte is read once from HBM and once from shared memory for all
+// heads.  The head_dim and token orders fed to the MMAs are permuted (a dot
+// product does not care) so that every shared-memory read is a conflict-free
+// 16-byte load of the swizzled tile.  Softmax statistics and accumulators are
+// fp32; P is fed to the second MMA as a bf16 high part plus a bf16 residual, so
+// the product keeps fp32-level accuracy.  Every wait is bounded.
+//
+// merge_kernel folds the partials of a (row, head) in a fixed order: a CTA per
+// (row, head, slice of head_dim).
 #include <cuda.h>
 
 #include "eta_common.cuh"
