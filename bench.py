@@ -45,9 +45,13 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC = os.path.join(ROOT, "profiles", "decode_kernel_dram_traffic.json")
 
 
-def ncu_traffic(name: str, target: float):
+def ncu_traffic(name: str, target: float, algorithmic_bytes: float):
+    """DRAM traffic per launch of the streaming kernel for this run: what ncu counted on a captured run of the same
+    workload, scaled by the algorithmic bytes (the union of surviving blocks, hence the bytes, changes with the
+    step's query; traffic grows in proportion)."""
     try:
-        return float(json.load(open(NCU_TRAFFIC))[f"{name}@{target:.2f}"]["dram_bytes_per_launch"])
+        e = json.load(open(NCU_TRAFFIC))[f"{name}@{target:.2f}"]
+        return float(e["dram_bytes_per_launch"]) * algorithmic_bytes / float(e["algorithmic_bytes_of_captured_run"])
     except Exception:
         return None
 
@@ -505,7 +509,8 @@ def run_ours(args):
             "gpu_launches": args.steps * (2 + eb.eta_decode_kernel_count()),
             "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": ncu_traffic(sp.name, main_target), "traffic_unit": "bytes per launch",
+                         "traffic": ncu_traffic(sp.name, main_target, ab["decode"]),
+                         "traffic_unit": "bytes per launch (ncu capture of this workload, scaled by the algorithmic bytes of this run)",
                          "algorithmic_bytes_per_launch": ab["decode"]},
             "prefill_build": {"ms": build_ms, "gbs": k_bytes / (build_ms * 1e-3) / 1e9},
             "calibration": cal,
