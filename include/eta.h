@@ -310,8 +310,9 @@ int eta_decode_kernel_count(void);
  * eta_profile_read waits for the most recent eta_decode to finish and writes the time from each launch to the
  * next, in milliseconds, to ms[0 .. count-1] (n >= 5), in the order append, predict, screen, decode, merge,
  * returning the count, or a negative status when no profiled eta_decode has run.  The first two are 0
- * unless those calls were made, in that order, right before the eta_decode.  Not thread-safe; leave disabled
- * in production.
+ * unless those calls were made, in that order, right before the eta_decode.  Process-wide state (one set of
+ * events, created on the device that is current at the first mark; calls are serialised by a lock): for one
+ * measuring thread on one device; leave disabled in production.
  */
 int eta_profile_enable(int on);
 int eta_profile_read(float* ms, int n);

@@ -40,6 +40,7 @@ int validate_desc(const eta_cache_desc* d) {
 // (append, predict, then the three kernels of eta_decode).  Event k is recorded just before launch k; event 5
 // after the last launch.
 constexpr int N_MARKS = 6;
+static std::mutex g_profile_mutex;       // the marks are process-wide state: serialised, meant for one measuring thread
 static bool g_profile = false;
 static cudaEvent_t g_ev[N_MARKS];
 static bool g_ev_made = false;
@@ -47,6 +48,7 @@ static unsigned g_ev_seen = 0;
 
 void profile_mark(int k, cudaStream_t s) {
     if (!g_profile) return;
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
     if (!g_ev_made) {
         for (int i = 0; i < N_MARKS; ++i) cudaEventCreate(&g_ev[i]);
         g_ev_made = true;
@@ -203,6 +205,7 @@ int eta_set_pdl(int on) {
 }
 
 int eta_profile_enable(int on) {
+    std::lock_guard<std::mutex> lock(eta::g_profile_mutex);
     if (on && !eta::g_profile) eta::g_ev_seen = 0;     // a new profiled run starts; a finished one stays readable
     eta::g_profile = on != 0;
     return ETA_OK;
@@ -211,6 +214,7 @@ int eta_profile_enable(int on) {
 int eta_profile_read(float* ms, int n) {
     using namespace eta;
     if (!ms || n < N_MARKS - 1) return ETA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
     if ((g_ev_seen & 0x3c) != 0x3c) return ETA_ERR_INVALID_ARG;      // no profiled eta_decode yet
     cudaError_t e = cudaEventSynchronize(g_ev[5]);
     for (int k = 0; k < N_MARKS - 1 && e == cudaSuccess; ++k) {

@@ -76,7 +76,7 @@ struct FastDiv {
 
 
 
-// Arguments of the screening and planning kernels (defined in eta_screen.cu, launched from eta_decode).
+// Arguments of the screening kernel (defined in eta_screen.cu, launched from eta_decode).
 struct ScreenArgs {
     const __nv_bfloat16* q;
     const __half* musig;
