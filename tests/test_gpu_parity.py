@@ -293,6 +293,44 @@ def test_plus_infinite_threshold_attends_rescue_pins_and_tail_only():
         assert cnt == sp.batch * sp.n_q_heads * lwb + expect_rescues
 
 
+def test_rescue_window_longer_than_four_segments_and_many_segment_counts():
+    """Two loops of the streaming kernel's set-up that ordinary shapes do not enter: a rescue window of more than
+    4 x 64 blocks (its statistics are then combined in rounds of four segments), and more segment counts than one
+    pass of the set-up loads (8 per thread x 416 threads = 3328; here 64 rows x 56 segments = 3584)."""
+    _eb()
+    d, b, B, Hkv, G = 64, 32, 8, 8, 1
+    T = 32 * 64 * 56
+    rng, K, V, lens = _rand_cache_t(77, B, Hkv, [T] * B, d, b)
+    lens = lens.copy()
+    lens[1] = T - 5 * b - 3                     # a shorter row with a tail, so that rows differ
+    q = torch.from_numpy(rng.standard_normal((B, Hkv * G, d))).to(torch.bfloat16)
+    c = orc.Cache(bits(K), bits(V), lens, b)
+    musig, mnorm = orc.block_summaries(c)
+    bound = orc.score_dual(bits(q), musig, mnorm, lens, b, 1.0)
+    # (a) a threshold nothing passes, the whole sequence as rescue window: the global argmax of 3584 bounds per head
+    inf = np.full((B, Hkv * G), np.inf, np.float32)
+    ref = orc.decode_step(bits(q), c, musig, mnorm, tau=inf, rescue_window=1 << 30)
+    out, sel, stats, status = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=inf, rescue_window=1 << 30)
+    assert status == 0
+    assert np.array_equal(sel, ref["sel"])
+    first = np.array([[int(np.nanargmax(bound[i, h, :int(lens[i]) // b])) for h in range(Hkv * G)] for i in range(B)])
+    assert np.array_equal(ref["rescued"], first) and (first >= 4 * 64).any()
+    mx, mean = output_errors(out, ref["out"])
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+    # (b) an ordinary sparse step on the same shape
+    tau = (np.nanquantile(bound, 0.95, axis=2) + 1e-4).astype(np.float32)
+    ref = orc.decode_step(bits(q), c, musig, mnorm, tau=tau, rescue_window=1000)
+    out, sel, stats, status = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=tau, rescue_window=1000)
+    assert status == 0
+    near = compare_masks(sel, ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G, rescued=ref["rescued"])
+    keep = heads_without_near_tie(near, B, Hkv * G)
+    assert keep.mean() > 0.9
+    mx, mean = output_errors(out[keep], ref["out"][keep])
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+    union = np.array([[int((sel[i, hk, :int(lens[i]) // b] != 0).sum()) for hk in range(Hkv)] for i in range(B)])
+    assert np.array_equal(stats, union)
+
+
 EDGE = [
     dict(d=128, b=64, lens=[1]),                    # a single token: tail only
     dict(d=128, b=64, lens=[63, 64, 65]),           # just below / at / above one block
