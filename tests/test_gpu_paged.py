@@ -167,3 +167,71 @@ def test_paged_arguments_are_validated():
     ok = torch.zeros((1, 4), dtype=torch.int32, device=dev)
     with pytest.raises(eb.EtaError):
         eb.eta_build_block_summaries_paged(pdesc, eb.page_table(ok, 0), Kp, lens, musig, mnorm)
+
+
+def test_shared_prefix_batch_whose_counts_do_not_fit_the_set_up_buffer():
+    """128 sequences that share one 311 K-token prefix through their page tables (1024 rows of 153 segments): the
+    streaming kernel's set-up cannot keep the per-segment counts of all rows in shared memory and reads them from
+    global memory window by window, and its row search runs over more than 32 rows.  The oracle is run on three
+    sampled sequences (each gathered into a contiguous cache of its own); every row is checked for the properties
+    that hold at any size (status, finite outputs, block counts equal to the mask's)."""
+    eb = _eb()
+    dev = torch.device("cuda:0")
+    B, Hkv, G, d, b = 128, 8, 1, 64, 32
+    nb_full = 152 * 64
+    t_cap = nb_full * b + b
+    rng = np.random.default_rng(4242)
+    K = torch.from_numpy(rng.standard_normal((1, Hkv, t_cap, d), dtype=np.float32)).to(torch.bfloat16)
+    V = torch.from_numpy(rng.standard_normal((1, Hkv, t_cap, d), dtype=np.float32)).to(torch.bfloat16)
+    q = torch.from_numpy(rng.standard_normal((B, Hkv * G, d), dtype=np.float32)).to(torch.bfloat16)
+    lens = np.full(B, nb_full * b + 7, np.int32)
+    lens[77] = 5000 * b                        # a shorter sharer that ends on a block boundary
+    lens[127] = 9000 * b + 31
+    lens[3] = 11                               # and one that holds a tail only
+    Kp, Vp, table1, n_pages = _scatter(K, V, [t_cap], b, seed=5, layout="phbd")
+    table = table1.expand(B, -1).contiguous()
+    pdesc = eb.paged_cache_desc(Kp, Vp, B, Hkv * G, t_cap=t_cap)
+    pages = eb.page_table(table, n_pages)
+    # the oracle's summaries of the shared prefix, the same bytes for every sharer
+    c1 = orc.Cache(bits(K), bits(V), np.asarray([t_cap], np.int32), b)
+    o_musig, o_mnorm = orc.block_summaries(c1)
+    musig, mnorm = eb.alloc_summaries(pdesc, dev)
+    musig.copy_(torch.from_numpy(o_musig.view(np.int16)).view(torch.float16).to(dev).expand_as(musig))
+    mnorm.copy_(torch.from_numpy(o_mnorm).to(dev).expand_as(mnorm))
+    lens_d = torch.from_numpy(lens).to(dev)
+    qd = q.to(dev)
+    params = eb.DecodeParams(z=1.0, beta=5.0, lwb=1, rescue_window=128)
+    bound = torch.full((B, Hkv * G, pdesc.nb_cap), float("nan"), dtype=torch.float32, device=dev)
+    eb.eta_score_dual(pdesc, params, qd, lens_d, musig, mnorm, bound)
+    tau = torch.nan_to_num(torch.nanquantile(bound, 0.97, dim=2), nan=0.0).add_(3e-4).contiguous()
+    del bound
+    out = torch.full((B, Hkv * G, d), float("nan"), dtype=torch.float32, device=dev)
+    sel = torch.zeros((B, Hkv, pdesc.nb_cap), dtype=torch.uint8, device=dev)
+    stats = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    nws = eb.eta_workspace_bytes(pdesc)
+    ws = torch.zeros(nws + 256, dtype=torch.uint8, device=dev)
+    off = (-ws.data_ptr()) % 256
+    ws = ws[off:off + nws]
+    eb.eta_decode_paged(pdesc, pages, params, qd, Kp, Vp, lens_d, musig, mnorm, tau, None, out, sel, ws,
+                        stats=stats, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    out_np, sel_np, stats_np, tau_np = out.cpu().numpy(), sel.cpu().numpy(), stats.cpu().numpy(), tau.cpu().numpy()
+    assert np.isfinite(out_np).all()
+    for i in range(B):
+        NB = int(lens[i]) // b
+        assert np.array_equal(stats_np[i], (sel_np[i, :, :NB] != 0).sum(axis=1))
+        assert not sel_np[i, :, NB:].any()
+    assert 0.01 < stats_np.sum() / ((lens // b).sum() * Hkv) < 0.10
+    for i in (0, 77, 127, 3):
+        T = int(lens[i])
+        ci = orc.Cache(bits(K), bits(V), np.asarray([T], np.int32), b)
+        ref = orc.decode_step(bits(q[i:i + 1]), ci, o_musig, o_mnorm, tau=tau_np[i:i + 1], z=1.0, beta=5.0, lwb=1,
+                              rescue_window=128)
+        near = compare_masks(sel_np[i:i + 1], ref["sel"], ref["bound"], tau_np[i:i + 1].astype(np.float64),
+                             np.asarray([T], np.int32), b, G, rescued=ref["rescued"])
+        keep = heads_without_near_tie(near, 1, Hkv * G)
+        assert keep.mean() >= 0.75
+        mx, mean = output_errors(out_np[i:i + 1][keep], ref["out"][keep])
+        assert mx <= 1e-2 and mean <= 1e-3, (i, mx, mean)
