@@ -200,3 +200,54 @@ def test_c5_frozen_constants_vs_predicted_thresholds_mixed_lengths():
     rf = s.decode_and_check(0, musig, mnorm, head_const=consts)
     rp = s.decode_and_check(0, musig, mnorm, bias=_bias("c5_frozen", 0.70))
     print("c5 frozen", rf, "predicted", rp)
+
+
+def test_one_sequence_of_seventeen_million_tokens():
+    """A single KV head of 17.8 M tokens (4.6 GB per tensor, 139 264 blocks of 128 tokens, 2177 segments): element
+    offsets inside K and V pass 2^31, a row's block lists are far longer than any other test's.  Full comparison with
+    the oracle: the summary build, the masks, the block count and all eight heads' outputs."""
+    eb = _eb()
+    dev = torch.device("cuda:0")
+    B, Hkv, G, d, b = 1, 1, 8, 128, 128
+    T = 17 * (1 << 20) + 77
+    t_cap = ((T + b - 1) // b) * b
+    gen = torch.Generator().manual_seed(20888)
+    K = torch.empty((B, Hkv, t_cap, d), dtype=torch.bfloat16)
+    V = torch.empty((B, Hkv, t_cap, d), dtype=torch.bfloat16)
+    step = 1 << 20
+    for t0 in range(0, t_cap, step):                          # drawn in chunks: the fp32 draws never exist all at once
+        n = min(step, t_cap - t0)
+        K[0, 0, t0:t0 + n] = torch.randn((n, d), generator=gen).to(torch.bfloat16)
+        V[0, 0, t0:t0 + n] = torch.randn((n, d), generator=gen).to(torch.bfloat16)
+    q = torch.randn((B, Hkv * G, d), generator=gen).to(torch.bfloat16)
+    lens = np.asarray([T], np.int32)
+    c = orc.Cache(bits(K), bits(V), lens, b)
+    musig, mnorm = orc.block_summaries(c)
+    NB = T // b
+    # summary build on the device
+    Kd, Vd = K.to(dev), V.to(dev)
+    st = eb.DecodeState(Kd, Vd, Hkv * G, b)
+    lens_d = torch.from_numpy(lens).to(dev)
+    eb.eta_build_block_summaries(st.desc, Kd, lens_d, st.musig, st.mnorm)
+    torch.cuda.synchronize()
+    assert fp16_ulp_distance(bits(st.musig.cpu())[0, :, :NB], musig[0, :, :NB]).max() <= 1
+    assert np.abs(st.mnorm.cpu().numpy()[0, :, :NB].view(np.int32) - mnorm[0, :, :NB].view(np.int32)).max() <= 4
+    # decode on the oracle's summary bytes, thresholds that keep about one block in 200 per head
+    bound = orc.score_dual(bits(q), musig, mnorm, lens, b, 1.0)
+    tau = (np.nanquantile(bound, 0.995, axis=2) + 3e-4).astype(np.float32)
+    ref = orc.decode_step(bits(q), c, musig, mnorm, tau=tau, lwb=2, rescue_window=128)
+    st.musig.copy_(torch.from_numpy(musig.view(np.int16)).view(torch.float16).to(dev))
+    st.mnorm.copy_(torch.from_numpy(mnorm).to(dev))
+    st.out.fill_(float("nan"))
+    eb.eta_decode(st.desc, eb.DecodeParams(lwb=2, rescue_window=128), q.to(dev), Kd, Vd, lens_d, st.musig, st.mnorm,
+                  torch.from_numpy(tau).to(dev), None, st.out, st.sel_mask, st.workspace, stats=st.stats, status=st.status)
+    torch.cuda.synchronize()
+    assert int(st.status.item()) == 0
+    sel, out = st.sel_mask.cpu().numpy(), st.out.cpu().numpy()
+    near = compare_masks(sel, ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G, rescued=ref["rescued"])
+    keep = heads_without_near_tie(near, B, Hkv * G)
+    assert keep.mean() >= 0.75
+    mx, mean = output_errors(out[keep], ref["out"][keep])
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+    assert int(st.stats.sum().item()) == int((sel[0, 0, :NB] != 0).sum())
+    assert 0.005 < st.stats.sum().item() / NB < 0.10
