@@ -105,3 +105,33 @@ def test_random_configuration_matches_the_oracle(seed):
         assert status == 0
         mx, mean = output_errors(out_d, dense)
         assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+
+
+@pytest.mark.parametrize("B,Hkv,G,d,b,longest", [(1024, 1, 4, 128, 64, 600), (256, 4, 2, 64, 32, 3000),
+                                                  (512, 2, 8, 128, 128, 1000)])
+def test_many_short_sequences_up_to_the_row_limit(B, Hkv, G, d, b, longest):
+    """Up to 1024 (sequence, KV head) rows of 1 .. `longest` tokens: far more rows than streaming CTAs, most pieces a
+    tile or two, many rows with a tail only."""
+    _build()
+    rng = np.random.default_rng(B)
+    lens = rng.integers(1, longest, size=B).astype(np.int32)
+    t_cap = ((int(lens.max()) + b - 1) // b) * b
+    K = torch.from_numpy(rng.standard_normal((B, Hkv, t_cap, d), dtype=np.float32)).to(torch.bfloat16)
+    V = torch.from_numpy(rng.standard_normal((B, Hkv, t_cap, d), dtype=np.float32)).to(torch.bfloat16)
+    q = torch.from_numpy(rng.standard_normal((B, Hkv * G, d), dtype=np.float32)).to(torch.bfloat16)
+    c = orc.Cache(bits(K), bits(V), lens, b)
+    musig, mnorm = orc.block_summaries(c)
+    bound = orc.score_dual(bits(q), musig, mnorm, lens, b, 1.0)
+    with np.errstate(all="ignore"), warnings.catch_warnings():
+        warnings.simplefilter("ignore")
+        tau = (np.nan_to_num(np.nanquantile(bound, 0.7, axis=2), nan=0.0) + 3e-4).astype(np.float32)
+    ref = orc.decode_step(bits(q), c, musig, mnorm, tau=tau, lwb=1, rescue_window=4)
+    out, sel, stats, status = gpu_decode(q, K, V, lens, b, musig, mnorm, tau=tau, lwb=1, rescue_window=4)
+    assert status == 0 and not np.isnan(out).any()
+    near = compare_masks(sel, ref["sel"], ref["bound"], tau.astype(np.float64), lens, b, G, rescued=ref["rescued"])
+    keep = heads_without_near_tie(near, B, Hkv * G)
+    assert keep.mean() > 0.95
+    mx, mean = output_errors(out[keep], ref["out"][keep])
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+    union = np.array([[int((sel[i, hk, :int(lens[i]) // b] != 0).sum()) for hk in range(Hkv)] for i in range(B)])
+    assert np.array_equal(stats, union)
