@@ -211,12 +211,12 @@ __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-// 4-D tiled copy global -> shared through a tensor map (no multicast).
+// 4-D tiled copy global -> shared through a tensor map, into this CTA's shared memory only.
 __device__ __forceinline__ void tma_load_4d(void* dst, const void* tmap, int x, int y, int z, int w, uint64_t* bar) {
     asm volatile("cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
                  ::"r"(smem_u32(dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
-// 5-D tiled copy (no multicast): used with the head_dim split into 64-column halves as an extra dimension, so one
+// 5-D tiled copy (this CTA's shared memory only): used with the head_dim split into 64-column halves as an extra dimension, so one
 // instruction brings both swizzled half tiles of a K or V tile.
 __device__ __forceinline__ void tma_load_5d(void* dst, const void* tmap, int c0, int c1, int c2, int c3, int c4,
                                             uint64_t* bar) {
